@@ -1,0 +1,202 @@
+/*
+ * dsbd.h -- C ABI of the B200 (sm_100a) hot path of dynamic-width speculative beam decoding:
+ * the per-step parallel verification of a forest of draft trees, one tree per input beam.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless a comment says "host".  The structs themselves
+ *     (dsbd_forest_t, ...) live in host memory and are read during the call only.
+ *   - The library never allocates, frees or synchronises: the caller owns every buffer,
+ *     passes a workspace of at least the size the matching *_workspace() query returns, and
+ *     every call is asynchronous on `stream`.  Workspaces may be reused by the next call on
+ *     the same stream; their contents are undefined afterwards.
+ *   - Return value: DSBD_OK, or a negative DSBD_ERR_* found by host-side checks (nothing was
+ *     launched).  Problems only the device can see (a draft token outside the vocabulary, a
+ *     distribution without mass, a bounded wait that ran out) are written to `*status`
+ *     (device int32, must be zero before the call, first error wins) and, per request, to
+ *     `req_error`; kernels never trap.
+ *   - There is no CPU fallback and no global state; the same inputs and (seed, step) give the
+ *     same outputs whatever the launch shape.
+ */
+#ifndef DSBD_H
+#define DSBD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *dsbd_stream_t;   /* a cudaStream_t */
+
+enum {
+    DSBD_OK = 0,
+    DSBD_ERR_INVALID_ARG = -1,
+    DSBD_ERR_UNSUPPORTED = -2,
+    DSBD_ERR_WORKSPACE_TOO_SMALL = -3,
+    DSBD_ERR_CUDA = -4
+};
+
+/* device-side codes written to *status / req_error */
+enum {
+    DSBD_DEV_BAD_TOKEN = 1,      /* draft token outside [0, V)                               */
+    DSBD_DEV_EXHAUSTED = 2,      /* a draw from a distribution without mass, or a rejection
+                                    that had probability zero                                */
+    DSBD_DEV_CAPACITY = 3,       /* more output beams than the request's out_off range holds */
+    DSBD_DEV_BAD_FOREST = 4,     /* parent index outside its tree, too many live beams/drafts */
+    DSBD_DEV_TIMEOUT = 5         /* a bounded wait gave up                                   */
+};
+
+/* limits of this build */
+#define DSBD_MAX_TREE_NODES 64   /* nodes per draft tree (forest attention)                  */
+#define DSBD_MAX_LIVE 64         /* beams of a request / live drafts of a layer (verify)     */
+
+/* The draft forest of one decode step (Section "Draft and Verification Scheme", Overview):
+ * B trees, one per input beam, grouped by request; tree b owns the nodes
+ * [beam_node_off[b], beam_node_off[b+1]), its root (the input beam itself) first, and every
+ * other node n has beam_node_off[b] <= parent[n] < n.  Depth d nodes are the drafts of
+ * draft layer d; max_depth is gamma, the number of draft layers. */
+typedef struct {
+    int32_t R, B, N, max_depth;
+    const int32_t *req_beam_off;   /* [R+1] trees of request r                               */
+    const int32_t *beam_node_off;  /* [B+1]                                                  */
+    const int32_t *parent;         /* [N]   global node id, -1 for a root                    */
+    const int32_t *token;          /* [N]   draft token id (ignored for roots)               */
+    const int32_t *draft_rank;     /* [N] or NULL: position of the node in the order in which
+                                      the small model drew the drafts of its layer; the accept
+                                      loop walks a layer by (draft_rank, node id).  The drafts
+                                      must be tested in an order that does not depend on their
+                                      values, so a forest whose node numbering is not the draw
+                                      order has to pass it.  NULL = ascending node id.       */
+    /* host-side facts about the arrays above; they size launches and are trusted */
+    int32_t max_tree_nodes;        /* max_b nodes of tree b, <= DSBD_MAX_TREE_NODES for
+                                      dsbd_forest_attention                                  */
+    int32_t max_req_beams;         /* max_r trees of request r, <= DSBD_MAX_LIVE             */
+    int32_t max_layer_nodes;       /* max over (request, depth >= 1) of the nodes at that
+                                      depth, <= DSBD_MAX_LIVE                                */
+} dsbd_forest_t;
+
+enum { DSBD_DTYPE_BF16 = 0, DSBD_DTYPE_F32 = 1 };
+
+/* Shapes of the forest attention (Section "Forest-based Parallel Decoding").
+ * Layouts, all contiguous:  q, out [N, Hq, d];  k_new, v_new [N, Hkv, d] (keys/values of the
+ * forest nodes themselves);  k_prefix, v_prefix: the KV cache of each input beam packed
+ * beam after beam, beam b as [Hkv, L_b, d] starting at element prefix_off[b]*Hkv*d, where
+ * L_b = prefix_off[b+1]-prefix_off[b] tokens (the cache excludes the root token).  Query
+ * head h uses KV head h / (Hq/Hkv).  All tensors share `dtype`; accumulation is fp32. */
+typedef struct {
+    int32_t Hq, Hkv, d;            /* d in {64, 128}; Hq % Hkv == 0                          */
+    int32_t dtype;                 /* DSBD_DTYPE_*                                           */
+    float scale;                   /* softmax scale, usually 1/sqrt(d)                       */
+    int64_t total_prefix;          /* host copy of prefix_off[B]                             */
+    int64_t max_prefix;            /* host: max_b L_b                                        */
+} dsbd_attn_desc_t;
+
+/* Forest-masked attention: for every node n and query head h,
+ *   out[n,h] = sum_j softmax_j(scale * q[n,h] . K_j) V_j
+ * over j in (KV prefix of n's beam) U (ancestors of n in its own tree) U {n}; nothing of any
+ * other tree or beam is visible ("topology-aware mask" extended from one tree to a forest,
+ * with a separate KV cache per input beam).  prefix_off: [B+1] int64, tokens.
+ * Errors: INVALID_ARG (null pointer, Hq % Hkv), UNSUPPORTED (d, dtype, tree larger than
+ * DSBD_MAX_TREE_NODES, pointers not 16-byte aligned), WORKSPACE_TOO_SMALL. */
+int dsbd_forest_attention(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
+                          const void *q, const void *k_new, const void *v_new,
+                          const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
+                          void *out, void *workspace, size_t workspace_bytes, int32_t *status,
+                          dsbd_stream_t stream);
+
+size_t dsbd_forest_attention_workspace(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc);
+
+/* Parameters of the verification (Section "Details", Algorithm 1, and Section
+ * "Dynamic-Width Speculative Beam Decoding"). */
+typedef struct {
+    int32_t V;                     /* vocabulary size                                        */
+    float temperature;             /* tau > 0: both models' logits are divided by it before
+                                      the per-node softmax                                   */
+    float thresh;                  /* threshold t of the width rule                          */
+    int32_t W_min, W_max, W_nom;   /* W_L^(l) = min(W_max, max(W_min, W~_L^(l)(t)));  W_nom is
+                                      the width of the extra layer sampled when all gamma
+                                      layers pass.  W_max = number of drafts gives the
+                                      paper's uncapped rule.                                 */
+    const int32_t *W_min_r;        /* optional per-request overrides, [R] each, or NULL      */
+    const int32_t *W_max_r;
+    const int32_t *W_nom_r;
+    uint64_t seed;                 /* Philox4x32-10 key                                      */
+    uint64_t step;                 /* decode-step counter, mixed into the Philox counter     */
+} dsbd_verify_params_t;
+
+/* node_status */
+enum { DSBD_NODE_UNREACHED = 0, DSBD_NODE_ACCEPTED = 1, DSBD_NODE_REJECTED = 2,
+       DSBD_NODE_CUT = 3, DSBD_NODE_PRUNED = 4 };
+/* out_source */
+enum { DSBD_SRC_DRAFT = 0, DSBD_SRC_RESIDUAL = 1, DSBD_SRC_FILL = 2, DSBD_SRC_EXTRA = 3 };
+
+/* Results of dsbd_verify_step.  Request r writes its output beams to the slots
+ * [out_off[r], out_off[r] + out_width[r]); the range must hold
+ * max(W_nom, W_min, min(W_max, nodes of the request)) slots. */
+typedef struct {
+    int32_t *l_last;        /* [R]  layer whose beams are returned: the first short layer, or
+                                    gamma+1 when every layer passed                          */
+    int32_t *out_width;     /* [R]  number of output beams                                   */
+    const int32_t *out_off; /* [R+1]                                                         */
+    int32_t *out_parent;    /* node the output beam extends                                  */
+    int32_t *out_node;      /* the draft node it is, or -1 if it was sampled                 */
+    int32_t *out_root_beam; /* input beam (tree) it descends from -> which KV cache to keep  */
+    int32_t *out_token;
+    float   *out_logp;      /* cumulative log-prob of the new beam under p and under q       */
+    float   *out_logq;
+    int32_t *out_source;    /* DSBD_SRC_*                                                    */
+    int8_t  *node_status;   /* [N]  DSBD_NODE_*                                              */
+    int32_t *layer_width;   /* [R*(gamma+1)] width chosen per layer, -1 where not run        */
+    float   *node_logp;     /* [N]  cumulative log-prob of every node under p and q          */
+    float   *node_logq;
+    float   *lse_p;         /* [N]  log-sum-exp of each tempered logits row                  */
+    float   *lse_q;
+    int32_t *req_error;     /* [R]  0 or a DSBD_DEV_* code                                   */
+} dsbd_verify_out_t;
+
+/* One verification step (Algorithm 1 with the dynamic width of Eqs. for P, P~, alpha_j, W_L):
+ *   1. for every node and both models: log-sum-exp of the tempered logits row, the log-prob
+ *      of each draft token given its parent, cumulative beam scores (roots: root_logp/q);
+ *   2. per request, layer by layer: live drafts = depth-l nodes whose parent was accepted;
+ *      p_beam, q_beam = joint over (accepted parents x V), Eq. 1; width W_L^(l) from the
+ *      acceptance-count recursion; drafts accepted with probability min(1, p'/q_beam) (the
+ *      direction the proof of Theorem 1 and the alpha_j formula use), p' reset to p_beam on an
+ *      accept and replaced by norm(max(0, p' - q_beam)) on a reject; stop at W_L^(l) accepts;
+ *   3. a layer with fewer accepts is completed by one draw from p' and draws from p_beam and
+ *      ends the step; if all gamma layers pass, W_nom beams are drawn from p_beam^(gamma+1).
+ * logits_p, logits_q: [N, row_stride] fp32, row n = next-token logits after node n of the
+ * large / small model (row_stride >= V, in elements; rows 16-byte aligned run fastest).
+ * root_logp, root_logq: [B] cumulative log-probs of the input beams.
+ * Randomness: Philox4x32-10, key (seed lo, seed hi ^ step hi), counter (index, layer*4+purpose,
+ * request, step lo), purpose 0 accept test of the index-th live draft, 1 residual draw,
+ * 2 index-th p_beam fill, 3 index-th extra-layer draw; u = ((word0 >> 8) + 0.5) * 2^-24.
+ * Draws are inverse-CDF over (live parent ascending, token ascending). */
+int dsbd_verify_step(const dsbd_forest_t *forest, const dsbd_verify_params_t *params,
+                     const float *logits_p, const float *logits_q, int64_t row_stride,
+                     const float *root_logp, const float *root_logq,
+                     const dsbd_verify_out_t *out, void *workspace, size_t workspace_bytes,
+                     int32_t *status, dsbd_stream_t stream);
+
+size_t dsbd_verify_workspace(const dsbd_forest_t *forest, const dsbd_verify_params_t *params);
+
+/* The context-dependent width of ONE layer (Eqs. for P(m,k), P~(m,i), alpha_j and
+ * W_L^(l) = max(W_min, W~_L^(l)(t)), capped by W_max) for a given live set: request r's live
+ * parents are live_nodes[live_off[r] .. live_off[r+1]) (ascending node ids) with cumulative
+ * scores node_logp/node_logq (indexed by node id), and m[r] live drafts follow them.
+ * Outputs: width[r]; optionally alpha[r*out_stride + j] = alpha_{j+1} (j < m[r]) and
+ * tail[r*out_stride + K] = P(at least K accepts), K <= m[r]; out_stride >= max m + 1. */
+int dsbd_select_width(const dsbd_forest_t *forest, const dsbd_verify_params_t *params,
+                      const float *logits_p, const float *logits_q, int64_t row_stride,
+                      const float *node_logp, const float *node_logq,
+                      const int32_t *live_off, const int32_t *live_nodes, const int32_t *m,
+                      int32_t *width, float *alpha, float *tail, int32_t out_stride,
+                      void *workspace, size_t workspace_bytes, int32_t *status,
+                      dsbd_stream_t stream);
+
+const char *dsbd_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

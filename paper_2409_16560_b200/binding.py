@@ -1,0 +1,304 @@
+"""ctypes binding of libdsbd.so: argument marshalling only.
+
+Every step of the hot path runs in the CUDA library; this module turns torch tensors into the
+device pointers of the C ABI declared in ``include/dsbd.h`` and checks return codes.  There is
+no CPU fallback: without the built library, or without a CUDA device, calls raise.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+OK = 0
+DTYPE_BF16, DTYPE_F32 = 0, 1
+NODE_UNREACHED, NODE_ACCEPTED, NODE_REJECTED, NODE_CUT, NODE_PRUNED = 0, 1, 2, 3, 4
+SRC_DRAFT, SRC_RESIDUAL, SRC_FILL, SRC_EXTRA = 0, 1, 2, 3
+MAX_TREE_NODES = 64
+MAX_LIVE = 64
+
+EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_verify_step",
+           "dsbd_verify_workspace", "dsbd_select_width", "dsbd_status_string"]
+
+_vp = C.c_void_p
+
+
+class ForestT(C.Structure):
+    _fields_ = [("R", C.c_int32), ("B", C.c_int32), ("N", C.c_int32), ("max_depth", C.c_int32),
+                ("req_beam_off", _vp), ("beam_node_off", _vp), ("parent", _vp), ("token", _vp),
+                ("draft_rank", _vp),
+                ("max_tree_nodes", C.c_int32), ("max_req_beams", C.c_int32),
+                ("max_layer_nodes", C.c_int32)]
+
+
+class AttnDescT(C.Structure):
+    _fields_ = [("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32), ("dtype", C.c_int32),
+                ("scale", C.c_float), ("total_prefix", C.c_int64), ("max_prefix", C.c_int64)]
+
+
+class VerifyParamsT(C.Structure):
+    _fields_ = [("V", C.c_int32), ("temperature", C.c_float), ("thresh", C.c_float),
+                ("W_min", C.c_int32), ("W_max", C.c_int32), ("W_nom", C.c_int32),
+                ("W_min_r", _vp), ("W_max_r", _vp), ("W_nom_r", _vp),
+                ("seed", C.c_uint64), ("step", C.c_uint64)]
+
+
+_OUT_FIELDS = ["l_last", "out_width", "out_off", "out_parent", "out_node", "out_root_beam",
+               "out_token", "out_logp", "out_logq", "out_source", "node_status", "layer_width",
+               "node_logp", "node_logq", "lse_p", "lse_q", "req_error"]
+
+
+class VerifyOutT(C.Structure):
+    _fields_ = [(n, _vp) for n in _OUT_FIELDS]
+
+
+_lib = None
+
+
+def lib_path():
+    return _build.LIB_PATH
+
+
+def load():
+    """Load libdsbd.so (building it when a compiler is at hand and it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if not os.path.exists(path) or _build.stale():
+        path = _build.build()
+    lib = C.CDLL(path)
+    lib.dsbd_status_string.restype = C.c_char_p
+    lib.dsbd_status_string.argtypes = [C.c_int]
+    lib.dsbd_forest_attention_workspace.restype = C.c_size_t
+    lib.dsbd_forest_attention_workspace.argtypes = [_vp, _vp]
+    lib.dsbd_verify_workspace.restype = C.c_size_t
+    lib.dsbd_verify_workspace.argtypes = [_vp, _vp]
+    lib.dsbd_forest_attention.restype = C.c_int
+    lib.dsbd_forest_attention.argtypes = [_vp] * 10 + [C.c_size_t, _vp, _vp]
+    lib.dsbd_verify_step.restype = C.c_int
+    lib.dsbd_verify_step.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_size_t,
+                                     _vp, _vp]
+    lib.dsbd_select_width.restype = C.c_int
+    lib.dsbd_select_width.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, _vp,
+                                      _vp, _vp, C.c_int32, _vp, C.c_size_t, _vp, _vp]
+    _lib = lib
+    return lib
+
+
+def status_string(code):
+    return load().dsbd_status_string(int(code)).decode()
+
+
+class DsbdError(RuntimeError):
+    def __init__(self, where, code):
+        super().__init__("%s: %s (%d)" % (where, status_string(code), code))
+        self.code = code
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _require_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise RuntimeError("dsbd: device tensors required; there is no CPU path")
+
+
+class Forest:
+    """Device copy of a draft forest plus the host-side facts the launches are sized by."""
+
+    def __init__(self, arrays, device):
+        a = {k: np.ascontiguousarray(arrays[k], dtype=np.int32)
+             for k in ("req_beam_off", "beam_node_off", "parent", "token")}
+        self.R, self.B, self.N = (int(arrays[k]) for k in ("R", "B", "N"))
+        self.max_depth = int(arrays["max_depth"])
+        self.host = a
+        rank = arrays.get("draft_rank")
+        self.dev = {k: torch.from_numpy(v).to(device) for k, v in a.items()}
+        self.dev["draft_rank"] = (torch.from_numpy(np.ascontiguousarray(rank, dtype=np.int32)).to(device)
+                                  if rank is not None else None)
+        tree_sizes = np.diff(a["beam_node_off"])
+        self.max_tree_nodes = int(tree_sizes.max())
+        self.max_req_beams = int(np.diff(a["req_beam_off"]).max())
+        # nodes per (request, depth)
+        depth = np.zeros(self.N, np.int64)
+        for n, p in enumerate(a["parent"]):
+            depth[n] = 0 if p < 0 else depth[p] + 1
+        tree_of = np.repeat(np.arange(self.B), tree_sizes)
+        req_of = np.searchsorted(a["req_beam_off"], tree_of, side="right") - 1
+        nz = depth > 0
+        if nz.any():
+            key = req_of[nz] * (int(depth.max()) + 1) + depth[nz]
+            self.max_layer_nodes = int(np.bincount(key).max())
+        else:
+            self.max_layer_nodes = 0
+        self.depth = depth
+        self.tree_of = tree_of
+        self.req_of = req_of
+        self.device = device
+
+    def struct(self):
+        f = ForestT()
+        f.R, f.B, f.N, f.max_depth = self.R, self.B, self.N, self.max_depth
+        for k in ("req_beam_off", "beam_node_off", "parent", "token", "draft_rank"):
+            setattr(f, k, _ptr(self.dev[k]))
+        f.max_tree_nodes = self.max_tree_nodes
+        f.max_req_beams = self.max_req_beams
+        f.max_layer_nodes = self.max_layer_nodes
+        return f
+
+
+def _attn_desc(Hq, Hkv, d, dtype, scale, prefix_off_host):
+    desc = AttnDescT()
+    desc.Hq, desc.Hkv, desc.d = Hq, Hkv, d
+    desc.dtype = DTYPE_BF16 if dtype == torch.bfloat16 else DTYPE_F32
+    desc.scale = float(scale)
+    desc.total_prefix = int(prefix_off_host[-1])
+    desc.max_prefix = int(np.diff(prefix_off_host).max()) if len(prefix_off_host) > 1 else 0
+    return desc
+
+
+def forest_attention_workspace(forest, Hq, Hkv, d, dtype, scale, prefix_off_host):
+    f = forest.struct()
+    desc = _attn_desc(Hq, Hkv, d, dtype, scale, prefix_off_host)
+    return int(load().dsbd_forest_attention_workspace(C.addressof(f), C.addressof(desc)))
+
+
+def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_prefix, prefix_off,
+                     prefix_off_host, out=None, workspace=None, status=None, stream=None):
+    """dsbd_forest_attention; returns (out, status tensor)."""
+    _require_cuda(q, k_new, v_new, k_prefix, v_prefix, prefix_off)
+    assert q.dtype in (torch.bfloat16, torch.float32)
+    f = forest.struct()
+    desc = _attn_desc(Hq, Hkv, d, q.dtype, scale, prefix_off_host)
+    if out is None:
+        out = torch.empty_like(q)
+    need = int(load().dsbd_forest_attention_workspace(C.addressof(f), C.addressof(desc)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=q.device)
+    rc = load().dsbd_forest_attention(C.addressof(f), C.addressof(desc), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                      _ptr(k_prefix), _ptr(v_prefix), _ptr(prefix_off), _ptr(out),
+                                      _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_forest_attention", rc)
+    return out, status
+
+
+def _params(params, keep):
+    p = VerifyParamsT()
+    p.V = int(params["V"])
+    p.temperature = float(params.get("temperature", 1.0))
+    p.thresh = float(params.get("thresh", 0.7))
+    p.W_min = int(params.get("W_min", 1))
+    p.W_max = int(params.get("W_max", 1 << 30))
+    p.W_nom = int(params.get("W_nom", 1))
+    for name in ("W_min_r", "W_max_r", "W_nom_r"):
+        t = params.get(name)
+        if t is not None:
+            _require_cuda(t)
+            assert t.dtype == torch.int32
+            keep.append(t)
+            setattr(p, name, _ptr(t))
+    p.seed = int(params.get("seed", 0))
+    p.step = int(params.get("step", 0))
+    return p
+
+
+def verify_workspace(forest, params):
+    keep = []
+    f = forest.struct()
+    p = _params(params, keep)
+    return int(load().dsbd_verify_workspace(C.addressof(f), C.addressof(p)))
+
+
+def alloc_verify_out(forest, out_off_host, device):
+    """Output buffers of dsbd_verify_step as a dict of device tensors."""
+    R, N, g = forest.R, forest.N, forest.max_depth
+    S = int(out_off_host[-1])
+    i32, f32 = torch.int32, torch.float32
+    o = {
+        "l_last": torch.zeros(R, dtype=i32, device=device),
+        "out_width": torch.zeros(R, dtype=i32, device=device),
+        "out_off": torch.from_numpy(np.ascontiguousarray(out_off_host, dtype=np.int32)).to(device),
+        "out_parent": torch.full((S,), -1, dtype=i32, device=device),
+        "out_node": torch.full((S,), -1, dtype=i32, device=device),
+        "out_root_beam": torch.full((S,), -1, dtype=i32, device=device),
+        "out_token": torch.full((S,), -1, dtype=i32, device=device),
+        "out_logp": torch.zeros(S, dtype=f32, device=device),
+        "out_logq": torch.zeros(S, dtype=f32, device=device),
+        "out_source": torch.full((S,), -1, dtype=i32, device=device),
+        "node_status": torch.zeros(N, dtype=torch.int8, device=device),
+        "layer_width": torch.full((R * (g + 1),), -1, dtype=i32, device=device),
+        "node_logp": torch.zeros(N, dtype=f32, device=device),
+        "node_logq": torch.zeros(N, dtype=f32, device=device),
+        "lse_p": torch.zeros(N, dtype=f32, device=device),
+        "lse_q": torch.zeros(N, dtype=f32, device=device),
+        "req_error": torch.zeros(R, dtype=i32, device=device),
+    }
+    return o
+
+
+def verify_step(forest, params, logits_p, logits_q, root_logp, root_logq, out, workspace=None,
+                status=None, stream=None, row_stride=None):
+    """dsbd_verify_step; `out` from alloc_verify_out.  Returns the status tensor."""
+    _require_cuda(logits_p, logits_q, root_logp, root_logq)
+    assert logits_p.dtype == torch.float32 and logits_q.dtype == torch.float32
+    keep = []
+    f = forest.struct()
+    p = _params(params, keep)
+    o = VerifyOutT()
+    for name in _OUT_FIELDS:
+        setattr(o, name, _ptr(out[name]))
+    need = int(load().dsbd_verify_workspace(C.addressof(f), C.addressof(p)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=logits_p.device)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=logits_p.device)
+    stride = int(row_stride) if row_stride is not None else logits_p.stride(0)
+    rc = load().dsbd_verify_step(C.addressof(f), C.addressof(p), _ptr(logits_p), _ptr(logits_q), stride,
+                                 _ptr(root_logp), _ptr(root_logq), C.addressof(o), _ptr(workspace),
+                                 workspace.numel(), _ptr(status), _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_verify_step", rc)
+    return status
+
+
+def select_width(forest, params, logits_p, logits_q, node_logp, node_logq, live_off, live_nodes, m,
+                 out_stride, workspace=None, status=None, stream=None, want_alpha=True):
+    """dsbd_select_width; returns (width[R], alpha[R,out_stride], tail[R,out_stride], status)."""
+    _require_cuda(logits_p, logits_q, node_logp, node_logq, live_off, live_nodes, m)
+    keep = []
+    f = forest.struct()
+    p = _params(params, keep)
+    dev = logits_p.device
+    width = torch.zeros(forest.R, dtype=torch.int32, device=dev)
+    alpha = torch.zeros(forest.R, out_stride, dtype=torch.float32, device=dev) if want_alpha else None
+    tail = torch.zeros(forest.R, out_stride, dtype=torch.float32, device=dev) if want_alpha else None
+    need = int(load().dsbd_verify_workspace(C.addressof(f), C.addressof(p)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rc = load().dsbd_select_width(C.addressof(f), C.addressof(p), _ptr(logits_p), _ptr(logits_q),
+                                  logits_p.stride(0), _ptr(node_logp), _ptr(node_logq), _ptr(live_off),
+                                  _ptr(live_nodes), _ptr(m), _ptr(width), _ptr(alpha), _ptr(tail),
+                                  int(out_stride), _ptr(workspace), workspace.numel(), _ptr(status),
+                                  _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_select_width", rc)
+    return width, alpha, tail, status

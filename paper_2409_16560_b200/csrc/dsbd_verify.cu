@@ -1,0 +1,976 @@
+// dsbd_verify_step / dsbd_select_width: the verification step of speculative beam decoding
+// (Algorithm 1 with the dynamic layer width) for sm_100a.
+//
+// Kernels
+//   k_tile_stats   one dense streaming pass over every logits row of both models: per
+//                  1024-token tile the row maximum and sum of exponentials (warp-autonomous,
+//                  128-bit loads, warp-shuffle reductions).  HBM-bound; this is the pass the
+//                  algorithmic bytes 8*N*V belong to.
+//   k_row_finish   per row: log-sum-exp from the tile statistics.
+//   k_tree_scores  per tree: log-prob of every draft token given its parent, cumulative beam
+//                  scores, node depths.
+//   k_verify       one thread-block cluster per request walks the layers: live set, beam
+//                  weights, the residual masses c_{j+1} = F(s_j) (cluster-wide passes over the
+//                  live rows, reduced through a tile-sum table), the acceptance-count
+//                  recursion, the accept loop and the inverse-CDF draws.
+//
+// The residual chain uses the closed form of the paper's recursion p_{k+1} = norm(max(p_k -
+// q_beam, 0)):  with F(s) = sum max(p_beam - s q_beam, 0), c_1 = 1, s_0 = 0, s_j = s_{j-1} + c_j
+// and c_{j+1} = F(s_j) one has p_j = max(p_beam - s_{j-1} q_beam, 0) / c_j, hence
+// alpha_j = 1 - c_{j+1}/c_j and the accept ratio of a draft x at run position j is
+// max(rho(x) - s_{j-1}, 0) / c_j with rho = p_beam(x)/q_beam(x).
+#include <cooperative_groups.h>
+#include <math.h>
+
+#include "dsbd_common.cuh"
+
+namespace cg = cooperative_groups;
+using namespace dsbd;
+
+namespace {
+
+constexpr int kTile = 1024;          // tokens per tile: 32 lanes x 8 x float4
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxLive = DSBD_MAX_LIVE;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr double kLn2 = 0.6931471805599453;
+
+struct TileStat { float mx; float sum; };   // max of the raw logits, sum exp((z-mx)/tau)
+
+__device__ __forceinline__ void load_tile(const float *__restrict__ row, int e0, int V, bool aligned,
+                                          int lane, float4 (&v)[8]) {
+    const float ninf = -INFINITY;
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int e = e0 + it * 128 + lane * 4;
+        if (aligned && e + 3 < V) {
+            v[it] = ldg_stream(reinterpret_cast<const float4 *>(row + e));
+        } else {
+            v[it].x = e < V ? __ldg(row + e) : ninf;
+            v[it].y = e + 1 < V ? __ldg(row + e + 1) : ninf;
+            v[it].z = e + 2 < V ? __ldg(row + e + 2) : ninf;
+            v[it].w = e + 3 < V ? __ldg(row + e + 3) : ninf;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Dense pass: tile statistics of every (model, row).  Item = (model, row, tile), tile fastest,
+// one warp per item.  rows == nullptr: all n_rows rows; else the listed rows (n_rows read
+// from *n_rows_dev when it is given).
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t stride, int V,
+             int T, int N, int n_rows, const int32_t *__restrict__ rows,
+             const int32_t *__restrict__ n_rows_dev, float k2, TileStat *__restrict__ stats) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    if (n_rows_dev) n_rows = *n_rows_dev;
+    const int64_t total = (int64_t)2 * n_rows * T;
+    for (int64_t item = warp; item < total; item += nwarps) {
+        const int t = (int)(item % T);
+        const int64_t rm = item / T;
+        const int model = (int)(rm / n_rows);
+        const int ri = (int)(rm % n_rows);
+        const int row = rows ? rows[ri] : ri;
+        const float *z = (model ? zq : zp) + (int64_t)row * stride;
+        const bool aligned = (reinterpret_cast<uintptr_t>(z) & 15) == 0;
+        float4 v[8];
+        load_tile(z, t * kTile, V, aligned, lane, v);
+        float mx = -INFINITY;
+#pragma unroll
+        for (int it = 0; it < 8; ++it)
+            mx = fmaxf(mx, fmaxf(fmaxf(v[it].x, v[it].y), fmaxf(v[it].z, v[it].w)));
+        mx = warp_max(mx);
+        float sum = 0.f;
+        if (mx > -INFINITY) {
+            const float b = -mx * k2;
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                sum += exp2f(fmaf(v[it].x, k2, b)) + exp2f(fmaf(v[it].y, k2, b)) +
+                       exp2f(fmaf(v[it].z, k2, b)) + exp2f(fmaf(v[it].w, k2, b));
+            }
+        }
+        sum = warp_sum(sum);
+        if (lane == 0) {
+            TileStat s; s.mx = mx; s.sum = sum;
+            stats[((int64_t)model * N + row) * T + t] = s;
+        }
+    }
+}
+
+// log-sum-exp of the tempered row from its tile statistics; one warp per (model, row).
+__global__ void k_row_finish(const TileStat *__restrict__ stats, int T, int N, int n_rows,
+                             const int32_t *__restrict__ rows, const int32_t *__restrict__ n_rows_dev,
+                             double inv_tau, double *__restrict__ lse /*[2][N]*/,
+                             float *__restrict__ lse_p_out, float *__restrict__ lse_q_out) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (n_rows_dev) n_rows = *n_rows_dev;
+    if (warp >= (int64_t)2 * n_rows) return;
+    const int model = (int)(warp / n_rows);
+    const int ri = (int)(warp % n_rows);
+    const int row = rows ? rows[ri] : ri;
+    const TileStat *s = stats + ((int64_t)model * N + row) * T;
+    double mx = -INFINITY;
+    for (int t = lane; t < T; t += 32) mx = fmax(mx, (double)s[t].mx);
+    mx = warp_max(mx);
+    double acc = 0.0;
+    if (mx > -INFINITY)
+        for (int t = lane; t < T; t += 32)
+            if (s[t].sum > 0.f) acc += (double)s[t].sum * exp(((double)s[t].mx - mx) * inv_tau);
+    acc = warp_sum(acc);
+    if (lane == 0) {
+        const double v = (mx > -INFINITY) ? mx * inv_tau + log(acc) : -INFINITY;
+        lse[(int64_t)model * N + row] = v;
+        if (model == 0 && lse_p_out) lse_p_out[row] = (float)v;
+        if (model == 1 && lse_q_out) lse_q_out[row] = (float)v;
+    }
+}
+
+// Cumulative beam scores along every tree (one thread per tree) and node depths.
+__global__ void k_tree_scores(int B, const int32_t *__restrict__ beam_node_off,
+                              const int32_t *__restrict__ parent, const int32_t *__restrict__ token,
+                              const float *__restrict__ zp, const float *__restrict__ zq,
+                              int64_t stride, int V, int max_depth, double inv_tau,
+                              const float *__restrict__ root_logp, const float *__restrict__ root_logq,
+                              const double *__restrict__ lse, int N, double *__restrict__ score /*[2][N]*/,
+                              int32_t *__restrict__ depth, float *__restrict__ node_logp,
+                              float *__restrict__ node_logq, int32_t *status) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int lo = beam_node_off[b], hi = beam_node_off[b + 1];
+    for (int n = lo; n < hi; ++n) {
+        double sp, sq;
+        int dep = 0;
+        const int par = parent[n];
+        if (n == lo) {
+            sp = (double)root_logp[b];
+            sq = (double)root_logq[b];
+            if (par != -1) report(status, DSBD_DEV_BAD_FOREST);
+        } else if (par < lo || par >= n) {
+            report(status, DSBD_DEV_BAD_FOREST);
+            sp = sq = -INFINITY;
+            dep = max_depth + 1;
+        } else {
+            const int tok = token[n];
+            dep = depth[par] + 1;
+            if (dep > max_depth) report(status, DSBD_DEV_BAD_FOREST);
+            if (tok < 0 || tok >= V) {
+                report(status, DSBD_DEV_BAD_TOKEN);
+                sp = sq = -INFINITY;
+            } else {
+                sp = score[par] + ((double)zp[(int64_t)par * stride + tok] * inv_tau - lse[par]);
+                sq = score[N + par] + ((double)zq[(int64_t)par * stride + tok] * inv_tau - lse[N + par]);
+            }
+        }
+        score[n] = sp;
+        score[N + n] = sq;
+        depth[n] = dep;
+        if (node_logp) node_logp[n] = (float)sp;
+        if (node_logq) node_logq[n] = (float)sq;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// The per-request kernel.
+// ---------------------------------------------------------------------------------------
+struct VerifyArgs {
+    // forest
+    int R, N, gamma;
+    const int32_t *req_beam_off, *beam_node_off, *parent, *token, *draft_rank;
+    // parameters
+    int V, T;
+    float k2;                 // log2(e)/tau
+    double inv_tau, thresh;
+    int W_min, W_max, W_nom;
+    const int32_t *W_min_r, *W_max_r, *W_nom_r;
+    uint64_t seed, step;
+    // inputs
+    const float *zp, *zq;
+    int64_t stride;
+    // workspace
+    const TileStat *stats;    // [2][N][T]
+    const double *lse;        // [2][N]
+    const double *score;      // [2][N]
+    const int32_t *depth;     // [N]
+    double *tile_sums;        // [R][2][max_m][max_live*T]
+    int max_m, max_live;
+    // outputs
+    dsbd_verify_out_t out;
+    int32_t *status;
+    // select-width mode
+    int select_mode;
+    const float *sel_logp, *sel_logq;
+    const int32_t *live_off, *live_nodes, *m_in;
+    int32_t *width_out;
+    float *alpha_out, *tail_out;
+    int out_stride;
+};
+
+struct Shared {
+    int nA, m, W, count, done, chain_len, err;
+    int A[kMaxLive];
+    int S[kMaxLive];
+    int S_parent_idx[kMaxLive];
+    int acc[kMaxLive];
+    float bp[kMaxLive], bq[kMaxLive];       // log2 of the beam weight minus lse*log2(e)
+    double lwp[kMaxLive], lwq[kMaxLive];    // natural log of the beam weights
+    double wp[kMaxLive];
+    double s_arr[kMaxLive + 2];             // s_0 .. s_m
+    double c_arr[kMaxLive + 2];             // c_1 .. c_{m+1} (index j)
+    double alpha[kMaxLive + 1];
+    double first[kMaxLive + 1];             // alpha_i prod_{j<i}(1-alpha_j)
+    double col_a[kMaxLive + 1], col_b[kMaxLive + 1];
+    double tail[kMaxLive + 2];
+    float s_cur;
+    int bank;
+};
+
+// mass of one cell of the residual max(p_beam - s q_beam, 0); s == 0 gives p_beam
+__device__ __forceinline__ float cell_mass(float zp, float zq, float k2, float bp, float bq, float s) {
+    const float a = exp2f(fmaf(zp, k2, bp));
+    const float b = exp2f(fmaf(zq, k2, bq));
+    return fmaxf(fmaf(-s, b, a), 0.f);
+}
+
+// One cluster-wide pass: tile sums of max(p_beam - s q_beam, 0) over the live rows.
+__device__ void residual_pass(const VerifyArgs &a, const Shared &sh, float s, double *sums,
+                              int cta_rank, int n_cta) {
+    const int lane = threadIdx.x & 31;
+    const int warp = cta_rank * kWarps + (threadIdx.x >> 5);
+    const int nwarps = n_cta * kWarps;
+    const int items = sh.nA * a.T;
+    for (int item = warp; item < items; item += nwarps) {
+        const int i = item / a.T, t = item - i * a.T;
+        const int row = sh.A[i];
+        const float *rp = a.zp + (int64_t)row * a.stride;
+        const float *rq = a.zq + (int64_t)row * a.stride;
+        const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
+        float4 vp[8], vq[8];
+        load_tile(rp, t * kTile, a.V, al, lane, vp);
+        load_tile(rq, t * kTile, a.V, al, lane, vq);
+        const float bp = sh.bp[i], bq = sh.bq[i];
+        float acc = 0.f;
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            acc += cell_mass(vp[it].x, vq[it].x, a.k2, bp, bq, s);
+            acc += cell_mass(vp[it].y, vq[it].y, a.k2, bp, bq, s);
+            acc += cell_mass(vp[it].z, vq[it].z, a.k2, bp, bq, s);
+            acc += cell_mass(vp[it].w, vq[it].w, a.k2, bp, bq, s);
+        }
+        const double tot = warp_sum((double)acc);
+        if (lane == 0) sums[item] = tot;
+    }
+}
+
+// Ordered sum of n doubles by one warp: lane-strided partial sums, then a butterfly.  The
+// order depends on n only, never on the launch shape.
+__device__ double ordered_sum(const double *v, int n, int lane) {
+    double acc = 0.0;
+    for (int i = lane; i < n; i += 32) acc += __ldcg(v + i);
+    return warp_sum(acc);
+}
+
+// Inverse-CDF search over tile masses (canonical order).  mass(i) must be the same on every
+// lane.  Returns the tile holding the first cell whose running sum reaches target, and the
+// mass before that tile; if rounding leaves the target beyond the total, the last tile with
+// mass.  -1 if there is no mass at all.
+template <class F>
+__device__ int locate_tile(F mass, int n, double target, int lane, double *before) {
+    double running = 0.0, last_before = 0.0;
+    int last = -1;
+    for (int base = 0; base < n; base += 32) {
+        const int i = base + lane;
+        const double v = i < n ? mass(i) : 0.0;
+        const double incl = warp_scan(v, lane);
+        const bool hit = v > 0.0 && running + incl >= target;
+        const unsigned hits = __ballot_sync(kFull, hit);
+        if (hits) {
+            const int l = __ffs(hits) - 1;
+            *before = running + __shfl_sync(kFull, incl - v, l);
+            return base + l;
+        }
+        const unsigned pos = __ballot_sync(kFull, v > 0.0);
+        if (pos) {
+            const int l = 31 - __clz(pos);
+            last = base + l;
+            last_before = running + __shfl_sync(kFull, incl - v, l);
+        }
+        running += __shfl_sync(kFull, incl, 31);
+    }
+    *before = last_before;
+    return last;
+}
+
+// Inverse-CDF search inside one tile of row `row` (and its q row when s > 0): the first
+// token whose running mass reaches `target`, else the last token with mass.  -1: no mass.
+__device__ int locate_token(const VerifyArgs &a, int row, int t, float bp, float bq, float s,
+                            double target, int lane) {
+    const float *rp = a.zp + (int64_t)row * a.stride;
+    const float *rq = a.zq + (int64_t)row * a.stride;
+    double running = 0.0;
+    int last = -1;
+    for (int it = 0; it < 8; ++it) {
+        const int e = t * kTile + it * 128 + lane * 4;
+        float mss[4];
+        double loc = 0.0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float mv = 0.f;
+            if (e + c < a.V) {
+                const float zpv = __ldg(rp + e + c);
+                mv = (s > 0.f) ? cell_mass(zpv, __ldg(rq + e + c), a.k2, bp, bq, s)
+                               : exp2f(fmaf(zpv, a.k2, bp));
+            }
+            mss[c] = mv;
+            loc += (double)mv;
+        }
+        const double incl = warp_scan(loc, lane);
+        const bool hit = loc > 0.0 && running + incl >= target;
+        const unsigned hits = __ballot_sync(kFull, hit);
+        if (hits) {
+            const int l = __ffs(hits) - 1;
+            int tok = -1;
+            if (lane == l) {
+                double cum = running + incl - loc;
+                int lastpos = -1;
+                for (int c = 0; c < 4; ++c) {
+                    cum += (double)mss[c];
+                    if (mss[c] > 0.f) {
+                        lastpos = c;
+                        if (cum >= target) { tok = e + c; break; }
+                    }
+                }
+                if (tok < 0) tok = e + lastpos;
+            }
+            return __shfl_sync(kFull, tok, l);
+        }
+        const unsigned pos = __ballot_sync(kFull, loc > 0.0);
+        if (pos) {
+            const int l = 31 - __clz(pos);
+            int lp = -1;
+            if (lane == l)
+                for (int c = 0; c < 4; ++c) if (mss[c] > 0.f) lp = e + c;
+            last = __shfl_sync(kFull, lp, l);
+        }
+        running += __shfl_sync(kFull, incl, 31);
+    }
+    return last;
+}
+
+__device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, int node, int tok,
+                            int source, bool writer, int *err) {
+    const int cap = a.out.out_off[r + 1] - a.out.out_off[r];
+    if (*n_out >= cap) { *err = DSBD_DEV_CAPACITY; return; }
+    if (writer) {
+        const int s = a.out.out_off[r] + *n_out;
+        // the tree of a node: walk to the root, then find which beam starts there
+        int root = parent;
+        while (a.parent[root] >= 0) root = a.parent[root];
+        int lo = a.req_beam_off[r], hi = a.req_beam_off[r + 1];
+        int beam = lo;
+        for (int b = lo; b < hi; ++b) if (a.beam_node_off[b] == root) beam = b;
+        a.out.out_parent[s] = parent;
+        a.out.out_node[s] = node;
+        a.out.out_root_beam[s] = beam;
+        a.out.out_token[s] = tok;
+        a.out.out_source[s] = source;
+        const double lp = (double)a.zp[(int64_t)parent * a.stride + tok] * a.inv_tau - a.lse[parent];
+        const double lq = (double)a.zq[(int64_t)parent * a.stride + tok] * a.inv_tau - a.lse[a.N + parent];
+        a.out.out_logp[s] = (float)(a.score[parent] + lp);
+        a.out.out_logq[s] = (float)(a.score[a.N + parent] + lq);
+    }
+    (*n_out)++;
+}
+
+// Beam weights of the live set: softmax of the cumulative scores over A (Eq. 1 factorised).
+__device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, const double *sq) {
+    double mp = -INFINITY, mq = -INFINITY;
+    for (int i = 0; i < sh.nA; ++i) { mp = fmax(mp, sp[i]); mq = fmax(mq, sq[i]); }
+    double tp = 0.0, tq = 0.0;
+    for (int i = 0; i < sh.nA; ++i) { tp += exp(sp[i] - mp); tq += exp(sq[i] - mq); }
+    for (int i = 0; i < sh.nA; ++i) {
+        const double wp = exp(sp[i] - mp) / tp, wq = exp(sq[i] - mq) / tq;
+        sh.wp[i] = wp;
+        sh.lwp[i] = log(wp);
+        sh.lwq[i] = log(wq);
+        const int row = sh.A[i];
+        sh.bp[i] = (float)((sh.lwp[i] - a.lse[row]) / kLn2);
+        sh.bq[i] = (float)((sh.lwq[i] - a.lse[a.N + row]) / kLn2);
+    }
+}
+
+// Acceptance-count recursion by one warp (lanes over n): tail[K] = P(at least K accepts),
+// returns W~ = max{K : tail[K] >= thresh}.
+__device__ int width_rule(Shared &sh, int m, double thresh, int lane) {
+    if (lane == 0) {
+        double none = 1.0;
+        for (int i = 1; i <= m; ++i) {
+            sh.first[i] = sh.alpha[i] * none;
+            none *= (1.0 - sh.alpha[i]);
+            sh.col_a[i] = none;                    // P(n, 0) = prod_{j<=n}(1 - alpha_j)
+        }
+        sh.col_a[0] = 1.0;
+        sh.tail[0] = 1.0;
+    }
+    __syncwarp();
+    double *prev = sh.col_a, *cur = sh.col_b;
+    double below = 0.0;
+    for (int k = 0; k <= m; ++k) {
+        // prev = P(., k); record tail
+        below += prev[m];
+        if (lane == 0) sh.tail[k + 1] = 1.0 - below;
+        if (k == m) break;
+        for (int n = lane; n <= m; n += 32) {
+            double acc = 0.0;
+            if (n >= k + 1)
+                for (int i = 1; i <= n; ++i) acc += sh.first[i] * prev[n - i];
+            cur[n] = acc;                          // P(n, k+1), zero for n < k+1
+        }
+        __syncwarp();
+        double *tmp = prev; prev = cur; cur = tmp;
+    }
+    __syncwarp();
+    int wt = 0;
+    for (int K = 0; K <= m; ++K) if (sh.tail[K] >= thresh) wt = K;
+    if (lane == 0) sh.tail[m + 1] = 0.0;
+    return wt;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_verify(VerifyArgs a) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int n_cta = (int)cluster.num_blocks();
+    const int cta_rank = (int)cluster.block_rank();
+    const int r = blockIdx.x / n_cta;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const bool writer = (cta_rank == 0);
+    __shared__ Shared sh;
+    __shared__ double sp_live[kMaxLive], sq_live[kMaxLive];
+
+    const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
+    const int n_lo = a.beam_node_off[b_lo], n_hi = a.beam_node_off[b_hi];
+    const int W_min = a.W_min_r ? a.W_min_r[r] : a.W_min;
+    const int W_max = a.W_max_r ? a.W_max_r[r] : a.W_max;
+    const int W_nom = a.W_nom_r ? a.W_nom_r[r] : a.W_nom;
+    double *sums_base = a.tile_sums + (int64_t)r * 2 * a.max_m * ((int64_t)a.max_live * a.T);
+    const int64_t slot_stride = (int64_t)a.max_live * a.T;
+    int n_out = 0;
+
+    // ---- set-up ----
+    if (warp == 0) {
+        if (lane == 0) {
+            sh.err = 0; sh.done = 0;
+            if (a.select_mode) {
+                const int lo = a.live_off[r], hi = a.live_off[r + 1];
+                sh.nA = hi - lo;
+                if (sh.nA > kMaxLive || sh.nA < 0) { sh.err = DSBD_DEV_BAD_FOREST; sh.nA = 0; }
+                for (int i = 0; i < sh.nA; ++i) {
+                    sh.A[i] = a.live_nodes[lo + i];
+                    sp_live[i] = (double)a.sel_logp[sh.A[i]];
+                    sq_live[i] = (double)a.sel_logq[sh.A[i]];
+                }
+            } else {
+                sh.nA = b_hi - b_lo;
+                if (sh.nA > kMaxLive) { sh.err = DSBD_DEV_BAD_FOREST; sh.nA = 0; }
+                for (int i = 0; i < sh.nA; ++i) {
+                    sh.A[i] = a.beam_node_off[b_lo + i];
+                    sp_live[i] = a.score[sh.A[i]];
+                    sq_live[i] = a.score[a.N + sh.A[i]];
+                }
+                if (writer) {
+                    for (int l = 0; l <= a.gamma; ++l) a.out.layer_width[(int64_t)r * (a.gamma + 1) + l] = -1;
+                    a.out.l_last[r] = a.gamma + 1;
+                    a.out.out_width[r] = 0;
+                }
+            }
+        }
+        __syncwarp();
+        if (!a.select_mode && writer)
+            for (int n = n_lo + lane; n < n_hi; n += 32)
+                a.out.node_status[n] = a.parent[n] < 0 ? DSBD_NODE_ACCEPTED : DSBD_NODE_UNREACHED;
+    }
+    __syncthreads();
+    // node_status is read back by this same CTA only through shared decisions below; the other
+    // CTAs of the cluster keep their own copy of every decision, so only rank 0 writes it.
+
+    const int n_layers = a.select_mode ? 1 : a.gamma;
+    // status of the nodes as this CTA sees it (every CTA takes identical decisions)
+    __shared__ int8_t st[kMaxLive * kMaxLive];     // nodes of one request, local index
+    const int n_req_nodes = n_hi - n_lo;
+    const bool st_ok = n_req_nodes <= kMaxLive * kMaxLive;
+    if (!a.select_mode) {
+        for (int n = threadIdx.x; n < n_req_nodes && st_ok; n += blockDim.x)
+            st[n] = a.parent[n_lo + n] < 0 ? DSBD_NODE_ACCEPTED : DSBD_NODE_UNREACHED;
+        if (!st_ok && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_FOREST;
+    }
+    __syncthreads();
+
+    for (int l = 1; l <= n_layers && !sh.done && !sh.err; ++l) {
+        // ---- live drafts of layer l, in draw order; beam weights ----
+        if (warp == 0) {
+            int m = 0;
+            if (a.select_mode) {
+                m = a.m_in[r];
+                if (m < 0 || m > kMaxLive) { if (lane == 0) sh.err = DSBD_DEV_BAD_FOREST; m = 0; }
+            } else {
+                for (int base = 0; base < n_req_nodes; base += 32) {
+                    const int n = base + lane;
+                    bool at_layer = false, live = false;
+                    if (n < n_req_nodes && a.depth[n_lo + n] == l) {
+                        at_layer = true;
+                        live = st[a.parent[n_lo + n] - n_lo] == DSBD_NODE_ACCEPTED;
+                        if (!live) {
+                            st[n] = DSBD_NODE_PRUNED;
+                            if (writer) a.out.node_status[n_lo + n] = DSBD_NODE_PRUNED;
+                        }
+                    }
+                    (void)at_layer;
+                    const unsigned mask = __ballot_sync(kFull, live);
+                    const int pos = m + __popc(mask & ((1u << lane) - 1));
+                    if (live) {
+                        if (pos < kMaxLive) sh.S[pos] = n_lo + n;
+                    }
+                    m += __popc(mask);
+                }
+                if (m > kMaxLive) { if (lane == 0) sh.err = DSBD_DEV_BAD_FOREST; m = 0; }
+                __syncwarp();
+                if (lane == 0 && a.draft_rank) {
+                    // insertion sort by (draft_rank, node id); ids are already ascending
+                    for (int i = 1; i < m; ++i) {
+                        const int n = sh.S[i];
+                        const int key = a.draft_rank[n];
+                        int j = i - 1;
+                        while (j >= 0 && a.draft_rank[sh.S[j]] > key) { sh.S[j + 1] = sh.S[j]; --j; }
+                        sh.S[j + 1] = n;
+                    }
+                }
+            }
+            if (lane == 0) {
+                sh.m = m;
+                live_weights(a, sh, sp_live, sq_live);
+                if (!a.select_mode)
+                    for (int i = 0; i < m; ++i) {
+                        const int par = a.parent[sh.S[i]];
+                        int ai = 0;
+                        while (ai < sh.nA && sh.A[ai] != par) ++ai;
+                        sh.S_parent_idx[i] = ai;
+                    }
+                sh.s_arr[0] = 0.0;
+                sh.c_arr[1] = 1.0;
+                sh.chain_len = 0;          // number of c_{j+1} known: j = 1..chain_len
+                sh.s_cur = 1.0f;
+                sh.bank = l & 1;
+            }
+        }
+        __syncthreads();
+        const int m = sh.m;
+
+        // ---- residual masses c_{j+1} = F(s_j), j = 1..m ----
+        for (int j = 1; j <= m && !sh.err; ++j) {
+            double *sums = sums_base + ((int64_t)sh.bank * a.max_m + (j - 1)) * slot_stride;
+            const double s_j = sh.s_arr[j - 1] + sh.c_arr[j];
+            residual_pass(a, sh, (float)s_j, sums, cta_rank, n_cta);
+            __threadfence();
+            cluster.sync();
+            bool stop = false;
+            if (warp == 0) {
+                const double c_next = ordered_sum(sums, sh.nA * a.T, lane);
+                if (lane == 0) {
+                    sh.s_arr[j] = s_j;
+                    sh.c_arr[j + 1] = c_next;
+                    sh.chain_len = j;
+                }
+            }
+            __syncthreads();
+            stop = !(sh.c_arr[j + 1] > 0.0);
+            if (stop) break;
+        }
+        __syncthreads();
+
+        // ---- width, accept loop, completion (warp 0) ----
+        if (warp == 0 && !sh.err) {
+            // alpha_j = 1 - c_{j+1}/c_j; once a residual has no mass every later alpha is 1
+            if (lane == 0) {
+                for (int j = 1; j <= m; ++j) {
+                    if (j <= sh.chain_len && sh.c_arr[j] > 0.0) {
+                        double al = 1.0 - sh.c_arr[j + 1] / sh.c_arr[j];
+                        if (!(sh.c_arr[j + 1] > 0.0)) al = 1.0;
+                        sh.alpha[j] = fmin(fmax(al, 0.0), 1.0);
+                    } else {
+                        sh.alpha[j] = 1.0;
+                    }
+                }
+            }
+            __syncwarp();
+            const int wt = width_rule(sh, m, a.thresh, lane);
+            int W = wt > W_min ? wt : W_min;
+            if (W > W_max) W = W_max;
+            if (a.select_mode) {
+                if (writer && lane == 0) {
+                    a.width_out[r] = W;
+                    if (a.alpha_out)
+                        for (int j = 0; j < m && j < a.out_stride; ++j)
+                            a.alpha_out[(int64_t)r * a.out_stride + j] = (float)sh.alpha[j + 1];
+                    if (a.tail_out)
+                        for (int K = 0; K <= m && K < a.out_stride; ++K)
+                            a.tail_out[(int64_t)r * a.out_stride + K] = (float)sh.tail[K];
+                }
+                if (lane == 0) sh.done = 1;
+            } else {
+                if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + (l - 1)] = W;
+                // accept loop (lane 0), Algorithm 1
+                int count = 0, j = 1, err = 0;
+                if (lane == 0) {
+                    for (int i = 0; i < m && count < W; ++i) {
+                        const int n = sh.S[i];
+                        const int ai = sh.S_parent_idx[i];
+                        const double lp = a.score[n] - a.score[a.parent[n]];
+                        const double lq = a.score[a.N + n] - a.score[a.N + a.parent[n]];
+                        double rho;
+                        if (lq == -INFINITY || sh.lwq[ai] == -INFINITY)
+                            rho = (lp > -INFINITY && sh.lwp[ai] > -INFINITY) ? INFINITY : 0.0;
+                        else
+                            rho = exp((sh.lwp[ai] - sh.lwq[ai]) + (lp - lq));
+                        double ratio;
+                        if (j == 1) ratio = rho;
+                        else ratio = fmax(rho - sh.s_arr[j - 1], 0.0) / sh.c_arr[j];
+                        if (ratio > 1.0) ratio = 1.0;
+                        const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l, 0u, (uint32_t)i);
+                        if (u <= ratio) {
+                            st[n - n_lo] = DSBD_NODE_ACCEPTED;
+                            if (writer) a.out.node_status[n] = DSBD_NODE_ACCEPTED;
+                            sh.acc[count++] = n;
+                            j = 1;
+                        } else {
+                            st[n - n_lo] = DSBD_NODE_REJECTED;
+                            if (writer) a.out.node_status[n] = DSBD_NODE_REJECTED;
+                            if (j <= sh.chain_len && sh.c_arr[j + 1] > 0.0) {
+                                ++j;
+                            } else {
+                                err = DSBD_DEV_EXHAUSTED;     // a rejection of probability zero
+                                j = 1;
+                            }
+                        }
+                    }
+                    for (int i = 0; i < m; ++i)
+                        if (st[sh.S[i] - n_lo] == DSBD_NODE_UNREACHED) {
+                            st[sh.S[i] - n_lo] = DSBD_NODE_CUT;
+                            if (writer) a.out.node_status[sh.S[i]] = DSBD_NODE_CUT;
+                        }
+                }
+                count = __shfl_sync(kFull, count, 0);
+                j = __shfl_sync(kFull, j, 0);
+                err = __shfl_sync(kFull, err, 0);
+                if (count < W) {
+                    // short layer: accepted drafts, one draw from p', the rest from p_beam
+                    if (lane == 0)
+                        for (int i = 0; i < count && !err; ++i)
+                            emit_output(a, r, &n_out, a.parent[sh.acc[i]], sh.acc[i], a.token[sh.acc[i]],
+                                        DSBD_SRC_DRAFT, writer, &err);
+                    n_out = __shfl_sync(kFull, n_out, 0);
+                    err = __shfl_sync(kFull, err, 0);
+                    int fill = 0;
+                    for (int kk = count; kk < W && !err; ++kk) {
+                        const bool residual = (kk == count);
+                        const bool use_res = residual && j > 1;
+                        const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l,
+                                                          residual ? 1u : 2u, residual ? 0u : (uint32_t)fill);
+                        int tile = -1;
+                        double before = 0.0;
+                        float s_res = 0.f;
+                        if (use_res) {
+                            const double *sums = sums_base + ((int64_t)sh.bank * a.max_m + (j - 2)) * slot_stride;
+                            s_res = (float)sh.s_arr[j - 1];
+                            const double target = u * sh.c_arr[j];
+                            tile = locate_tile([&](int i) { return __ldcg(sums + i); }, sh.nA * a.T,
+                                               target, lane, &before);
+                            before = target - before;
+                        } else {
+                            double z = 0.0;
+                            for (int i = 0; i < sh.nA; ++i) z += sh.wp[i];
+                            const double target = u * z;
+                            const int T = a.T;
+                            tile = locate_tile([&](int i) {
+                                const int ia = i / T;
+                                const int row = sh.A[ia];
+                                const TileStat ts = a.stats[(int64_t)row * T + (i - ia * T)];
+                                if (!(ts.sum > 0.f)) return 0.0;
+                                return sh.wp[ia] * (double)ts.sum *
+                                       exp((double)ts.mx * a.inv_tau - a.lse[row]);
+                            }, sh.nA * a.T, target, lane, &before);
+                            before = target - before;
+                        }
+                        int tok = -1, ia = 0;
+                        if (tile >= 0) {
+                            ia = tile / a.T;
+                            tok = locate_token(a, sh.A[ia], tile - ia * a.T, sh.bp[ia], sh.bq[ia], s_res,
+                                               before, lane);
+                        }
+                        if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
+                        if (lane == 0)
+                            emit_output(a, r, &n_out, sh.A[ia], -1, tok,
+                                        residual ? DSBD_SRC_RESIDUAL : DSBD_SRC_FILL, writer, &err);
+                        n_out = __shfl_sync(kFull, n_out, 0);
+                        err = __shfl_sync(kFull, err, 0);
+                        if (!residual) ++fill;
+                    }
+                    if (lane == 0) {
+                        sh.done = 1;
+                        if (writer) a.out.l_last[r] = l;
+                    }
+                } else if (lane == 0) {
+                    // the accepted drafts, ascending node id, are the next layer's input beams
+                    int nA = 0;
+                    for (int n = 0; n < n_req_nodes; ++n)
+                        if (a.depth[n_lo + n] == l && st[n] == DSBD_NODE_ACCEPTED) {
+                            sh.A[nA] = n_lo + n;
+                            sp_live[nA] = a.score[n_lo + n];
+                            sq_live[nA] = a.score[a.N + n_lo + n];
+                            ++nA;
+                        }
+                    sh.nA = nA;
+                }
+                if (lane == 0 && err) sh.err = err;
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- every layer passed: W_nom beams from p_beam^(gamma+1) ----
+    if (!a.select_mode && warp == 0 && !sh.done && !sh.err) {
+        if (lane == 0) live_weights(a, sh, sp_live, sq_live);
+        __syncwarp();
+        int err = 0;
+        if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
+        for (int kk = 0; kk < W_nom && !err; ++kk) {
+            const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1), 3u, (uint32_t)kk);
+            double z = 0.0;
+            for (int i = 0; i < sh.nA; ++i) z += sh.wp[i];
+            const double target = u * z;
+            const int T = a.T;
+            double before = 0.0;
+            const int tile = locate_tile([&](int i) {
+                const int ia = i / T;
+                const int row = sh.A[ia];
+                const TileStat ts = a.stats[(int64_t)row * T + (i - ia * T)];
+                if (!(ts.sum > 0.f)) return 0.0;
+                return sh.wp[ia] * (double)ts.sum * exp((double)ts.mx * a.inv_tau - a.lse[row]);
+            }, sh.nA * a.T, target, lane, &before);
+            int tok = -1, ia = 0;
+            if (tile >= 0) {
+                ia = tile / a.T;
+                tok = locate_token(a, sh.A[ia], tile - ia * a.T, sh.bp[ia], sh.bq[ia], 0.f,
+                                   target - before, lane);
+            }
+            if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
+            if (lane == 0)
+                emit_output(a, r, &n_out, sh.A[ia], -1, tok, DSBD_SRC_EXTRA, writer, &err);
+            n_out = __shfl_sync(kFull, n_out, 0);
+            err = __shfl_sync(kFull, err, 0);
+        }
+        if (lane == 0 && err) sh.err = err;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && writer) {
+        if (!a.select_mode) {
+            a.out.out_width[r] = n_out;
+            if (a.out.req_error) a.out.req_error[r] = sh.err;
+        }
+        if (sh.err) report(a.status, sh.err);
+    }
+}
+
+// ------------------------------------------------------------------------------ host side
+struct Layout {
+    size_t stats, lse, score, depth, sums, total;
+    int T, max_m, max_live;
+};
+
+Layout make_layout(const dsbd_forest_t *f, int V) {
+    Layout L;
+    L.T = (V + kTile - 1) / kTile;
+    L.max_live = f->max_req_beams > f->max_layer_nodes ? f->max_req_beams : f->max_layer_nodes;
+    if (L.max_live < 1) L.max_live = 1;
+    L.max_m = f->max_layer_nodes > 1 ? f->max_layer_nodes : 1;
+    size_t off = 0;
+    L.stats = off; off = align_up(off + sizeof(TileStat) * 2 * (size_t)f->N * L.T, 256);
+    L.lse = off;   off = align_up(off + sizeof(double) * 2 * (size_t)f->N, 256);
+    L.score = off; off = align_up(off + sizeof(double) * 2 * (size_t)f->N, 256);
+    L.depth = off; off = align_up(off + sizeof(int32_t) * (size_t)f->N, 256);
+    L.sums = off;
+    off = align_up(off + sizeof(double) * (size_t)f->R * 2 * L.max_m * (size_t)L.max_live * L.T, 256);
+    L.total = off;
+    return L;
+}
+
+int check_forest(const dsbd_forest_t *f) {
+    if (!f || f->R <= 0 || f->B <= 0 || f->N <= 0 || f->max_depth < 0) return DSBD_ERR_INVALID_ARG;
+    if (!f->req_beam_off || !f->beam_node_off || !f->parent || !f->token) return DSBD_ERR_INVALID_ARG;
+    if (f->max_req_beams <= 0 || f->max_layer_nodes < 0) return DSBD_ERR_INVALID_ARG;
+    if (f->max_req_beams > DSBD_MAX_LIVE || f->max_layer_nodes > DSBD_MAX_LIVE) return DSBD_ERR_UNSUPPORTED;
+    return DSBD_OK;
+}
+
+int check_params(const dsbd_verify_params_t *p) {
+    if (!p || p->V <= 0 || !(p->temperature > 0.f)) return DSBD_ERR_INVALID_ARG;
+    if (p->W_min < 1 && !p->W_min_r) return DSBD_ERR_INVALID_ARG;
+    return DSBD_OK;
+}
+
+int cluster_size_for(int tiles) {
+    if (tiles >= 64) return 8;
+    if (tiles >= 32) return 4;
+    if (tiles >= 16) return 2;
+    return 1;
+}
+
+int launch_verify(const VerifyArgs &args, int R, int tiles, cudaStream_t stream) {
+    const int cs = cluster_size_for(tiles);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(R * cs));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_verify, args) == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
+
+int stats_grid(int64_t items) {
+    // enough warps to cover the items, capped at a few waves of a 148-SM part
+    int64_t blocks = (items + kWarps - 1) / kWarps;
+    const int64_t cap = 148 * 8 * 4;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+}  // namespace
+
+extern "C" size_t dsbd_verify_workspace(const dsbd_forest_t *forest, const dsbd_verify_params_t *params) {
+    if (check_forest(forest) != DSBD_OK || check_params(params) != DSBD_OK) return 0;
+    return make_layout(forest, params->V).total;
+}
+
+extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params_t *p,
+                                const float *logits_p, const float *logits_q, int64_t row_stride,
+                                const float *root_logp, const float *root_logq,
+                                const dsbd_verify_out_t *out, void *workspace, size_t workspace_bytes,
+                                int32_t *status, dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    int rc = check_forest(f);
+    if (rc) return rc;
+    rc = check_params(p);
+    if (rc) return rc;
+    if (!logits_p || !logits_q || !root_logp || !root_logq || !out || !workspace || !status)
+        return DSBD_ERR_INVALID_ARG;
+    if (row_stride < p->V) return DSBD_ERR_INVALID_ARG;
+    if (!out->l_last || !out->out_width || !out->out_off || !out->out_parent || !out->out_node ||
+        !out->out_root_beam || !out->out_token || !out->out_logp || !out->out_logq ||
+        !out->out_source || !out->node_status || !out->layer_width)
+        return DSBD_ERR_INVALID_ARG;
+    const Layout L = make_layout(f, p->V);
+    if (workspace_bytes < L.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    TileStat *stats = reinterpret_cast<TileStat *>(ws + L.stats);
+    double *lse = reinterpret_cast<double *>(ws + L.lse);
+    double *score = reinterpret_cast<double *>(ws + L.score);
+    int32_t *depth = reinterpret_cast<int32_t *>(ws + L.depth);
+    const double inv_tau = 1.0 / (double)p->temperature;
+    const float k2 = (float)((double)kLog2e * inv_tau);
+
+    const int64_t items = (int64_t)2 * f->N * L.T;
+    k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_p, logits_q, row_stride, p->V, L.T,
+                                                            f->N, f->N, nullptr, nullptr, k2, stats);
+    {
+        const int64_t warps = (int64_t)2 * f->N;
+        k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
+            stats, L.T, f->N, f->N, nullptr, nullptr, inv_tau, lse, out->lse_p, out->lse_q);
+    }
+    k_tree_scores<<<(f->B + 127) / 128, 128, 0, stream>>>(
+        f->B, f->beam_node_off, f->parent, f->token, logits_p, logits_q, row_stride, p->V, f->max_depth,
+        inv_tau, root_logp, root_logq, lse, f->N, score, depth, out->node_logp, out->node_logq, status);
+    if (cudaGetLastError() != cudaSuccess) return DSBD_ERR_CUDA;
+
+    VerifyArgs a = {};
+    a.R = f->R; a.N = f->N; a.gamma = f->max_depth;
+    a.req_beam_off = f->req_beam_off; a.beam_node_off = f->beam_node_off;
+    a.parent = f->parent; a.token = f->token; a.draft_rank = f->draft_rank;
+    a.V = p->V; a.T = L.T; a.k2 = k2; a.inv_tau = inv_tau; a.thresh = (double)p->thresh;
+    a.W_min = p->W_min; a.W_max = p->W_max; a.W_nom = p->W_nom;
+    a.W_min_r = p->W_min_r; a.W_max_r = p->W_max_r; a.W_nom_r = p->W_nom_r;
+    a.seed = p->seed; a.step = p->step;
+    a.zp = logits_p; a.zq = logits_q; a.stride = row_stride;
+    a.stats = stats; a.lse = lse; a.score = score; a.depth = depth;
+    a.tile_sums = reinterpret_cast<double *>(ws + L.sums);
+    a.max_m = L.max_m; a.max_live = L.max_live;
+    a.out = *out; a.status = status; a.select_mode = 0;
+    return launch_verify(a, f->R, L.max_live * L.T, stream);
+}
+
+extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_params_t *p,
+                                 const float *logits_p, const float *logits_q, int64_t row_stride,
+                                 const float *node_logp, const float *node_logq,
+                                 const int32_t *live_off, const int32_t *live_nodes, const int32_t *m,
+                                 int32_t *width, float *alpha, float *tail, int32_t out_stride,
+                                 void *workspace, size_t workspace_bytes, int32_t *status,
+                                 dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    int rc = check_forest(f);
+    if (rc) return rc;
+    rc = check_params(p);
+    if (rc) return rc;
+    if (!logits_p || !logits_q || !node_logp || !node_logq || !live_off || !live_nodes || !m ||
+        !width || !workspace || !status)
+        return DSBD_ERR_INVALID_ARG;
+    if (row_stride < p->V || ((alpha || tail) && out_stride < 1)) return DSBD_ERR_INVALID_ARG;
+    const Layout L = make_layout(f, p->V);
+    if (workspace_bytes < L.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    TileStat *stats = reinterpret_cast<TileStat *>(ws + L.stats);
+    double *lse = reinterpret_cast<double *>(ws + L.lse);
+    const double inv_tau = 1.0 / (double)p->temperature;
+    const float k2 = (float)((double)kLog2e * inv_tau);
+
+    // statistics of the live rows only; their number is live_off[R], known on the device
+    const int max_rows = f->R * L.max_live < f->N ? f->R * L.max_live : f->N;
+    const int64_t items = (int64_t)2 * max_rows * L.T;
+    k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_p, logits_q, row_stride, p->V, L.T,
+                                                            f->N, 0, live_nodes, live_off + f->R, k2, stats);
+    {
+        const int64_t warps = (int64_t)2 * max_rows;
+        k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
+            stats, L.T, f->N, 0, live_nodes, live_off + f->R, inv_tau, lse, nullptr, nullptr);
+    }
+    if (cudaGetLastError() != cudaSuccess) return DSBD_ERR_CUDA;
+
+    VerifyArgs a = {};
+    a.R = f->R; a.N = f->N; a.gamma = f->max_depth;
+    a.req_beam_off = f->req_beam_off; a.beam_node_off = f->beam_node_off;
+    a.parent = f->parent; a.token = f->token; a.draft_rank = f->draft_rank;
+    a.V = p->V; a.T = L.T; a.k2 = k2; a.inv_tau = inv_tau; a.thresh = (double)p->thresh;
+    a.W_min = p->W_min; a.W_max = p->W_max; a.W_nom = p->W_nom;
+    a.W_min_r = p->W_min_r; a.W_max_r = p->W_max_r; a.W_nom_r = p->W_nom_r;
+    a.seed = p->seed; a.step = p->step;
+    a.zp = logits_p; a.zq = logits_q; a.stride = row_stride;
+    a.stats = stats; a.lse = lse; a.score = nullptr; a.depth = nullptr;
+    a.tile_sums = reinterpret_cast<double *>(ws + L.sums);
+    a.max_m = L.max_m; a.max_live = L.max_live;
+    a.status = status; a.select_mode = 1;
+    a.sel_logp = node_logp; a.sel_logq = node_logq;
+    a.live_off = live_off; a.live_nodes = live_nodes; a.m_in = m;
+    a.width_out = width; a.alpha_out = alpha; a.tail_out = tail; a.out_stride = out_stride;
+    return launch_verify(a, f->R, L.max_live * L.T, stream);
+}

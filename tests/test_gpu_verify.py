@@ -1,0 +1,234 @@
+"""GPU parity of dsbd_verify_step / dsbd_select_width against the oracle (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2409_16560_b200 as dsbd
+from paper_2409_16560_b200 import inputs
+from parity_util import (check_exempt, compare_verify, run_gpu_verify, sub_forest, to_host_f32)
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle(forest, params, zp, zq, rp, rq, threads=8):
+    return oracle.verify_step(forest, params, zp, zq, rp.astype(np.float64), rq.astype(np.float64),
+                              threads=threads)
+
+
+def _both(data, steps, thresh=None):
+    f, prm = data["forest"], dict(data["params"])
+    if thresh is not None:
+        prm["thresh"] = thresh
+    zp_h, zq_h = to_host_f32(data["logits_p"]), to_host_f32(data["logits_q"])
+    rp_h, rq_h = to_host_f32(data["root_logp"]), to_host_f32(data["root_logq"])
+    exempt = decisions = 0
+    for step in steps:
+        prm["step"] = step
+        gpu, status = run_gpu_verify(f, prm, data["logits_p"], data["logits_q"], data["root_logp"],
+                                     data["root_logq"])
+        assert status == 0
+        ref = _oracle(f, prm, zp_h, zq_h, rp_h, rq_h)
+        e, d = compare_verify(ref, gpu, f)
+        exempt += e
+        decisions += d
+    check_exempt(exempt, decisions)
+    return exempt, decisions
+
+
+@pytest.mark.parametrize("name,steps", [("C1", range(40)), ("C2", range(40)), ("C3", range(6)),
+                                        ("C4", range(3))])
+def test_configs_full_size(name, steps):
+    data = inputs.generate(inputs.config(name), "cuda", parts=("verify",))
+    _both(data, steps)
+
+
+@pytest.mark.parametrize("thresh,wmin", [(0.9, 1), (0.3, 1), (0.7, 8)])
+def test_other_width_settings(thresh, wmin):
+    data = inputs.generate(inputs.config("C3", R=2, V=5000), "cuda", parts=("verify",))
+    data["params"]["W_min_r"] = None
+    data["params"]["W_min"] = wmin
+    _both(data, range(8), thresh=thresh)
+
+
+def test_c5_sampled_requests():
+    """Full C5 on the GPU; the oracle verifies a seeded sample of its requests."""
+    spec = inputs.config("C5")
+    data = inputs.generate(spec, "cuda", parts=("verify",))
+    f, prm = data["forest"], dict(data["params"])
+    gpu, status = run_gpu_verify(f, prm, data["logits_p"], data["logits_q"], data["root_logp"],
+                                 data["root_logq"])
+    assert status == 0
+    reqs = sorted(np.random.default_rng(1).choice(f["R"], size=4, replace=False).tolist())
+    sub, nodes, beams = sub_forest(f, reqs)
+    idx = torch.as_tensor(nodes, device="cuda")
+    bidx = torch.as_tensor(beams, device="cuda")
+    sprm = dict(prm, W_min_r=np.asarray(prm["W_min_r"])[reqs], req_id=np.asarray(reqs, np.int32))
+    ref = _oracle(sub, sprm, to_host_f32(data["logits_p"][idx]), to_host_f32(data["logits_q"][idx]),
+                  to_host_f32(data["root_logp"][bidx]), to_host_f32(data["root_logq"][bidx]))
+    # bring the GPU's results for those requests into the sub-forest numbering
+    remap = np.full(f["N"] + 1, -1, np.int64)
+    remap[nodes] = np.arange(len(nodes))
+    bremap = np.full(f["B"] + 1, -1, np.int64)
+    bremap[beams] = np.arange(len(beams))
+    off_full = oracle.default_out_off(f, prm)
+    g = {k: gpu[k][reqs] for k in ("l_last", "out_width", "req_error", "layer_width")}
+    for k in ("node_status", "node_logp", "node_logq", "lse_p", "lse_q"):
+        g[k] = gpu[k][nodes]
+    for k in ("out_parent", "out_node", "out_root_beam", "out_token", "out_source", "out_logp", "out_logq"):
+        g[k] = np.zeros(int(ref["out_off"][-1]), gpu[k].dtype)
+    for i, r in enumerate(reqs):
+        w = int(gpu["out_width"][r])
+        src = slice(off_full[r], off_full[r] + w)
+        dst = slice(ref["out_off"][i], ref["out_off"][i] + w)
+        g["out_parent"][dst] = remap[gpu["out_parent"][src]]
+        g["out_node"][dst] = np.where(gpu["out_node"][src] >= 0, remap[gpu["out_node"][src]], -1)
+        g["out_root_beam"][dst] = bremap[gpu["out_root_beam"][src]]
+        for k in ("out_token", "out_source", "out_logp", "out_logq"):
+            g[k][dst] = gpu[k][src]
+    e, d = compare_verify(ref, g, sub, req_ids=reqs)
+    check_exempt(e, d * 25)     # 4 of 64 requests of one step: judge the rate, not one event
+    # properties that hold for every request
+    assert np.all(gpu["req_error"] == 0)
+    assert np.all((gpu["l_last"] >= 1) & (gpu["l_last"] <= f["max_depth"] + 1))
+    assert np.all(gpu["out_width"] >= 1)
+
+
+def _random_problem(rng, R, V, gamma, max_w, stride_pad=0, ninf_frac=0.0, tree="chain"):
+    widths = rng.integers(1, max_w + 1, size=R)
+    spec = dict(R=R, W=(1, max_w), tree=inputs._chain(gamma) if tree == "chain" else inputs._binary(gamma),
+                prefix=(1, 1))
+    forest, widths, _ = inputs.build_forest(spec, rng)
+    N, B = forest["N"], forest["B"]
+    stride = V + stride_pad
+    zp = rng.normal(0, 2.5, size=(N, stride)).astype(np.float32)
+    zq = (zp + rng.normal(0, 1.0, size=(N, stride))).astype(np.float32)
+    if ninf_frac > 0:
+        mask = rng.uniform(size=(1, stride)) < ninf_frac      # the same vocabulary entries for p and q
+        zp[np.broadcast_to(mask, zp.shape)] = -np.inf
+        zq[np.broadcast_to(mask, zq.shape)] = -np.inf
+    tok = np.zeros(N, np.int32)
+    for n in range(N):
+        p = forest["parent"][n]
+        if p >= 0:
+            z = zq[p, :V].astype(np.float64)
+            pr = np.exp(z - z.max()); pr /= pr.sum()
+            tok[n] = rng.choice(V, p=pr)
+    forest["token"] = tok
+    rp = rng.normal(0, 1, B).astype(np.float32)
+    rq = (rp + rng.normal(0, 0.5, B)).astype(np.float32)
+    prm = dict(V=V, temperature=0.9, thresh=0.6, W_min=1, W_max=max_w, W_nom=max_w, seed=5, step=0,
+               W_min_r=np.minimum(2, widths).astype(np.int32))
+    return forest, prm, zp, zq, rp, rq, stride
+
+
+@pytest.mark.parametrize("V,pad,ninf,tree", [(1023, 0, 0.0, "chain"), (1025, 3, 0.0, "chain"),
+                                             (4097, 0, 0.0, "binary"), (777, 1, 0.2, "chain"),
+                                             (3000, 0, 0.3, "binary"), (5, 0, 0.0, "chain")])
+def test_ragged_vocab_unaligned_rows_masked_entries(V, pad, ninf, tree):
+    rng = np.random.default_rng(V)
+    exempt = decisions = 0
+    for trial in range(6):
+        forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=5, V=V, gamma=3, max_w=4,
+                                                              stride_pad=pad, ninf_frac=ninf, tree=tree)
+        prm["step"] = trial
+        dz = lambda a: torch.as_tensor(a).cuda()
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq), row_stride=stride)
+        assert status == 0
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64),
+                                 row_stride=stride)
+        e, d = compare_verify(ref, gpu, forest)
+        exempt += e
+        decisions += d
+    check_exempt(exempt, decisions)
+
+
+def test_roots_only_forest_goes_straight_to_the_extra_layer():
+    rng = np.random.default_rng(3)
+    V, B = 2000, 3
+    forest = dict(R=1, B=B, N=B, max_depth=0, req_beam_off=np.array([0, B], np.int32),
+                  beam_node_off=np.arange(B + 1, dtype=np.int32), parent=np.full(B, -1, np.int32),
+                  token=np.zeros(B, np.int32))
+    zp = rng.normal(0, 2, size=(B, V)).astype(np.float32)
+    zq = rng.normal(0, 2, size=(B, V)).astype(np.float32)
+    rp = rng.normal(0, 1, B).astype(np.float32)
+    prm = dict(V=V, thresh=0.7, W_min=1, W_max=4, W_nom=4, seed=9)
+    exempt = decisions = 0
+    for step in range(20):
+        prm["step"] = step
+        dz = lambda a: torch.as_tensor(a).cuda()
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rp))
+        assert status == 0 and gpu["l_last"][0] == 1 and gpu["out_width"][0] == 4
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rp.astype(np.float64))
+        e, d = compare_verify(ref, gpu, forest)
+        exempt += e; decisions += d
+    check_exempt(exempt, decisions)
+
+
+def test_draft_rank_order_and_equal_models():
+    rng = np.random.default_rng(4)
+    forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=3, V=500, gamma=3, max_w=4, tree="binary")
+    # a draw order that disagrees with the node numbering
+    forest["draft_rank"] = rng.permutation(forest["N"]).astype(np.int32)
+    dz = lambda a: torch.as_tensor(a).cuda()
+    gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+    ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64))
+    assert status == 0
+    compare_verify(ref, gpu, forest)
+    # p == q: every draft up to the width is accepted
+    prm2 = dict(prm, W_min_r=None, W_min=1, W_max=64, W_nom=2)
+    gpu, status = run_gpu_verify(forest, prm2, dz(zp), dz(zp), dz(rp), dz(rp))
+    ref = oracle.verify_step(forest, prm2, zp, zp, rp.astype(np.float64), rp.astype(np.float64))
+    assert status == 0 and np.all(gpu["l_last"] == forest["max_depth"] + 1)
+    compare_verify(ref, gpu, forest)
+    assert not np.any(gpu["node_status"] == dsbd.binding.NODE_REJECTED)
+
+
+def test_bad_token_is_reported_not_trapped():
+    rng = np.random.default_rng(6)
+    forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=2, V=300, gamma=2, max_w=2)
+    forest["token"][forest["N"] - 1] = 300
+    dz = lambda a: torch.as_tensor(a).cuda()
+    gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+    assert status == 1          # DSBD_DEV_BAD_TOKEN
+
+
+def test_host_side_errors():
+    rng = np.random.default_rng(7)
+    forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=1, V=64, gamma=1, max_w=2)
+    f = dsbd.Forest(forest, "cuda")
+    out = dsbd.alloc_verify_out(f, oracle.default_out_off(forest, prm), "cuda")
+    dz = lambda a: torch.as_tensor(a).cuda()
+    prm_dev = dict(prm, W_min_r=None)
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(dsbd.DsbdError) as e:
+        dsbd.verify_step(f, prm_dev, dz(zp), dz(zq), dz(rp), dz(rq), out, workspace=small)
+    assert e.value.code == -3
+    with pytest.raises(dsbd.DsbdError) as e:
+        dsbd.verify_step(f, dict(prm_dev, temperature=0.0), dz(zp), dz(zq), dz(rp), dz(rq), out)
+    assert e.value.code == -1
+
+
+def test_select_width_matches_oracle():
+    rng = np.random.default_rng(8)
+    forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=4, V=3000, gamma=2, max_w=5)
+    prm = dict(prm, W_min_r=None)
+    rbo, bno = forest["req_beam_off"], forest["beam_node_off"]
+    live = [bno[rbo[r]:rbo[r + 1]] for r in range(forest["R"])]      # the roots
+    live_off = np.concatenate([[0], np.cumsum([len(x) for x in live])]).astype(np.int32)
+    live_nodes = np.concatenate(live).astype(np.int32)
+    m = np.array([len(x) for x in live], np.int32)
+    sp = rng.normal(0, 1, forest["N"]).astype(np.float32)
+    sq = rng.normal(0, 1, forest["N"]).astype(np.float32)
+    f = dsbd.Forest(forest, "cuda")
+    dz = lambda a: torch.as_tensor(a).cuda()
+    width, alpha, tail, status = dsbd.select_width(f, prm, dz(zp), dz(zq), dz(sp), dz(sq), dz(live_off),
+                                                   dz(live_nodes), dz(m), out_stride=8)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    w_ref, a_ref, t_ref = oracle.select_width(forest, prm, zp, zq, sp.astype(np.float64),
+                                              sq.astype(np.float64), live_off, live_nodes, m)
+    assert np.array_equal(width.cpu().numpy(), w_ref)
+    for r in range(forest["R"]):
+        assert np.abs(alpha[r, :m[r]].cpu().numpy() - a_ref[r, :m[r]]).max() < 2e-5
+        assert np.abs(tail[r, :m[r] + 1].cpu().numpy() - t_ref[r, :m[r] + 1]).max() < 2e-5
