@@ -1,0 +1,394 @@
+"""Benchmark of the DSBD hot path: one step = forest attention + verification step over one
+batch of synthetic input (configuration C5 by default: 64 requests x 8 beams x depth-8 chain
+drafts = 4608 forest nodes, 32 query / 8 KV heads x 128, bf16 KV prefix 4096 per beam, fp32
+logits over a 128256-token vocabulary).
+
+  python bench.py --gpus N --steps K --warmup W            the CUDA library
+  python bench.py --impl reference --steps K --warmup W    the CPU oracle on a bounded sample
+
+Prints ONE JSON line.  `value` = forest nodes verified per second with every input resident in
+HBM; `e2e` = the same through the C-ABI call with host buffers (pinned host -> device copies
+of the step's inputs and a device -> host read of its results inside the timed region).
+Multi-GPU: requests are independent, so each rank runs its own batch (weak scaling), with no
+data-path collective; time is the max over ranks.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified forest nodes/sec per decode step"
+UNIT = "nodes/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1] or [l for (_, l) in self.lines]
+        for line in rows:
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); mx.append(float(p[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def _cpu_baseline(data_host, spec, threads, budget_s=20.0):
+    """The oracle, as it stands, on a bounded sample of the workload: verification of a few
+    requests and attention of a few trees; returns nodes/s of the whole step extrapolated
+    from per-node times, and a description of the sample."""
+    import oracle
+    forest = data_host["forest"]
+    rbo, bno = forest["req_beam_off"], forest["beam_node_off"]
+    # verification: one request at a time until a third of the budget is used
+    n_ver, t_ver, reqs = 0, 0.0, 0
+    for r in range(forest["R"]):
+        sub = data_host["verify_sub"](r)
+        t0 = time.perf_counter()
+        oracle.verify_step(*sub, trace=False, threads=threads)
+        t_ver += time.perf_counter() - t0
+        n_ver += sub[0]["N"]
+        reqs += 1
+        if t_ver > budget_s / 2 or reqs >= data_host["max_reqs"]:
+            break
+    n_att, t_att, beams = 0, 0.0, 0
+    for b in range(forest["B"]):
+        sub = data_host["attn_sub"](b)
+        t0 = time.perf_counter()
+        oracle.forest_attention(*sub, threads=threads)
+        t_att += time.perf_counter() - t0
+        n_att += sub[0]["N"]
+        beams += 1
+        if t_att > budget_s / 2 or beams >= data_host["max_beams"]:
+            break
+    per_node = t_ver / n_ver + t_att / n_att
+    return {"value": 1.0 / per_node, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "%d of %d requests verified (%.1f s), attention of %d of %d trees (%.1f s); "
+                      "nodes/s = 1 / (verify s/node + attention s/node)" % (
+                          reqs, forest["R"], t_ver, beams, forest["B"], t_att)}
+
+
+def _host_views(data, spec):
+    """Closures that cut per-request / per-tree oracle inputs out of the device tensors."""
+    import torch
+    forest, prm, poff = data["forest"], data["params"], data["prefix_off"]
+    rbo, bno = forest["req_beam_off"], forest["beam_node_off"]
+    Hkv, d = spec["Hkv"], spec["d"]
+    h = lambda x: x.detach().float().cpu().numpy()
+
+    def sub_tree_forest(b_lo, b_hi):
+        n0, n1 = int(bno[b_lo]), int(bno[b_hi])
+        par = forest["parent"][n0:n1]
+        return dict(R=1, B=b_hi - b_lo, N=n1 - n0, max_depth=forest["max_depth"],
+                    req_beam_off=np.array([0, b_hi - b_lo], np.int32),
+                    beam_node_off=(bno[b_lo:b_hi + 1] - n0).astype(np.int32),
+                    parent=np.where(par >= 0, par - n0, -1).astype(np.int32),
+                    token=forest["token"][n0:n1].astype(np.int32)), n0, n1
+
+    def verify_sub(r):
+        f, n0, n1 = sub_tree_forest(int(rbo[r]), int(rbo[r + 1]))
+        p = dict(prm, W_min_r=np.asarray(prm["W_min_r"])[r:r + 1], req_id=np.array([r], np.int32))
+        return (f, p, h(data["logits_p"][n0:n1]), h(data["logits_q"][n0:n1]),
+                h(data["root_logp"][rbo[r]:rbo[r + 1]]).astype(np.float64),
+                h(data["root_logq"][rbo[r]:rbo[r + 1]]).astype(np.float64))
+
+    def attn_sub(b):
+        f, n0, n1 = sub_tree_forest(b, b + 1)
+        s, e = int(poff[b]) * Hkv * d, int(poff[b + 1]) * Hkv * d
+        return (f, spec["Hq"], Hkv, d, 1.0 / np.sqrt(d), h(data["q"][n0:n1]), h(data["k_new"][n0:n1]),
+                h(data["v_new"][n0:n1]), h(data["k_prefix"][s:e]), h(data["v_prefix"][s:e]),
+                np.array([0, poff[b + 1] - poff[b]], np.int64))
+
+    return dict(forest=forest, verify_sub=verify_sub, attn_sub=attn_sub, max_reqs=8, max_beams=8)
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2409_16560_b200 import inputs
+    spec = inputs.config(args.workload)
+    # a slice of the workload is enough for the sample: fewer requests, same shapes
+    small = dict(spec, R=min(spec["R"], 2))
+    data = inputs.generate(small, "cpu")
+    views = _host_views(data, small)
+    views["max_reqs"], views["max_beams"] = 1, 1
+    threads = os.cpu_count() or 1
+    for _ in range(args.warmup):
+        _cpu_baseline(views, small, threads, budget_s=1e9)
+    t0 = time.perf_counter()
+    vals = [_cpu_baseline(views, small, threads, budget_s=1e9) for _ in range(args.steps)]
+    dt = time.perf_counter() - t0
+    value = float(np.mean([v["value"] for v in vals]))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": args.workload, "sample": vals[-1]["sample"]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": vals[-1]["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="dsbd", choices=["dsbd", "reference"])
+    ap.add_argument("--workload", default="C5")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2409_16560_b200 as dsbd
+    from paper_2409_16560_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    dsbd.load()
+
+    spec = inputs.config(args.workload)
+    spec["seed"] = spec["seed"] + 1000 * rank            # every rank verifies its own requests
+    data = inputs.generate(spec, dev)
+    forest, prm, poff = data["forest"], dict(data["params"]), data["prefix_off"]
+    f = dsbd.Forest(forest, dev)
+    prm_dev = dict(prm, W_min_r=torch.as_tensor(prm["W_min_r"]).to(dev))
+    out_off = dsbd.default_out_off(forest, prm)
+    vout = dsbd.alloc_verify_out(f, out_off, dev)
+    poff_dev = torch.as_tensor(poff).to(dev)
+    scale = inputs.default_scale(spec["d"])
+    attn_out = torch.empty_like(data["q"])
+    ws_a = torch.empty(max(dsbd.forest_attention_workspace(f, spec["Hq"], spec["Hkv"], spec["d"],
+                                                           data["q"].dtype, scale, poff), 256),
+                       dtype=torch.uint8, device=dev)
+    ws_v = torch.empty(max(dsbd.verify_workspace(f, prm_dev), 256), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    lse_p = torch.empty(f.N, dtype=torch.float32, device=dev)
+    lse_q = torch.empty(f.N, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def attention():
+        dsbd.forest_attention(f, spec["Hq"], spec["Hkv"], spec["d"], scale, data["q"], data["k_new"],
+                              data["v_new"], data["k_prefix"], data["v_prefix"], poff_dev, poff,
+                              out=attn_out, workspace=ws_a, status=status, stream=stream)
+
+    def verify(step):
+        prm_dev["step"] = step
+        dsbd.verify_step(f, prm_dev, data["logits_p"], data["logits_q"], data["root_logp"],
+                         data["root_logq"], vout, workspace=ws_v, status=status, stream=stream)
+
+    def one_step(step):
+        attention()
+        verify(step)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for s in range(args.warmup):
+        one_step(s)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4 * args.steps + 1)]
+    t_wall0 = time.time()
+    barrier()
+    ev[0].record(stream)
+    e_attn, e_ver = [], []
+    for s in range(args.steps):
+        a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
+        a2 = torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        attention()
+        a1.record(stream)
+        verify(args.warmup + s)
+        a2.record(stream)
+        e_attn.append((a0, a1)); e_ver.append((a1, a2))
+    ev[1].record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    total_ms = ev[0].elapsed_time(ev[1])
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in e_attn]))
+    ver_ms = float(np.mean([a.elapsed_time(b) for a, b in e_ver]))
+    assert int(status.item()) == 0, "device status %d" % int(status.item())
+
+    # the dense logits pass alone (the kernel the verify roofline is quoted on)
+    torch.cuda.synchronize()
+    d0 = torch.cuda.Event(enable_timing=True); d1 = torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        dsbd.node_stats(f, prm_dev, data["logits_p"], data["logits_q"], lse_p, lse_q, workspace=ws_v, stream=stream)
+    n_dense = max(args.steps, 5)
+    d0.record(stream)
+    for _ in range(n_dense):
+        dsbd.node_stats(f, prm_dev, data["logits_p"], data["logits_q"], lse_p, lse_q, workspace=ws_v, stream=stream)
+    d1.record(stream)
+    torch.cuda.synchronize()
+    dense_ms = d0.elapsed_time(d1) / n_dense
+
+    # end to end through the C ABI with host buffers
+    e2e = None
+    if args.e2e_steps > 0:
+        names = ["q", "k_new", "v_new", "k_prefix", "v_prefix", "logits_p", "logits_q", "root_logp", "root_logq"]
+        host = {k: data[k].cpu().pin_memory() for k in names}
+        host_forest = {k: torch.from_numpy(np.ascontiguousarray(forest[k], dtype=np.int32)).pin_memory()
+                       for k in ("req_beam_off", "beam_node_off", "parent", "token")}
+        h2d = sum(v.numel() * v.element_size() for v in host.values()) + \
+            sum(v.numel() * v.element_size() for v in host_forest.values())
+        res_keys = ["l_last", "out_width", "out_parent", "out_node", "out_root_beam", "out_token", "out_logp",
+                    "out_logq", "out_source", "node_status", "layer_width"]
+        host_res = {k: torch.empty_like(vout[k], device="cpu").pin_memory() for k in res_keys}
+        host_attn = torch.empty_like(attn_out, device="cpu").pin_memory()
+        d2h = sum(v.numel() * v.element_size() for v in host_res.values()) + host_attn.numel() * host_attn.element_size()
+
+        def e2e_step(step):
+            for k in names:
+                data[k].copy_(host[k], non_blocking=True)
+            for k, v in host_forest.items():
+                f.dev[k].copy_(v, non_blocking=True)
+            one_step(step)
+            host_attn.copy_(attn_out, non_blocking=True)
+            for k in res_keys:
+                host_res[k].copy_(vout[k], non_blocking=True)
+
+        e2e_step(0)
+        barrier()
+        s0 = torch.cuda.Event(enable_timing=True); s1 = torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for s in range(args.e2e_steps):
+            e2e_step(s + 1)
+        s1.record(stream)
+        barrier()
+        te = torch.tensor([s0.elapsed_time(s1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e = {"value": f.N * world * args.e2e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps}
+        del host
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    a_bytes = inputs.attention_bytes(spec, forest, poff)
+    v_bytes = inputs.verify_bytes(spec, forest)
+    kernels = {
+        "forest_attention": {"bytes": a_bytes, "ms": attn_ms, "gbs": a_bytes / attn_ms * 1e-6},
+        "verify_dense_pass": {"bytes": v_bytes, "ms": dense_ms, "gbs": v_bytes / dense_ms * 1e-6},
+        "verify_step_total": {"bytes": v_bytes, "ms": ver_ms, "gbs": v_bytes / ver_ms * 1e-6},
+    }
+    for k in kernels.values():
+        k["frac_of_%s_peak" % peak_kind] = k["gbs"] / peak
+        k["frac_of_8TBs_nominal"] = k["gbs"] / 8000.0
+    dom = "forest_attention" if attn_ms >= dense_ms else "verify_dense_pass"
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak,
+                "traffic": None}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            roofline["traffic"] = json.load(open(prof)).get(args.workload, {}).get(dom)
+        except (ValueError, OSError):
+            pass
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = _cpu_baseline(_host_views(data, spec), spec, os.cpu_count() or 1)
+
+    ms_per_step = total_ms / args.steps
+    line = {"metric": METRIC, "value": f.N * world / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 attention / f32 logits", "data": "synthetic",
+            "config": {"workload": args.workload, "requests": f.R, "beams": f.B, "nodes": f.N,
+                       "heads": "%dq/%dkv x %d" % (spec["Hq"], spec["Hkv"], spec["d"]), "vocab": spec["V"],
+                       "prefix": list(spec["prefix"]), "temperature": spec["temperature"],
+                       "thresh": prm["thresh"], "l2": "inputs (%.1f GB) far exceed the 126 MB L2; no flush" % (
+                           (a_bytes + v_bytes) * 1e-9),
+                       "parallelism": "replicas x%d" % world},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * args.steps,
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

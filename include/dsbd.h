@@ -180,6 +180,16 @@ int dsbd_verify_step(const dsbd_forest_t *forest, const dsbd_verify_params_t *pa
 
 size_t dsbd_verify_workspace(const dsbd_forest_t *forest, const dsbd_verify_params_t *params);
 
+/* Step 1 of dsbd_verify_step on its own: the large and the small model's next-token
+ * distribution of every node (Overview: "predict the distribution for the next token of each
+ * node in parallel"), returned as the log-sum-exp of each tempered logits row,
+ * lse_p[n] = log sum_v exp(logits_p[n,v]/tau), lse_q likewise ([N] each).  One dense pass over
+ * both logits tensors; workspace as for dsbd_verify_step. */
+int dsbd_node_stats(const dsbd_forest_t *forest, const dsbd_verify_params_t *params,
+                    const float *logits_p, const float *logits_q, int64_t row_stride,
+                    float *lse_p, float *lse_q, void *workspace, size_t workspace_bytes,
+                    dsbd_stream_t stream);
+
 /* The context-dependent width of ONE layer (Eqs. for P(m,k), P~(m,i), alpha_j and
  * W_L^(l) = max(W_min, W~_L^(l)(t)), capped by W_max) for a given live set: request r's live
  * parents are live_nodes[live_off[r] .. live_off[r+1]) (ascending node ids) with cumulative

@@ -20,7 +20,7 @@ MAX_TREE_NODES = 64
 MAX_LIVE = 64
 
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_verify_step",
-           "dsbd_verify_workspace", "dsbd_select_width", "dsbd_status_string"]
+           "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_status_string"]
 
 _vp = C.c_void_p
 
@@ -81,6 +81,8 @@ def load():
     lib.dsbd_verify_step.restype = C.c_int
     lib.dsbd_verify_step.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_size_t,
                                      _vp, _vp]
+    lib.dsbd_node_stats.restype = C.c_int
+    lib.dsbd_node_stats.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_size_t, _vp]
     lib.dsbd_select_width.restype = C.c_int
     lib.dsbd_select_width.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, _vp,
                                       _vp, _vp, C.c_int32, _vp, C.c_size_t, _vp, _vp]
@@ -226,6 +228,22 @@ def verify_workspace(forest, params):
     return int(load().dsbd_verify_workspace(C.addressof(f), C.addressof(p)))
 
 
+def default_out_off(arrays, params):
+    """Output slot ranges that hold any outcome: max(W_nom, W_min, min(W_max, nodes)) per request."""
+    R = int(arrays["R"])
+    nodes = np.diff(np.asarray(arrays["beam_node_off"])[np.asarray(arrays["req_beam_off"])])
+
+    def per_request(name, default):
+        v = params.get(name + "_r")
+        if v is not None:
+            return np.asarray(v.cpu() if torch.is_tensor(v) else v, dtype=np.int64)
+        return np.full(R, int(params.get(name, default)), dtype=np.int64)
+
+    cap = np.maximum(np.maximum(per_request("W_nom", 1), per_request("W_min", 1)),
+                     np.minimum(per_request("W_max", 1 << 30), nodes))
+    return np.concatenate([[0], np.cumsum(cap)]).astype(np.int32)
+
+
 def alloc_verify_out(forest, out_off_host, device):
     """Output buffers of dsbd_verify_step as a dict of device tensors."""
     R, N, g = forest.R, forest.N, forest.max_depth
@@ -276,6 +294,28 @@ def verify_step(forest, params, logits_p, logits_q, root_logp, root_logq, out, w
     if rc != OK:
         raise DsbdError("dsbd_verify_step", rc)
     return status
+
+
+def node_stats(forest, params, logits_p, logits_q, lse_p=None, lse_q=None, workspace=None, stream=None):
+    """dsbd_node_stats; returns (lse_p[N], lse_q[N])."""
+    _require_cuda(logits_p, logits_q)
+    keep = []
+    f = forest.struct()
+    p = _params(params, keep)
+    dev = logits_p.device
+    if lse_p is None:
+        lse_p = torch.empty(forest.N, dtype=torch.float32, device=dev)
+    if lse_q is None:
+        lse_q = torch.empty(forest.N, dtype=torch.float32, device=dev)
+    need = int(load().dsbd_verify_workspace(C.addressof(f), C.addressof(p)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    rc = load().dsbd_node_stats(C.addressof(f), C.addressof(p), _ptr(logits_p), _ptr(logits_q),
+                                logits_p.stride(0), _ptr(lse_p), _ptr(lse_q), _ptr(workspace),
+                                workspace.numel(), _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_node_stats", rc)
+    return lse_p, lse_q
 
 
 def select_width(forest, params, logits_p, logits_q, node_logp, node_logq, live_off, live_nodes, m,

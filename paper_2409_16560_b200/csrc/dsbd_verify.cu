@@ -919,6 +919,34 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
     return launch_verify(a, f->R, L.max_live * L.T, stream);
 }
 
+extern "C" int dsbd_node_stats(const dsbd_forest_t *f, const dsbd_verify_params_t *p,
+                               const float *logits_p, const float *logits_q, int64_t row_stride,
+                               float *lse_p, float *lse_q, void *workspace, size_t workspace_bytes,
+                               dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    int rc = check_forest(f);
+    if (rc) return rc;
+    rc = check_params(p);
+    if (rc) return rc;
+    if (!logits_p || !logits_q || !lse_p || !lse_q || !workspace || row_stride < p->V)
+        return DSBD_ERR_INVALID_ARG;
+    const Layout L = make_layout(f, p->V);
+    if (workspace_bytes < L.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    TileStat *stats = reinterpret_cast<TileStat *>(ws + L.stats);
+    double *lse = reinterpret_cast<double *>(ws + L.lse);
+    const double inv_tau = 1.0 / (double)p->temperature;
+    const float k2 = (float)((double)kLog2e * inv_tau);
+    const int64_t items = (int64_t)2 * f->N * L.T;
+    k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_p, logits_q, row_stride, p->V, L.T,
+                                                            f->N, f->N, nullptr, nullptr, k2, stats);
+    const int64_t warps = (int64_t)2 * f->N;
+    k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
+        stats, L.T, f->N, f->N, nullptr, nullptr, inv_tau, lse, lse_p, lse_q);
+    return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
+
 extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_params_t *p,
                                  const float *logits_p, const float *logits_q, int64_t row_stride,
                                  const float *node_logp, const float *node_logq,
