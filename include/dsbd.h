@@ -190,6 +190,29 @@ int dsbd_node_stats(const dsbd_forest_t *forest, const dsbd_verify_params_t *par
                     float *lse_p, float *lse_q, void *workspace, size_t workspace_bytes,
                     dsbd_stream_t stream);
 
+/* dsbd_node_stats for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a property of the library, not of the method.)  Some callers have no
+ * way to hand over a workspace: a plug-in that runs after its host process has given every
+ * byte of device memory to the host's own pool, or a latency-critical section that must not
+ * call cudaMalloc because cudaMalloc synchronises the whole device.  For them the scratch of
+ * the two kernels lives in a fixed array of DSBD_STATIC_SCRATCH_BYTES inside the library
+ * image; every GPU that loads the library holds that array until the process exits.
+ *   - Same inputs, outputs and results as dsbd_node_stats; the call allocates and frees
+ *     nothing and calls no routine that does.
+ *   - Limit: 8*2*N*ceil(V/1024) bytes (rounded up to 256) + 16*N bytes must fit into
+ *     DSBD_STATIC_SCRATCH_BYTES, e.g. about 4100 rows of a 128256-token vocabulary; larger problems
+ *     are refused with DSBD_ERR_WORKSPACE_TOO_SMALL and nothing is launched.
+ *   - The first call on a device looks up the device address of the array (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array, which still holds what the last call left in it.  The
+ *     kernels overwrite every entry before they read it, so nothing needs clearing, but two
+ *     calls that overlap on the GPU (different streams, or several host threads) race on it:
+ *     serialise them. */
+#define DSBD_STATIC_SCRATCH_BYTES (8u << 20)
+int dsbd_node_stats_static(const dsbd_forest_t *forest, const dsbd_verify_params_t *params,
+                           const float *logits_p, const float *logits_q, int64_t row_stride,
+                           float *lse_p, float *lse_q, dsbd_stream_t stream);
+
 /* The context-dependent width of ONE layer (Eqs. for P(m,k), P~(m,i), alpha_j and
  * W_L^(l) = max(W_min, W~_L^(l)(t)), capped by W_max) for a given live set: request r's live
  * parents are live_nodes[live_off[r] .. live_off[r+1]) (ascending node ids) with cumulative

@@ -20,7 +20,8 @@ MAX_TREE_NODES = 64
 MAX_LIVE = 64
 
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_verify_step",
-           "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_status_string"]
+           "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
+           "dsbd_status_string"]
 
 _vp = C.c_void_p
 
@@ -83,6 +84,8 @@ def load():
                                      _vp, _vp]
     lib.dsbd_node_stats.restype = C.c_int
     lib.dsbd_node_stats.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_size_t, _vp]
+    lib.dsbd_node_stats_static.restype = C.c_int
+    lib.dsbd_node_stats_static.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp]
     lib.dsbd_select_width.restype = C.c_int
     lib.dsbd_select_width.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, _vp,
                                       _vp, _vp, C.c_int32, _vp, C.c_size_t, _vp, _vp]
@@ -315,6 +318,26 @@ def node_stats(forest, params, logits_p, logits_q, lse_p=None, lse_q=None, works
                                 workspace.numel(), _stream(stream))
     if rc != OK:
         raise DsbdError("dsbd_node_stats", rc)
+    return lse_p, lse_q
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def node_stats_static(forest, params, logits_p, logits_q, lse_p, lse_q, stream=None):
+    """dsbd_node_stats_static: dsbd_node_stats without a workspace, for callers that cannot
+    allocate device memory; the outputs lse_p, lse_q ([N] fp32 each) are the caller's.  The
+    binding itself allocates nothing either.  Problems that need more than
+    STATIC_SCRATCH_BYTES of scratch raise DsbdError (workspace too small).  Calls share one
+    scratch array per GPU: do not let two of them overlap on the device."""
+    _require_cuda(logits_p, logits_q, lse_p, lse_q)
+    keep = []
+    f = forest.struct()
+    p = _params(params, keep)
+    rc = load().dsbd_node_stats_static(C.addressof(f), C.addressof(p), _ptr(logits_p), _ptr(logits_q),
+                                       logits_p.stride(0), _ptr(lse_p), _ptr(lse_q), _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_node_stats_static", rc)
     return lse_p, lse_q
 
 

@@ -947,6 +947,65 @@ extern "C" int dsbd_node_stats(const dsbd_forest_t *f, const dsbd_verify_params_
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------------
+// dsbd_node_stats_static: the same two kernels as dsbd_node_stats, with their scratch (tile
+// statistics and double-precision row sums) in a fixed array that is part of the library image
+// instead of a caller-supplied workspace.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[DSBD_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char *g_static_scratch_ptr[kMaxDevices];   // device address of the array, per device
+
+// The array's name is only a host-side handle; the device address a kernel can use has to be
+// asked for, once per device, while that device is current.
+int static_scratch_address(unsigned char **ptr) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DSBD_ERR_CUDA;
+    unsigned char *p = __atomic_load_n(&g_static_scratch_ptr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        void *addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return DSBD_ERR_CUDA;
+        p = static_cast<unsigned char *>(addr);
+        __atomic_store_n(&g_static_scratch_ptr[dev], p, __ATOMIC_RELEASE);
+    }
+    *ptr = p;
+    return DSBD_OK;
+}
+}  // namespace
+
+extern "C" int dsbd_node_stats_static(const dsbd_forest_t *f, const dsbd_verify_params_t *p,
+                                      const float *logits_p, const float *logits_q, int64_t row_stride,
+                                      float *lse_p, float *lse_q, dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    int rc = check_forest(f);
+    if (rc) return rc;
+    rc = check_params(p);
+    if (rc) return rc;
+    if (!logits_p || !logits_q || !lse_p || !lse_q || row_stride < p->V) return DSBD_ERR_INVALID_ARG;
+    // scratch this call needs: tile statistics of both models, then the double row sums
+    const int T = (p->V + kTile - 1) / kTile;
+    const size_t stats_bytes = align_up(sizeof(TileStat) * 2 * (size_t)f->N * T, 256);
+    const size_t need = stats_bytes + sizeof(double) * 2 * (size_t)f->N;
+    if (need > (size_t)DSBD_STATIC_SCRATCH_BYTES) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    unsigned char *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    // Nothing here has to start from zero: both kernels overwrite every entry they later read.
+    TileStat *stats = reinterpret_cast<TileStat *>(scratch);
+    double *lse = reinterpret_cast<double *>(scratch + stats_bytes);
+    const double inv_tau = 1.0 / (double)p->temperature;
+    const float k2 = (float)((double)kLog2e * inv_tau);
+    const int64_t items = (int64_t)2 * f->N * T;
+    k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_p, logits_q, row_stride, p->V, T,
+                                                            f->N, f->N, nullptr, nullptr, k2, stats);
+    const int64_t warps = (int64_t)2 * f->N;
+    k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
+        stats, T, f->N, f->N, nullptr, nullptr, inv_tau, lse, lse_p, lse_q);
+    return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
+
 extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_params_t *p,
                                  const float *logits_p, const float *logits_q, int64_t row_stride,
                                  const float *node_logp, const float *node_logq,
