@@ -11,7 +11,10 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
-#include "dsbd_common.cuh"
+#include <stdlib.h>
+#include <string.h>
+
+#include "dsbd_attention.cuh"
 
 using namespace dsbd;
 
@@ -238,6 +241,11 @@ extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_des
                            reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(k_prefix) |
                            reinterpret_cast<uintptr_t>(v_prefix) | reinterpret_cast<uintptr_t>(out);
     if (bits & 15) return DSBD_ERR_UNSUPPORTED;
+
+    // DSBD_ATTN_IMPL=simt forces the CUDA-core kernel (debugging aid)
+    const char *impl = getenv("DSBD_ATTN_IMPL");
+    if (!(impl && strcmp(impl, "simt") == 0) && attention_tc_supported(f, d))
+        return launch_attention_tc(f, d, q, k_new, v_new, k_prefix, v_prefix, prefix_off, out, status, stream);
 
     AttnArgs a = {};
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;

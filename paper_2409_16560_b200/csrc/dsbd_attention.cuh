@@ -1,0 +1,16 @@
+// Internal interface between the attention entry point and its tensor-core kernel.
+#pragma once
+
+#include "dsbd_common.cuh"
+
+namespace dsbd {
+
+// True when the tcgen05 kernel covers this problem (bf16, d = 128, at most 128 query rows and
+// 64 nodes per tree, a non-empty KV prefix).
+bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
+
+int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
+                        const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
+                        void *out, int32_t *status, cudaStream_t stream);
+
+}  // namespace dsbd

@@ -1,0 +1,492 @@
+// Forest attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16, d = 128.
+//
+// Work unit = (beam, KV head): all query rows of the beam's draft tree that map to this KV head
+// (row = node * group + head, at most 128) against the beam's KV prefix, streamed once in
+// 64-token tiles, followed by one tile holding the tree's own keys/values under the
+// ancestor-or-self mask.
+//
+// CTA = 6 warps, two CTAs per SM:
+//   warps 0-3  softmax: warp w owns TMEM lanes 32w..32w+31 = query rows 32w..32w+31, one row per
+//              thread, so row max / row sum are thread-local.  They also stage Q (swizzled, by
+//              hand) at the start of a unit and write O at its end.
+//   warp 4     TMA producer: K and V tiles (2 x 64x64 bf16 boxes each, 128-byte swizzle) into a
+//              ring of shared-memory stages, completion on mbarriers.
+//   warp 5     MMA issuer (one lane): S = Q K^T (M128 N64 K16 x 8, both operands K-major in
+//              shared memory) into TMEM; after the softmax warps have written P (bf16) to TMEM,
+//              O += P V (A from TMEM, B = the V tile as an MN-major shared-memory operand).
+// O stays in TMEM for the whole unit; its rows are rescaled only when a row maximum grows by
+// more than 2^8 (the rescale is a TMEM load/scale/store by the row's own thread).
+// Every mbarrier wait is bounded; on a time-out the kernel records DSBD_DEV_TIMEOUT, lets its
+// copies land, frees its TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "dsbd_attention.cuh"
+
+using namespace dsbd;
+
+namespace {
+
+constexpr int kD = 128;                 // head dim
+constexpr int kBN = 64;                 // tokens per tile
+constexpr int kStages = 2;
+constexpr int kRows = 128;              // UMMA M
+constexpr int kThreadsTc = 192;
+constexpr uint32_t kQBytes = kRows * kD * 2;          // 32 KB: two 128-row x 128-byte halves
+constexpr uint32_t kTileBytes = kBN * kD * 2;         // 16 KB per K or V tile (two 8 KB boxes)
+constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K then V
+constexpr uint32_t kSmemBytes = 1024 + kQBytes + kStages * kStageBytes;
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColP = 64, kColO = 128;
+constexpr long long kWaitCycles = 2000000000ll;   // about a second
+
+struct TcArgs {
+    int B, N, Hq, Hkv, group, n_units;
+    float scale_log2;
+    const int32_t *beam_node_off, *parent;
+    const int64_t *prefix_off;
+    const __nv_bfloat16 *q;
+    __nv_bfloat16 *out;
+    int32_t *status;
+};
+
+struct Barriers {
+    unsigned long long kv_full[kStages], kv_empty[kStages], s_full, p_full, q_full, o_full;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(void *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(void *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try(void *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if it gave up (time-out here, or another role already aborted).
+__device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, Barriers *sb, int32_t *status) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if (*reinterpret_cast<volatile int *>(&sb->abort)) return false;
+        if (clock64() - t0 > kWaitCycles) break;
+    }
+    *reinterpret_cast<volatile int *>(&sb->abort) = 1;
+    report(status, DSBD_DEV_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, void *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(void *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
+        "%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+        "%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (128-byte swizzle, 8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t saddr) {
+    // leading offset unused for swizzled K-major (1), stride offset 1024 B, version 1, SWIZZLE_128B
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t desc_mn_major(uint32_t saddr, uint32_t lbo_bytes) {
+    // leading offset = distance between 64-element groups along N, stride offset = 8 k-rows
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+__global__ void __launch_bounds__(kThreadsTc, 2)
+k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_constant__ CUtensorMap map_vp,
+                 const __grid_constant__ CUtensorMap map_kn, const __grid_constant__ CUtensorMap map_vn,
+                 TcArgs a) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ Barriers sb;
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char *q_s = smem;                               // [2 halves][128 rows][128 B], swizzled
+    unsigned char *stage_s = smem + kQBytes;                 // [stages][K 16 KB | V 16 KB]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sb.kv_full[s], 1); mbar_init(&sb.kv_empty[s], 1); }
+        mbar_init(&sb.s_full, 1);
+        mbar_init(&sb.p_full, 4);
+        mbar_init(&sb.q_full, 128);
+        mbar_init(&sb.o_full, 1);
+        sb.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sb.tmem_base)),
+                     "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&sb.tmem_base);
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t tile = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+                const int b = u / a.Hkv, g = u - b * a.Hkv;
+                const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
+                const int64_t row0 = a.prefix_off[b] * a.Hkv + (int64_t)g * L;
+                const int nt_p = (int)((L + kBN - 1) / kBN);
+                const int n_lo = a.beam_node_off[b];
+                for (int j = 0; j <= nt_p && ok; ++j, ++tile) {
+                    const int s = tile % kStages;
+                    const uint32_t par = (tile / kStages) & 1;
+                    ok = mbar_wait(&sb.kv_empty[s], par ^ 1, &sb, a.status);
+                    if (!ok) break;
+                    unsigned char *ks = stage_s + s * kStageBytes, *vs = ks + kTileBytes;
+                    mbar_expect_tx(&sb.kv_full[s], kStageBytes);
+                    if (j < nt_p) {
+                        const int y = (int)(row0 + (int64_t)j * kBN);
+                        tma_load_2d(ks, &map_kp, 0, y, &sb.kv_full[s]);
+                        tma_load_2d(ks + kTileBytes / 2, &map_kp, 64, y, &sb.kv_full[s]);
+                        tma_load_2d(vs, &map_vp, 0, y, &sb.kv_full[s]);
+                        tma_load_2d(vs + kTileBytes / 2, &map_vp, 64, y, &sb.kv_full[s]);
+                    } else {
+                        const int x = g * kD;
+                        tma_load_2d(ks, &map_kn, x, n_lo, &sb.kv_full[s]);
+                        tma_load_2d(ks + kTileBytes / 2, &map_kn, x + 64, n_lo, &sb.kv_full[s]);
+                        tma_load_2d(vs, &map_vn, x, n_lo, &sb.kv_full[s]);
+                        tma_load_2d(vs + kTileBytes / 2, &map_vn, x + 64, n_lo, &sb.kv_full[s]);
+                    }
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA goes away
+                for (uint32_t k = 0; k < (uint32_t)kStages && k < tile; ++k) {
+                    const uint32_t t = tile - 1 - k;
+                    const long long t0 = clock64();
+                    while (!mbar_try(&sb.kv_full[t % kStages], (t / kStages) & 1))
+                        if (clock64() - t0 > kWaitCycles) break;
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(kRows, kBN, 0);
+            constexpr uint32_t idesc_o = instr_desc(kRows, kD, 1);
+            uint32_t tile = 0, unit = 0;
+            bool ok = true;
+            const uint64_t qd = desc_k_major(smem_u32(q_s));
+            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++unit) {
+                const int b = u / a.Hkv;
+                const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
+                const int nt = (int)((L + kBN - 1) / kBN) + 1;
+                ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
+                for (int j = 0; j < nt && ok; ++j, ++tile) {
+                    const int s = tile % kStages;
+                    ok = mbar_wait(&sb.kv_full[s], (tile / kStages) & 1, &sb, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t k_addr = smem_u32(stage_s + s * kStageBytes);
+                    const uint64_t kd = desc_k_major(k_addr);
+#pragma unroll
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint64_t ad = qd + (uint64_t)((ks / 4) * ((kRows * 128) >> 4) + (ks % 4) * 2);
+                        const uint64_t bd = kd + (uint64_t)((ks / 4) * ((kBN * 128) >> 4) + (ks % 4) * 2);
+                        mma_ss(tmem + kColS, ad, bd, idesc_s, ks > 0);
+                    }
+                    tc_commit(&sb.s_full);
+                    ok = mbar_wait(&sb.p_full, tile & 1, &sb, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t vd = desc_mn_major(k_addr + kTileBytes, kBN * 128);
+#pragma unroll
+                    for (int ks = 0; ks < kBN / 16; ++ks)
+                        mma_ts(tmem + kColO, tmem + kColP + ks * 8, vd + (uint64_t)(ks * ((16 * 128) >> 4)), idesc_o,
+                               (j > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(&sb.kv_empty[s]);
+                }
+                if (ok) tc_commit(&sb.o_full);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warps
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        uint32_t tile = 0, unit = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++unit) {
+            const int b = u / a.Hkv, g = u - b * a.Hkv;
+            const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
+            const int nt_p = (int)((L + kBN - 1) / kBN);
+            const int n_lo = a.beam_node_off[b];
+            const int n_tree = a.beam_node_off[b + 1] - n_lo;
+            const int M = n_tree * a.group;
+            const bool warp_active = warp * 32 < M;
+            const bool active = row < M;
+            const int node = active ? row / a.group : 0;
+            const int hq = g * a.group + (active ? row - node * a.group : 0);
+            // ---- stage Q (rows >= M zero) and the ancestor masks; the previous unit's MMAs are done
+            {
+                const int t128 = threadIdx.x;                        // 0..127
+                for (int i = t128; i < kRows * 16; i += 128) {
+                    const int r = i >> 4, c = i & 15;                // row, 16-byte chunk of the 256-byte row
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (r < M) {
+                        const int nd = r / a.group, hh = g * a.group + (r - nd * a.group);
+                        v = *reinterpret_cast<const uint4 *>(a.q + ((int64_t)(n_lo + nd) * a.Hq + hh) * kD + c * 8);
+                    }
+                    const int half = c >> 3, cc = c & 7;
+                    *reinterpret_cast<uint4 *>(q_s + half * (kRows * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&sb.q_full);
+            }
+            // ancestor-or-self mask of this row's node: walk up the tree
+            unsigned long long my_anc = 0;
+            {
+                int n = node;
+                for (int hop = 0; hop < DSBD_MAX_TREE_NODES && n >= 0 && n < n_tree; ++hop) {
+                    my_anc |= 1ull << n;
+                    const int par = a.parent[n_lo + n];
+                    if (par >= n_lo + n) { report(a.status, DSBD_DEV_BAD_FOREST); break; }
+                    n = par < 0 ? -1 : par - n_lo;
+                }
+            }
+            float m_ref = -INFINITY, l_run = 0.f;
+            for (int j = 0; j <= nt_p && ok; ++j, ++tile) {
+                ok = mbar_wait(&sb.s_full, tile & 1, &sb, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                if (warp_active) {
+                    uint32_t sv[2][32];
+                    tmem_ld32(tmem + lane_base + kColS, sv[0]);
+                    tmem_ld32(tmem + lane_base + kColS + 32, sv[1]);
+                    tmem_wait_ld();
+                    float mx = -INFINITY;
+                    const bool tree = (j == nt_p);
+                    // visibility of the tile's 64 tokens for this row, as a bit mask
+                    unsigned long long vis;
+                    if (tree) vis = my_anc & (n_tree >= 64 ? ~0ull : ((1ull << n_tree) - 1));
+                    else {
+                        const int64_t left = L - (int64_t)j * kBN;
+                        vis = left >= 64 ? ~0ull : ((1ull << left) - 1);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) {
+                        const float xv = ((vis >> c) & 1ull) ? __uint_as_float(sv[c >> 5][c & 31]) * a.scale_log2
+                                                             : -INFINITY;
+                        sv[c >> 5][c & 31] = __float_as_uint(xv);
+                        mx = fmaxf(mx, xv);
+                    }
+                    // lazy rescale: move the reference only when some row of the warp needs it
+                    const bool need = mx > m_ref + 8.f;
+                    if (__any_sync(kFull, need)) {
+                        const float m_new = need ? mx : m_ref;
+                        const float f = (m_ref == -INFINITY) ? 0.f : exp2f(m_ref - m_new);
+                        l_run *= f;
+                        if (j > 0) {
+#pragma unroll
+                            for (int cc = 0; cc < 4; ++cc) {
+                                uint32_t ov[32];
+                                tmem_ld32(tmem + lane_base + kColO + cc * 32, ov);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * f);
+                                tmem_st32(tmem + lane_base + kColO + cc * 32, ov);
+                            }
+                        }
+                        m_ref = m_new;
+                    }
+                    uint32_t pv[32];
+                    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float p0 = exp2f(__uint_as_float(sv[(2 * c) >> 5][(2 * c) & 31]) - m_use);
+                        const float p1 = exp2f(__uint_as_float(sv[(2 * c + 1) >> 5][(2 * c + 1) & 31]) - m_use);
+                        const uint32_t pk = pack_bf16(p0, p1);
+                        // the row sum must match what the tensor core will see: the rounded values
+                        l_run += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+                        pv[c] = pk;
+                    }
+                    tmem_st32(tmem + lane_base + kColP, pv);
+                    tmem_wait_st();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sb.p_full);
+            }
+            if (!ok) break;
+            // ---- unit done: O / l -> global
+            ok = mbar_wait(&sb.o_full, unit & 1, &sb, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            if (warp_active) {
+                const float inv = active ? 1.f / l_run : 0.f;
+                __nv_bfloat16 *dst = a.out + ((int64_t)(n_lo + node) * a.Hq + hq) * kD;
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t ov[32];
+                    tmem_ld32(tmem + lane_base + kColO + cc * 32, ov);
+                    tmem_wait_ld();
+                    if (active) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                            w.y = pack_bf16(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                            w.z = pack_bf16(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                            w.w = pack_bf16(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(dst + cc * 32 + c) = w;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// [rows, cols] bf16 row-major with `pitch` bytes between rows; boxes of 64 cols x 64 rows.
+bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t pitch) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBN};
+    const cuuint32_t el[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, el,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+namespace dsbd {
+
+bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+    if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
+    if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows) return false;
+    if (f->max_tree_nodes > kBN) return false;
+    if (d->total_prefix <= 0) return false;
+    if ((int64_t)d->total_prefix * d->Hkv >= (int64_t)1 << 31) return false;
+    return encode_fn() != nullptr;
+}
+
+int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
+                        const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
+                        void *out, int32_t *status, cudaStream_t stream) {
+    CUtensorMap kp, vp, kn, vn;
+    const uint64_t prows = (uint64_t)d->total_prefix * d->Hkv;
+    if (!make_map(&kp, k_prefix, kD, prows, kD * 2) || !make_map(&vp, v_prefix, kD, prows, kD * 2) ||
+        !make_map(&kn, k_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2) ||
+        !make_map(&vn, v_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2))
+        return DSBD_ERR_CUDA;
+    TcArgs a = {};
+    a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;
+    a.n_units = f->B * d->Hkv;
+    a.scale_log2 = d->scale * 1.4426950408889634f;
+    a.beam_node_off = f->beam_node_off; a.parent = f->parent; a.prefix_off = prefix_off;
+    a.q = static_cast<const __nv_bfloat16 *>(q);
+    a.out = static_cast<__nv_bfloat16 *>(out);
+    a.status = status;
+    if (cudaFuncSetAttribute(k_forest_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
+        cudaSuccess)
+        return DSBD_ERR_CUDA;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int grid = sms * 2;
+    if (grid > a.n_units) grid = a.n_units;
+    k_forest_attn_tc<<<grid, kThreadsTc, kSmemBytes, stream>>>(kp, vp, kn, vn, a);
+    return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
+
+}  // namespace dsbd
