@@ -196,6 +196,8 @@ def main():
     ap.add_argument("--workload", default="C5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--requests", type=int, default=0,
+                    help="override the number of requests of the workload (profiling on a smaller case)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -217,6 +219,8 @@ def main():
     dsbd.load()
 
     spec = inputs.config(args.workload)
+    if args.requests > 0:
+        spec["R"] = args.requests
     spec["seed"] = spec["seed"] + 1000 * rank            # every rank verifies its own requests
     data = inputs.generate(spec, dev)
     forest, prm, poff = data["forest"], dict(data["params"]), data["prefix_off"]

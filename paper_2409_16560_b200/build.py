@@ -10,7 +10,7 @@ LIB_PATH = os.path.join(BUILD_DIR, "libdsbd.so")
 SOURCES = ["dsbd_api.cu", "dsbd_verify.cu", "dsbd_attention.cu", "dsbd_attention_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xptxas=-v", "-Xcompiler", "-fPIC",
-              "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+              "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("DSBD_NVCC_EXTRA", "").split()
 
 
 def _deps():

@@ -55,6 +55,23 @@ __device__ __forceinline__ void load_tile(const float *__restrict__ row, int e0,
     }
 }
 
+__device__ __forceinline__ void load_half_tile(const float *__restrict__ row, int e0, int V, bool aligned,
+                                               int lane, float4 (&v)[4]) {
+    const float ninf = -INFINITY;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int e = e0 + it * 128 + lane * 4;
+        if (aligned && e + 3 < V) {
+            v[it] = ldg_stream(reinterpret_cast<const float4 *>(row + e));
+        } else {
+            v[it].x = e < V ? __ldg(row + e) : ninf;
+            v[it].y = e + 1 < V ? __ldg(row + e + 1) : ninf;
+            v[it].z = e + 2 < V ? __ldg(row + e + 2) : ninf;
+            v[it].w = e + 3 < V ? __ldg(row + e + 3) : ninf;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------
 // Dense pass: tile statistics of every (model, row).  Item = (model, row, tile), tile fastest,
 // one warp per item.  rows == nullptr: all n_rows rows; else the listed rows (n_rows read
@@ -197,6 +214,8 @@ struct VerifyArgs {
     const double *score;      // [2][N]
     const int32_t *depth;     // [N]
     double *tile_sums;        // [R][2][max_m][max_live*T]
+    unsigned long long *hist; // [R][2 banks][kBins+1] fixed-point ratio histograms (p<<32 | q)
+    unsigned long long *dbg;  // phase time stamps (DSBD_PHASE_TIMING builds only)
     int max_m, max_live;
     // outputs
     dsbd_verify_out_t out;
@@ -225,8 +244,8 @@ struct Shared {
     double first[kMaxLive + 1];             // alpha_i prod_{j<i}(1-alpha_j)
     double col_a[kMaxLive + 1], col_b[kMaxLive + 1];
     double tail[kMaxLive + 2];
-    float s_cur;
-    int bank;
+    int bank, need_exact, res_j, run_j, chain_pos;
+    double rho[kMaxLive], uu[kMaxLive];     // per live draft: p_beam/q_beam and its uniform
 };
 
 // mass of one cell of the residual max(p_beam - s q_beam, 0); s == 0 gives p_beam
@@ -249,17 +268,20 @@ __device__ void residual_pass(const VerifyArgs &a, const Shared &sh, float s, do
         const float *rp = a.zp + (int64_t)row * a.stride;
         const float *rq = a.zq + (int64_t)row * a.stride;
         const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
-        float4 vp[8], vq[8];
-        load_tile(rp, t * kTile, a.V, al, lane, vp);
-        load_tile(rq, t * kTile, a.V, al, lane, vq);
         const float bp = sh.bp[i], bq = sh.bq[i];
         float acc = 0.f;
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            acc += cell_mass(vp[it].x, vq[it].x, a.k2, bp, bq, s);
-            acc += cell_mass(vp[it].y, vq[it].y, a.k2, bp, bq, s);
-            acc += cell_mass(vp[it].z, vq[it].z, a.k2, bp, bq, s);
-            acc += cell_mass(vp[it].w, vq[it].w, a.k2, bp, bq, s);
+        for (int half = 0; half < 2; ++half) {
+            float4 vp[4], vq[4];
+            load_half_tile(rp, t * kTile + half * (kTile / 2), a.V, al, lane, vp);
+            load_half_tile(rq, t * kTile + half * (kTile / 2), a.V, al, lane, vq);
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                acc += cell_mass(vp[it].x, vq[it].x, a.k2, bp, bq, s);
+                acc += cell_mass(vp[it].y, vq[it].y, a.k2, bp, bq, s);
+                acc += cell_mass(vp[it].z, vq[it].z, a.k2, bp, bq, s);
+                acc += cell_mass(vp[it].w, vq[it].w, a.k2, bp, bq, s);
+            }
         }
         const double tot = warp_sum((double)acc);
         if (lane == 0) sums[item] = tot;
@@ -387,20 +409,25 @@ __device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, 
 }
 
 // Beam weights of the live set: softmax of the cumulative scores over A (Eq. 1 factorised).
-__device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, const double *sq) {
+// Called by all lanes of one warp; beam i is handled by lane i % 32.
+__device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, const double *sq, int lane) {
     double mp = -INFINITY, mq = -INFINITY;
-    for (int i = 0; i < sh.nA; ++i) { mp = fmax(mp, sp[i]); mq = fmax(mq, sq[i]); }
+    for (int i = lane; i < sh.nA; i += 32) { mp = fmax(mp, sp[i]); mq = fmax(mq, sq[i]); }
+    mp = warp_max(mp); mq = warp_max(mq);
     double tp = 0.0, tq = 0.0;
-    for (int i = 0; i < sh.nA; ++i) { tp += exp(sp[i] - mp); tq += exp(sq[i] - mq); }
-    for (int i = 0; i < sh.nA; ++i) {
-        const double wp = exp(sp[i] - mp) / tp, wq = exp(sq[i] - mq) / tq;
-        sh.wp[i] = wp;
-        sh.lwp[i] = log(wp);
-        sh.lwq[i] = log(wq);
+    for (int i = lane; i < sh.nA; i += 32) { tp += exp(sp[i] - mp); tq += exp(sq[i] - mq); }
+    tp = warp_sum(tp); tq = warp_sum(tq);
+    const double ltp = log(tp), ltq = log(tq);
+    for (int i = lane; i < sh.nA; i += 32) {
+        const double lwp = (sp[i] - mp) - ltp, lwq = (sq[i] - mq) - ltq;
+        sh.wp[i] = exp(lwp);
+        sh.lwp[i] = lwp;
+        sh.lwq[i] = lwq;
         const int row = sh.A[i];
-        sh.bp[i] = (float)((sh.lwp[i] - a.lse[row]) / kLn2);
-        sh.bq[i] = (float)((sh.lwq[i] - a.lse[a.N + row]) / kLn2);
+        sh.bp[i] = (float)((lwp - a.lse[row]) / kLn2);
+        sh.bq[i] = (float)((lwq - a.lse[a.N + row]) / kLn2);
     }
+    __syncwarp();
 }
 
 // Acceptance-count recursion by one warp (lanes over n): tail[K] = P(at least K accepts),
@@ -440,7 +467,105 @@ __device__ int width_rule(Shared &sh, int m, double thresh, int lane) {
     return wt;
 }
 
-__global__ void __launch_bounds__(kThreads)
+// ---------------------------------------------------------------------------------------
+// Ratio histogram of one layer.  Every cell with rho = p_beam/q_beam > 1 adds its p and q mass
+// (fixed point, 2^-31) to the bin of log2(rho); bin kBins collects rho beyond the last edge.
+// F(s) for any s in [1, top] is then (sum of the bins above s) plus the straddled bin, whose
+// contribution is bracketed from its two sums and its edges.  Integer sums make the result
+// independent of the order in which warps and CTAs add.
+// ---------------------------------------------------------------------------------------
+constexpr int kBins = 4096;
+constexpr float kFix = 2147483648.f;          // 2^31
+constexpr double kUnfix = 1.0 / 2147483648.0;
+constexpr double kGapTol = 2.5e-7;            // bracket width above which F(s) is recomputed exactly
+
+__device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, uint32_t *hp,
+                               uint32_t *hq, int cta_rank, int n_cta) {
+    const int lane = threadIdx.x & 31;
+    const int warp = cta_rank * kWarps + (threadIdx.x >> 5);
+    const int nwarps = n_cta * kWarps;
+    const int items = sh.nA * a.T * 2;                   // half tiles of 512 tokens
+    uint32_t over_p = 0u, over_q = 0u;                   // cells beyond the last edge: always above s
+    for (int item = warp; item < items; item += nwarps) {
+        const int tile = item >> 1, half = item & 1;
+        const int i = tile / a.T, t = tile - i * a.T;
+        const int row = sh.A[i];
+        const float *rp = a.zp + (int64_t)row * a.stride;
+        const float *rq = a.zq + (int64_t)row * a.stride;
+        const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
+        float4 vp[4], vq[4];
+        const int e0 = t * kTile + half * (kTile / 2);
+        load_half_tile(rp, e0, a.V, al, lane, vp);
+        load_half_tile(rq, e0, a.V, al, lane, vq);
+        const float bp = sh.bp[i], bq = sh.bq[i];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const float zp4[4] = {vp[it].x, vp[it].y, vp[it].z, vp[it].w};
+            const float zq4[4] = {vq[it].x, vq[it].y, vq[it].z, vq[it].w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float xp = fmaf(zp4[c], a.k2, bp), xq = fmaf(zq4[c], a.k2, bq);
+                const float dl = xp - xq;                       // log2(rho); NaN compares false
+                if (dl > 0.f) {
+                    const uint32_t fp = __float2uint_rn(exp2f(xp) * kFix);
+                    const uint32_t fq = __float2uint_rn(exp2f(xq) * kFix);
+                    const float bf = dl * binscale;
+                    if (bf < (float)kBins) {
+                        const int bin = (int)bf;
+                        atomicAdd(hp + bin, fp);
+                        atomicAdd(hq + bin, fq);
+                    } else {
+                        over_p += fp;
+                        over_q += fq;
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        over_p += __shfl_xor_sync(kFull, over_p, o);
+        over_q += __shfl_xor_sync(kFull, over_q, o);
+    }
+    if (lane == 0 && (over_p | over_q)) { atomicAdd(hp + kBins, over_p); atomicAdd(hq + kBins, over_q); }
+}
+
+// One completion draw (residual if s_res > 0 else p_beam) by warp 0; returns the token or -1
+// and the index of the live parent.
+__device__ int draw_cell(const VerifyArgs &a, const Shared &sh, double u, bool use_res, float s_res,
+                         double z_res, const double *res_sums, int lane, int *ia_out) {
+    int tile = -1;
+    double before = 0.0, target;
+    if (use_res) {
+        target = u * z_res;
+        tile = locate_tile([&](int i) { return __ldcg(res_sums + i); }, sh.nA * a.T, target, lane, &before);
+    } else {
+        double z = 0.0;
+        for (int i = 0; i < sh.nA; ++i) z += sh.wp[i];
+        target = u * z;
+        const int T = a.T;
+        tile = locate_tile([&](int i) {
+            const int ia = i / T;
+            const int row = sh.A[ia];
+            const TileStat ts = a.stats[(int64_t)row * T + (i - ia * T)];
+            if (!(ts.sum > 0.f)) return 0.0;
+            return sh.wp[ia] * (double)ts.sum * exp((double)ts.mx * a.inv_tau - a.lse[row]);
+        }, sh.nA * a.T, target, lane, &before);
+    }
+    if (tile < 0) return -1;
+    const int ia = tile / a.T;
+    *ia_out = ia;
+    return locate_token(a, sh.A[ia], tile - ia * a.T, sh.bp[ia], sh.bq[ia], use_res ? s_res : 0.f,
+                        target - before, lane);
+}
+
+#ifdef DSBD_PHASE_TIMING
+#define TS(slot) do { if (threadIdx.x == 0 && writer) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); a.dbg[(int64_t)r * 256 + ts_n] = ((unsigned long long)(slot) << 48) | (t_ & 0xFFFFFFFFFFFFull); if (ts_n < 255) ++ts_n; } } while (0)
+#else
+#define TS(slot) do {} while (0)
+#endif
+
+__global__ void __launch_bounds__(kThreads, 4)
 k_verify(VerifyArgs a) {
     cg::cluster_group cluster = cg::this_cluster();
     const int n_cta = (int)cluster.num_blocks();
@@ -451,6 +576,8 @@ k_verify(VerifyArgs a) {
     const bool writer = (cta_rank == 0);
     __shared__ Shared sh;
     __shared__ double sp_live[kMaxLive], sq_live[kMaxLive];
+    __shared__ int8_t st[kMaxLive * kMaxLive];     // status of the request's nodes, local index
+    __shared__ uint32_t hp[kBins + 2], hq[kBins + 2];   // p and q mass per ratio bin, fixed point
 
     const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
     const int n_lo = a.beam_node_off[b_lo], n_hi = a.beam_node_off[b_hi];
@@ -459,9 +586,14 @@ k_verify(VerifyArgs a) {
     const int W_nom = a.W_nom_r ? a.W_nom_r[r] : a.W_nom;
     double *sums_base = a.tile_sums + (int64_t)r * 2 * a.max_m * ((int64_t)a.max_live * a.T);
     const int64_t slot_stride = (int64_t)a.max_live * a.T;
+    unsigned long long *ghist = a.hist + (int64_t)r * 2 * (kBins + 1);     // [2 banks][kBins+1]
+    const int hist_len = kBins + 1;
     int n_out = 0;
+    int ts_n = 0; (void)ts_n;
 
     // ---- set-up ----
+    TS(1);
+    for (int i = cta_rank * kThreads + threadIdx.x; i < 2 * hist_len; i += n_cta * kThreads) ghist[i] = 0ull;
     if (warp == 0) {
         if (lane == 0) {
             sh.err = 0; sh.done = 0;
@@ -494,24 +626,22 @@ k_verify(VerifyArgs a) {
             for (int n = n_lo + lane; n < n_hi; n += 32)
                 a.out.node_status[n] = a.parent[n] < 0 ? DSBD_NODE_ACCEPTED : DSBD_NODE_UNREACHED;
     }
-    __syncthreads();
-    // node_status is read back by this same CTA only through shared decisions below; the other
-    // CTAs of the cluster keep their own copy of every decision, so only rank 0 writes it.
-
+    // Every CTA of the cluster takes identical decisions from identical data, so each keeps its
+    // own copy of the node statuses and only rank 0 writes results.
     const int n_layers = a.select_mode ? 1 : a.gamma;
-    // status of the nodes as this CTA sees it (every CTA takes identical decisions)
-    __shared__ int8_t st[kMaxLive * kMaxLive];     // nodes of one request, local index
     const int n_req_nodes = n_hi - n_lo;
     const bool st_ok = n_req_nodes <= kMaxLive * kMaxLive;
-    if (!a.select_mode) {
+    if (!a.select_mode)
         for (int n = threadIdx.x; n < n_req_nodes && st_ok; n += blockDim.x)
             st[n] = a.parent[n_lo + n] < 0 ? DSBD_NODE_ACCEPTED : DSBD_NODE_UNREACHED;
-        if (!st_ok && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_FOREST;
-    }
+    __threadfence();
+    cluster.sync();                                   // the histogram banks are zero from here on
+    if (!a.select_mode && !st_ok && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_FOREST;
     __syncthreads();
 
     for (int l = 1; l <= n_layers && !sh.done && !sh.err; ++l) {
         // ---- live drafts of layer l, in draw order; beam weights ----
+        TS(2);
         if (warp == 0) {
             int m = 0;
             if (a.select_mode) {
@@ -520,21 +650,17 @@ k_verify(VerifyArgs a) {
             } else {
                 for (int base = 0; base < n_req_nodes; base += 32) {
                     const int n = base + lane;
-                    bool at_layer = false, live = false;
+                    bool live = false;
                     if (n < n_req_nodes && a.depth[n_lo + n] == l) {
-                        at_layer = true;
                         live = st[a.parent[n_lo + n] - n_lo] == DSBD_NODE_ACCEPTED;
                         if (!live) {
                             st[n] = DSBD_NODE_PRUNED;
                             if (writer) a.out.node_status[n_lo + n] = DSBD_NODE_PRUNED;
                         }
                     }
-                    (void)at_layer;
                     const unsigned mask = __ballot_sync(kFull, live);
                     const int pos = m + __popc(mask & ((1u << lane) - 1));
-                    if (live) {
-                        if (pos < kMaxLive) sh.S[pos] = n_lo + n;
-                    }
+                    if (live && pos < kMaxLive) sh.S[pos] = n_lo + n;
                     m += __popc(mask);
                 }
                 if (m > kMaxLive) { if (lane == 0) sh.err = DSBD_DEV_BAD_FOREST; m = 0; }
@@ -550,52 +676,140 @@ k_verify(VerifyArgs a) {
                     }
                 }
             }
+            __syncwarp();
+            live_weights(a, sh, sp_live, sq_live, lane);
             if (lane == 0) {
                 sh.m = m;
-                live_weights(a, sh, sp_live, sq_live);
-                if (!a.select_mode)
-                    for (int i = 0; i < m; ++i) {
-                        const int par = a.parent[sh.S[i]];
-                        int ai = 0;
-                        while (ai < sh.nA && sh.A[ai] != par) ++ai;
-                        sh.S_parent_idx[i] = ai;
-                    }
                 sh.s_arr[0] = 0.0;
                 sh.c_arr[1] = 1.0;
-                sh.chain_len = 0;          // number of c_{j+1} known: j = 1..chain_len
-                sh.s_cur = 1.0f;
+                sh.chain_len = 0;          // c_{j+1} is known for j = 1..chain_len
                 sh.bank = l & 1;
             }
+            // per live draft: index of its parent in A, rho = p_beam/q_beam of its cell, its uniform
+            if (!a.select_mode)
+                for (int i = lane; i < m; i += 32) {
+                    const int n = sh.S[i];
+                    const int par = a.parent[n];
+                    int ai = 0;
+                    while (ai < sh.nA && sh.A[ai] != par) ++ai;
+                    sh.S_parent_idx[i] = ai;
+                    const double lp = a.score[n] - a.score[par];
+                    const double lq = a.score[a.N + n] - a.score[a.N + par];
+                    double rho;
+                    if (lq == -INFINITY || sh.lwq[ai] == -INFINITY)
+                        rho = (lp > -INFINITY && sh.lwp[ai] > -INFINITY) ? INFINITY : 0.0;
+                    else
+                        rho = exp((sh.lwp[ai] - sh.lwq[ai]) + (lp - lq));
+                    sh.rho[i] = rho;
+                    sh.uu[i] = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l, 0u, (uint32_t)i);
+                }
         }
+        for (int i = threadIdx.x; i < kBins + 2; i += blockDim.x) { hp[i] = 0u; hq[i] = 0u; }
         __syncthreads();
         const int m = sh.m;
+        TS(3);
 
-        // ---- residual masses c_{j+1} = F(s_j), j = 1..m ----
-        for (int j = 1; j <= m && !sh.err; ++j) {
-            double *sums = sums_base + ((int64_t)sh.bank * a.max_m + (j - 1)) * slot_stride;
-            const double s_j = sh.s_arr[j - 1] + sh.c_arr[j];
-            residual_pass(a, sh, (float)s_j, sums, cta_rank, n_cta);
+        if (m >= 1 && !sh.err) {
+            // ---- one pass: ratio histogram of the layer over the live rows ----
+            const double top = log2((double)(m > 2 ? m : 2));          // s_j <= j <= m
+            const float binscale = (float)((double)kBins / top);
+            unsigned long long *gh = ghist + sh.bank * hist_len;
+            histogram_pass(a, sh, binscale, hp, hq, cta_rank, n_cta);
+            __syncthreads();
+            TS(4);
+            for (int i = threadIdx.x; i <= kBins; i += blockDim.x)
+                if (hp[i] | hq[i]) atomicAdd(gh + i, ((unsigned long long)hp[i] << 32) | hq[i]);
             __threadfence();
             cluster.sync();
-            bool stop = false;
-            if (warp == 0) {
-                const double c_next = ordered_sum(sums, sh.nA * a.T, lane);
-                if (lane == 0) {
-                    sh.s_arr[j] = s_j;
-                    sh.c_arr[j + 1] = c_next;
-                    sh.chain_len = j;
-                }
+            TS(5);
+            for (int i = threadIdx.x; i <= kBins; i += blockDim.x) {
+                const unsigned long long v = __ldcg(gh + i);
+                hp[i] = (uint32_t)(v >> 32);
+                hq[i] = (uint32_t)v;
             }
             __syncthreads();
-            stop = !(sh.c_arr[j + 1] > 0.0);
-            if (stop) break;
+            cluster.sync();                            // everyone has read the bank: it can be cleared
+            for (int i = cta_rank * kThreads + threadIdx.x; i < hist_len; i += n_cta * kThreads) gh[i] = 0ull;
+            TS(6);
+            // in-place suffix sums: hp[k] = p mass of the bins >= k (warp 0, 129 bins per lane)
+            if (warp == 0) {
+                constexpr int per = (kBins + 1 + 31) / 32;
+                const int lo = lane * per, hi = min(lo + per, kBins + 1);
+                uint32_t mp_ = 0u, mq_ = 0u;
+                for (int i = lo; i < hi; ++i) { mp_ += hp[i]; mq_ += hq[i]; }
+                uint32_t ap = mp_, aq = mq_;              // inclusive scan from the top lane down
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t tp = __shfl_down_sync(kFull, ap, o), tq = __shfl_down_sync(kFull, aq, o);
+                    if (lane + o < 32) { ap += tp; aq += tq; }
+                }
+                uint32_t rp_ = ap - mp_, rq_ = aq - mq_;  // mass of the lanes above
+                for (int i = hi - 1; i >= lo; --i) {
+                    rp_ += hp[i]; rq_ += hq[i];
+                    hp[i] = rp_; hq[i] = rq_;
+                }
+                if (lane == 0) { hp[kBins + 1] = 0u; hq[kBins + 1] = 0u; }
+            }
+            __syncthreads();
+
+            TS(7);
+            int j0 = 1;
+            while (j0 <= m) {
+                if (threadIdx.x == 0) {
+                    int j = j0;
+                    int need = 0;
+                    for (; j <= m; ++j) {
+                        const double s_j = sh.s_arr[j - 1] + sh.c_arr[j];
+                        sh.s_arr[j] = s_j;
+                        sh.chain_len = j;
+                        double c_next;
+                        if (j == 1) {
+                            c_next = ((double)hp[0] - (double)hq[0]) * kUnfix;
+                        } else {
+                            int k = (int)(log2(s_j) * (double)binscale);
+                            if (k < 0) k = 0;
+                            if (k >= kBins) { need = 1; break; }      // cannot happen for s_j <= m
+                            const double Pa = (double)hp[k + 1] * kUnfix, Qa = (double)hq[k + 1] * kUnfix;
+                            const double Pk = (double)(hp[k] - hp[k + 1]) * kUnfix;
+                            const double Qk = (double)(hq[k] - hq[k + 1]) * kUnfix;
+                            const double r_lo = (double)exp2f((float)k / binscale) * (1.0 - 2e-6);
+                            const double r_hi = (double)exp2f((float)(k + 1) / binscale) * (1.0 + 2e-6);
+                            const double lo_b = fmax(Pk - s_j * Qk, 0.0);
+                            double q_hi = (Pk - r_lo * Qk) / (r_hi - r_lo);
+                            q_hi = fmin(fmax(q_hi, 0.0), Qk);
+                            const double hi_b = fmax(q_hi * (r_hi - s_j), lo_b);
+                            if (hi_b - lo_b > kGapTol) { need = 1; break; }
+                            c_next = fmax(Pa - s_j * Qa, 0.0) + 0.5 * (lo_b + hi_b);
+                        }
+                        sh.c_arr[j + 1] = c_next;
+                        if (!(c_next > 0.0)) { j = m; }               // chain exhausted: stop walking
+                    }
+                    sh.need_exact = need;
+                    sh.chain_pos = need ? j : m + 1;
+                }
+                __syncthreads();
+                if (!sh.need_exact) break;
+                const int j = sh.chain_pos;
+                double *sums = sums_base + ((int64_t)sh.bank * a.max_m + (j - 1)) * slot_stride;
+                residual_pass(a, sh, (float)sh.s_arr[j], sums, cta_rank, n_cta);
+                __threadfence();
+                cluster.sync();
+                if (warp == 0) {
+                    const double c_next = ordered_sum(sums, sh.nA * a.T, lane);
+                    if (lane == 0) sh.c_arr[j + 1] = c_next;
+                }
+                __syncthreads();
+                if (!(sh.c_arr[j + 1] > 0.0)) break;
+                j0 = j + 1;
+            }
         }
         __syncthreads();
 
-        // ---- width, accept loop, completion (warp 0) ----
+        TS(8);
+        // ---- width and accept loop (warp 0) ----
         if (warp == 0 && !sh.err) {
-            // alpha_j = 1 - c_{j+1}/c_j; once a residual has no mass every later alpha is 1
             if (lane == 0) {
+                // alpha_j = 1 - c_{j+1}/c_j; once a residual has no mass every later alpha is 1
                 for (int j = 1; j <= m; ++j) {
                     if (j <= sh.chain_len && sh.c_arr[j] > 0.0) {
                         double al = 1.0 - sh.c_arr[j + 1] / sh.c_arr[j];
@@ -605,6 +819,7 @@ k_verify(VerifyArgs a) {
                         sh.alpha[j] = 1.0;
                     }
                 }
+                sh.res_j = 0;
             }
             __syncwarp();
             const int wt = width_rule(sh, m, a.thresh, lane);
@@ -621,161 +836,127 @@ k_verify(VerifyArgs a) {
                             a.tail_out[(int64_t)r * a.out_stride + K] = (float)sh.tail[K];
                 }
                 if (lane == 0) sh.done = 1;
-            } else {
-                if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + (l - 1)] = W;
-                // accept loop (lane 0), Algorithm 1
+            } else if (lane == 0) {
+                if (writer) a.out.layer_width[(int64_t)r * (a.gamma + 1) + (l - 1)] = W;
                 int count = 0, j = 1, err = 0;
-                if (lane == 0) {
-                    for (int i = 0; i < m && count < W; ++i) {
-                        const int n = sh.S[i];
-                        const int ai = sh.S_parent_idx[i];
-                        const double lp = a.score[n] - a.score[a.parent[n]];
-                        const double lq = a.score[a.N + n] - a.score[a.N + a.parent[n]];
-                        double rho;
-                        if (lq == -INFINITY || sh.lwq[ai] == -INFINITY)
-                            rho = (lp > -INFINITY && sh.lwp[ai] > -INFINITY) ? INFINITY : 0.0;
-                        else
-                            rho = exp((sh.lwp[ai] - sh.lwq[ai]) + (lp - lq));
-                        double ratio;
-                        if (j == 1) ratio = rho;
-                        else ratio = fmax(rho - sh.s_arr[j - 1], 0.0) / sh.c_arr[j];
-                        if (ratio > 1.0) ratio = 1.0;
-                        const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l, 0u, (uint32_t)i);
-                        if (u <= ratio) {
-                            st[n - n_lo] = DSBD_NODE_ACCEPTED;
-                            if (writer) a.out.node_status[n] = DSBD_NODE_ACCEPTED;
-                            sh.acc[count++] = n;
-                            j = 1;
+                for (int i = 0; i < m && count < W; ++i) {
+                    const int n = sh.S[i];
+                    const double rho = sh.rho[i];
+                    double ratio;
+                    if (j == 1) ratio = rho;
+                    else ratio = fmax(rho - sh.s_arr[j - 1], 0.0) / sh.c_arr[j];
+                    if (ratio > 1.0) ratio = 1.0;
+                    const double u = sh.uu[i];
+                    if (u <= ratio) {
+                        st[n - n_lo] = DSBD_NODE_ACCEPTED;
+                        if (writer) a.out.node_status[n] = DSBD_NODE_ACCEPTED;
+                        sh.acc[count++] = n;
+                        j = 1;
+                    } else {
+                        st[n - n_lo] = DSBD_NODE_REJECTED;
+                        if (writer) a.out.node_status[n] = DSBD_NODE_REJECTED;
+                        if (j <= sh.chain_len && sh.c_arr[j + 1] > 0.0) {
+                            ++j;
                         } else {
-                            st[n - n_lo] = DSBD_NODE_REJECTED;
-                            if (writer) a.out.node_status[n] = DSBD_NODE_REJECTED;
-                            if (j <= sh.chain_len && sh.c_arr[j + 1] > 0.0) {
-                                ++j;
-                            } else {
-                                err = DSBD_DEV_EXHAUSTED;     // a rejection of probability zero
-                                j = 1;
-                            }
+                            err = DSBD_DEV_EXHAUSTED;     // a rejection of probability zero
+                            j = 1;
                         }
                     }
-                    for (int i = 0; i < m; ++i)
-                        if (st[sh.S[i] - n_lo] == DSBD_NODE_UNREACHED) {
-                            st[sh.S[i] - n_lo] = DSBD_NODE_CUT;
-                            if (writer) a.out.node_status[sh.S[i]] = DSBD_NODE_CUT;
-                        }
                 }
-                count = __shfl_sync(kFull, count, 0);
-                j = __shfl_sync(kFull, j, 0);
+                for (int i = 0; i < m; ++i)
+                    if (st[sh.S[i] - n_lo] == DSBD_NODE_UNREACHED) {
+                        st[sh.S[i] - n_lo] = DSBD_NODE_CUT;
+                        if (writer) a.out.node_status[sh.S[i]] = DSBD_NODE_CUT;
+                    }
+                sh.W = W;
+                sh.count = count;
+                sh.res_j = (count < W && j > 1) ? j : 0;   // residual draw at run position j needs tile sums
+                sh.run_j = j;
+                if (err) sh.err = err;
+            }
+        }
+        __syncthreads();
+
+        TS(9);
+        // ---- a residual draw locates its tile through tile sums of max(p_beam - s_{j-1} q_beam, 0) ----
+        double *res_sums = sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride;   // slot 0 of the bank
+        if (!a.select_mode && !sh.err && sh.res_j > 1) {
+            residual_pass(a, sh, (float)sh.s_arr[sh.res_j - 1], res_sums, cta_rank, n_cta);
+            __threadfence();
+            cluster.sync();
+        }
+
+        TS(10);
+        // ---- completion of a short layer, or the next layer's input beams (warp 0) ----
+        if (warp == 0 && !a.select_mode && !sh.err) {
+            const int W = sh.W, count = sh.count, j = sh.run_j;
+            int err = 0;
+            if (count < W) {
+                if (lane == 0)
+                    for (int i = 0; i < count && !err; ++i)
+                        emit_output(a, r, &n_out, a.parent[sh.acc[i]], sh.acc[i], a.token[sh.acc[i]],
+                                    DSBD_SRC_DRAFT, writer, &err);
+                n_out = __shfl_sync(kFull, n_out, 0);
                 err = __shfl_sync(kFull, err, 0);
-                if (count < W) {
-                    // short layer: accepted drafts, one draw from p', the rest from p_beam
+                int fill = 0;
+                for (int kk = count; kk < W && !err; ++kk) {
+                    const bool residual = (kk == count);
+                    const bool use_res = residual && j > 1;
+                    const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l,
+                                                      residual ? 1u : 2u, residual ? 0u : (uint32_t)fill);
+                    double z_res = 0.0;
+                    if (use_res) z_res = ordered_sum(res_sums, sh.nA * a.T, lane);
+                    int ia = 0;
+                    const int tok = draw_cell(a, sh, u, use_res, use_res ? (float)sh.s_arr[j - 1] : 0.f, z_res,
+                                              res_sums, lane, &ia);
+                    if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
                     if (lane == 0)
-                        for (int i = 0; i < count && !err; ++i)
-                            emit_output(a, r, &n_out, a.parent[sh.acc[i]], sh.acc[i], a.token[sh.acc[i]],
-                                        DSBD_SRC_DRAFT, writer, &err);
+                        emit_output(a, r, &n_out, sh.A[ia], -1, tok, residual ? DSBD_SRC_RESIDUAL : DSBD_SRC_FILL,
+                                    writer, &err);
                     n_out = __shfl_sync(kFull, n_out, 0);
                     err = __shfl_sync(kFull, err, 0);
-                    int fill = 0;
-                    for (int kk = count; kk < W && !err; ++kk) {
-                        const bool residual = (kk == count);
-                        const bool use_res = residual && j > 1;
-                        const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l,
-                                                          residual ? 1u : 2u, residual ? 0u : (uint32_t)fill);
-                        int tile = -1;
-                        double before = 0.0;
-                        float s_res = 0.f;
-                        if (use_res) {
-                            const double *sums = sums_base + ((int64_t)sh.bank * a.max_m + (j - 2)) * slot_stride;
-                            s_res = (float)sh.s_arr[j - 1];
-                            const double target = u * sh.c_arr[j];
-                            tile = locate_tile([&](int i) { return __ldcg(sums + i); }, sh.nA * a.T,
-                                               target, lane, &before);
-                            before = target - before;
-                        } else {
-                            double z = 0.0;
-                            for (int i = 0; i < sh.nA; ++i) z += sh.wp[i];
-                            const double target = u * z;
-                            const int T = a.T;
-                            tile = locate_tile([&](int i) {
-                                const int ia = i / T;
-                                const int row = sh.A[ia];
-                                const TileStat ts = a.stats[(int64_t)row * T + (i - ia * T)];
-                                if (!(ts.sum > 0.f)) return 0.0;
-                                return sh.wp[ia] * (double)ts.sum *
-                                       exp((double)ts.mx * a.inv_tau - a.lse[row]);
-                            }, sh.nA * a.T, target, lane, &before);
-                            before = target - before;
-                        }
-                        int tok = -1, ia = 0;
-                        if (tile >= 0) {
-                            ia = tile / a.T;
-                            tok = locate_token(a, sh.A[ia], tile - ia * a.T, sh.bp[ia], sh.bq[ia], s_res,
-                                               before, lane);
-                        }
-                        if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
-                        if (lane == 0)
-                            emit_output(a, r, &n_out, sh.A[ia], -1, tok,
-                                        residual ? DSBD_SRC_RESIDUAL : DSBD_SRC_FILL, writer, &err);
-                        n_out = __shfl_sync(kFull, n_out, 0);
-                        err = __shfl_sync(kFull, err, 0);
-                        if (!residual) ++fill;
-                    }
-                    if (lane == 0) {
-                        sh.done = 1;
-                        if (writer) a.out.l_last[r] = l;
-                    }
-                } else if (lane == 0) {
-                    // the accepted drafts, ascending node id, are the next layer's input beams
-                    int nA = 0;
-                    for (int n = 0; n < n_req_nodes; ++n)
-                        if (a.depth[n_lo + n] == l && st[n] == DSBD_NODE_ACCEPTED) {
-                            sh.A[nA] = n_lo + n;
-                            sp_live[nA] = a.score[n_lo + n];
-                            sq_live[nA] = a.score[a.N + n_lo + n];
-                            ++nA;
-                        }
-                    sh.nA = nA;
+                    if (!residual) ++fill;
                 }
-                if (lane == 0 && err) sh.err = err;
+                if (lane == 0) {
+                    sh.done = 1;
+                    if (writer) a.out.l_last[r] = l;
+                }
+            } else if (lane == 0) {
+                // the accepted drafts, ascending node id, are the next layer's input beams
+                int nA = 0;
+                for (int n = 0; n < n_req_nodes; ++n)
+                    if (a.depth[n_lo + n] == l && st[n] == DSBD_NODE_ACCEPTED) {
+                        sh.A[nA] = n_lo + n;
+                        sp_live[nA] = a.score[n_lo + n];
+                        sq_live[nA] = a.score[a.N + n_lo + n];
+                        ++nA;
+                    }
+                sh.nA = nA;
             }
+            if (lane == 0 && err) sh.err = err;
         }
         __syncthreads();
     }
 
+    TS(11);
     // ---- every layer passed: W_nom beams from p_beam^(gamma+1) ----
     if (!a.select_mode && warp == 0 && !sh.done && !sh.err) {
-        if (lane == 0) live_weights(a, sh, sp_live, sq_live);
-        __syncwarp();
+        live_weights(a, sh, sp_live, sq_live, lane);
         int err = 0;
         if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
         for (int kk = 0; kk < W_nom && !err; ++kk) {
             const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1), 3u, (uint32_t)kk);
-            double z = 0.0;
-            for (int i = 0; i < sh.nA; ++i) z += sh.wp[i];
-            const double target = u * z;
-            const int T = a.T;
-            double before = 0.0;
-            const int tile = locate_tile([&](int i) {
-                const int ia = i / T;
-                const int row = sh.A[ia];
-                const TileStat ts = a.stats[(int64_t)row * T + (i - ia * T)];
-                if (!(ts.sum > 0.f)) return 0.0;
-                return sh.wp[ia] * (double)ts.sum * exp((double)ts.mx * a.inv_tau - a.lse[row]);
-            }, sh.nA * a.T, target, lane, &before);
-            int tok = -1, ia = 0;
-            if (tile >= 0) {
-                ia = tile / a.T;
-                tok = locate_token(a, sh.A[ia], tile - ia * a.T, sh.bp[ia], sh.bq[ia], 0.f,
-                                   target - before, lane);
-            }
+            int ia = 0;
+            const int tok = draw_cell(a, sh, u, false, 0.f, 0.0, nullptr, lane, &ia);
             if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
-            if (lane == 0)
-                emit_output(a, r, &n_out, sh.A[ia], -1, tok, DSBD_SRC_EXTRA, writer, &err);
+            if (lane == 0) emit_output(a, r, &n_out, sh.A[ia], -1, tok, DSBD_SRC_EXTRA, writer, &err);
             n_out = __shfl_sync(kFull, n_out, 0);
             err = __shfl_sync(kFull, err, 0);
         }
         if (lane == 0 && err) sh.err = err;
     }
     __syncthreads();
+    TS(12);
     if (threadIdx.x == 0 && writer) {
         if (!a.select_mode) {
             a.out.out_width[r] = n_out;
@@ -787,7 +968,7 @@ k_verify(VerifyArgs a) {
 
 // ------------------------------------------------------------------------------ host side
 struct Layout {
-    size_t stats, lse, score, depth, sums, total;
+    size_t stats, lse, score, depth, sums, hist, total;
     int T, max_m, max_live;
 };
 
@@ -804,6 +985,11 @@ Layout make_layout(const dsbd_forest_t *f, int V) {
     L.depth = off; off = align_up(off + sizeof(int32_t) * (size_t)f->N, 256);
     L.sums = off;
     off = align_up(off + sizeof(double) * (size_t)f->R * 2 * L.max_m * (size_t)L.max_live * L.T, 256);
+    L.hist = off;
+    off = align_up(off + sizeof(unsigned long long) * (size_t)f->R * 2 * (4096 + 1), 256);
+#ifdef DSBD_PHASE_TIMING
+    off = align_up(off + sizeof(unsigned long long) * (size_t)f->R * 256, 256);
+#endif
     L.total = off;
     return L;
 }
@@ -822,15 +1008,21 @@ int check_params(const dsbd_verify_params_t *p) {
     return DSBD_OK;
 }
 
-int cluster_size_for(int tiles) {
-    if (tiles >= 64) return 8;
-    if (tiles >= 32) return 4;
-    if (tiles >= 16) return 2;
-    return 1;
+// Cluster size: as many CTAs per request as its tile count can use, but few enough that all
+// requests are resident at once (four CTAs per SM fit).
+int cluster_size_for(int tiles, int R) {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int cs = 1;
+    if (tiles >= 64) cs = 8;
+    else if (tiles >= 32) cs = 4;
+    else if (tiles >= 16) cs = 2;
+    while (cs > 1 && (long long)R * cs > 4ll * sms) cs >>= 1;
+    return cs;
 }
 
 int launch_verify(const VerifyArgs &args, int R, int tiles, cudaStream_t stream) {
-    const int cs = cluster_size_for(tiles);
+    const int cs = cluster_size_for(tiles, R);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(R * cs));
     cfg.blockDim = dim3(kThreads);
@@ -915,6 +1107,10 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
     a.stats = stats; a.lse = lse; a.score = score; a.depth = depth;
     a.tile_sums = reinterpret_cast<double *>(ws + L.sums);
     a.max_m = L.max_m; a.max_live = L.max_live;
+    a.hist = reinterpret_cast<unsigned long long *>(ws + L.hist);
+#ifdef DSBD_PHASE_TIMING
+    a.dbg = reinterpret_cast<unsigned long long *>(ws + L.total) - (size_t)f->R * 256;
+#endif
     a.out = *out; a.status = status; a.select_mode = 0;
     return launch_verify(a, f->R, L.max_live * L.T, stream);
 }
@@ -1055,6 +1251,10 @@ extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_param
     a.stats = stats; a.lse = lse; a.score = nullptr; a.depth = nullptr;
     a.tile_sums = reinterpret_cast<double *>(ws + L.sums);
     a.max_m = L.max_m; a.max_live = L.max_live;
+    a.hist = reinterpret_cast<unsigned long long *>(ws + L.hist);
+#ifdef DSBD_PHASE_TIMING
+    a.dbg = reinterpret_cast<unsigned long long *>(ws + L.total) - (size_t)f->R * 256;
+#endif
     a.status = status; a.select_mode = 1;
     a.sel_logp = node_logp; a.sel_logq = node_logq;
     a.live_off = live_off; a.live_nodes = live_nodes; a.m_in = m;
