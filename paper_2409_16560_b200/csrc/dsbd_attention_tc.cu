@@ -12,8 +12,10 @@
 //   warp 4     TMA producer: K and V tiles (2 x 64x64 bf16 boxes each, 128-byte swizzle) into a
 //              ring of shared-memory stages, completion on mbarriers.
 //   warp 5     MMA issuer (one lane): S = Q K^T (M128 N64 K16 x 8, both operands K-major in
-//              shared memory) into TMEM; after the softmax warps have written P (bf16) to TMEM,
-//              O += P V (A from TMEM, B = the V tile as an MN-major shared-memory operand).
+//              shared memory) into one of two S buffers in TMEM, one tile ahead, so that it runs
+//              while the softmax warps work on the previous tile; after they have written P
+//              (bf16, over the S buffer they just read), O += P V (A from TMEM, B = the V tile
+//              as an MN-major shared-memory operand).
 // O stays in TMEM for the whole unit; its rows are rescaled only when a row maximum grows by
 // more than 2^8 (the rescale is a TMEM load/scale/store by the row's own thread).
 // Every mbarrier wait is bounded; on a time-out the kernel records DSBD_DEV_TIMEOUT, lets its
@@ -30,15 +32,21 @@ namespace {
 
 constexpr int kD = 128;                 // head dim
 constexpr int kBN = 64;                 // tokens per tile
-constexpr int kStages = 2;
+constexpr int kMaxStages = 3;
 constexpr int kRows = 128;              // UMMA M
 constexpr int kThreadsTc = 192;
-constexpr uint32_t kQBytes = kRows * kD * 2;          // 32 KB: two 128-row x 128-byte halves
 constexpr uint32_t kTileBytes = kBN * kD * 2;         // 16 KB per K or V tile (two 8 KB boxes)
 constexpr uint32_t kStageBytes = 2 * kTileBytes;      // K then V
-constexpr uint32_t kSmemBytes = 1024 + kQBytes + kStages * kStageBytes;
+// Shared memory of one CTA: Q (QROWS rows x 256 B as two swizzled halves), the K/V stage ring,
+// then the mbarriers.  With at most 64 query rows only 64 rows of Q are stored: the MMA still
+// runs with M = 128, and the A-operand rows 64..127 then alias the bytes that follow Q.  Rows of
+// an MMA are independent and rows >= M are never read back, so whatever those bytes hold is
+// harmless; the 16 KB saved buy a third stage at two CTAs per SM.
+constexpr uint32_t smem_bytes(int qrows, int stages) { return qrows * kD * 2 + stages * kStageBytes; }
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 64, kColO = 128;
+// TMEM columns: two S buffers of 64 fp32 columns (P, bf16 pairs, overwrites the first 32 columns
+// of its S buffer once S has been read), then O (128 fp32 columns).
+constexpr uint32_t kColS = 0, kColO = 128;
 constexpr long long kWaitCycles = 2000000000ll;   // about a second
 
 struct TcArgs {
@@ -52,7 +60,7 @@ struct TcArgs {
 };
 
 struct Barriers {
-    unsigned long long kv_full[kStages], kv_empty[kStages], s_full, p_full, q_full, o_full;
+    unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages], s_full[2], p_full[2], pv_done, q_full, o_full;
     uint32_t tmem_base;
     int abort;
 };
@@ -162,21 +170,26 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
+template <int QROWS, int kStages>
 __global__ void __launch_bounds__(kThreadsTc, 2)
 k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_constant__ CUtensorMap map_vp,
                  const __grid_constant__ CUtensorMap map_kn, const __grid_constant__ CUtensorMap map_vn,
                  TcArgs a) {
-    extern __shared__ unsigned char smem_raw[];
-    __shared__ Barriers sb;
-    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char *q_s = smem;                               // [2 halves][128 rows][128 B], swizzled
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr uint32_t kQBytes = QROWS * kD * 2;
+    unsigned char *q_s = smem;                               // [2 halves][QROWS rows][128 B], swizzled
     unsigned char *stage_s = smem + kQBytes;                 // [stages][K 16 KB | V 16 KB]
+    __shared__ Barriers sb;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((smem_u32(smem) & 1023u) != 0u) {                    // the swizzled operands need 1024-byte alignment
+        if (threadIdx.x == 0) report(a.status, DSBD_DEV_BAD_FOREST);
+        return;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&sb.kv_full[s], 1); mbar_init(&sb.kv_empty[s], 1); }
-        mbar_init(&sb.s_full, 1);
-        mbar_init(&sb.p_full, 4);
+        for (int b = 0; b < 2; ++b) { mbar_init(&sb.s_full[b], 1); mbar_init(&sb.p_full[b], 4); }
+        mbar_init(&sb.pv_done, 1);
         mbar_init(&sb.q_full, 128);
         mbar_init(&sb.o_full, 1);
         sb.abort = 0;
@@ -248,29 +261,36 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
                 const int nt = (int)((L + kBN - 1) / kBN) + 1;
                 ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
-                for (int j = 0; j < nt && ok; ++j, ++tile) {
-                    const int s = tile % kStages;
-                    ok = mbar_wait(&sb.kv_full[s], (tile / kStages) & 1, &sb, a.status);
-                    if (!ok) break;
+                // S(t) = Q K(t)^T into S buffer t & 1; issued one tile ahead of the P V product so
+                // that it runs while the softmax warps work on the previous tile
+                auto issue_s = [&](uint32_t t) -> bool {
+                    const int s = t % kStages;
+                    if (!mbar_wait(&sb.kv_full[s], (t / kStages) & 1, &sb, a.status)) return false;
                     tc_fence_after();
-                    const uint32_t k_addr = smem_u32(stage_s + s * kStageBytes);
-                    const uint64_t kd = desc_k_major(k_addr);
+                    const uint64_t kd = desc_k_major(smem_u32(stage_s + s * kStageBytes));
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint64_t ad = qd + (uint64_t)((ks / 4) * ((kRows * 128) >> 4) + (ks % 4) * 2);
+                        const uint64_t ad = qd + (uint64_t)((ks / 4) * ((QROWS * 128) >> 4) + (ks % 4) * 2);
                         const uint64_t bd = kd + (uint64_t)((ks / 4) * ((kBN * 128) >> 4) + (ks % 4) * 2);
-                        mma_ss(tmem + kColS, ad, bd, idesc_s, ks > 0);
+                        mma_ss(tmem + kColS + (t & 1) * 64, ad, bd, idesc_s, ks > 0);
                     }
-                    tc_commit(&sb.s_full);
-                    ok = mbar_wait(&sb.p_full, tile & 1, &sb, a.status);
+                    tc_commit(&sb.s_full[t & 1]);
+                    return true;
+                };
+                if (ok) ok = issue_s(tile);
+                for (int j = 0; j < nt && ok; ++j, ++tile) {
+                    if (j + 1 < nt) { ok = issue_s(tile + 1); if (!ok) break; }
+                    const int s = tile % kStages;
+                    ok = mbar_wait(&sb.p_full[tile & 1], (tile >> 1) & 1, &sb, a.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t vd = desc_mn_major(k_addr + kTileBytes, kBN * 128);
+                    const uint64_t vd = desc_mn_major(smem_u32(stage_s + s * kStageBytes) + kTileBytes, kBN * 128);
 #pragma unroll
                     for (int ks = 0; ks < kBN / 16; ++ks)
-                        mma_ts(tmem + kColO, tmem + kColP + ks * 8, vd + (uint64_t)(ks * ((16 * 128) >> 4)), idesc_o,
-                               (j > 0 || ks > 0) ? 1u : 0u);
+                        mma_ts(tmem + kColO, tmem + kColS + (tile & 1) * 64 + ks * 8,
+                               vd + (uint64_t)(ks * ((16 * 128) >> 4)), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
                     tc_commit(&sb.kv_empty[s]);
+                    tc_commit(&sb.pv_done);
                 }
                 if (ok) tc_commit(&sb.o_full);
             }
@@ -295,7 +315,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             // ---- stage Q (rows >= M zero) and the ancestor masks; the previous unit's MMAs are done
             {
                 const int t128 = threadIdx.x;                        // 0..127
-                for (int i = t128; i < kRows * 16; i += 128) {
+                for (int i = t128; i < QROWS * 16; i += 128) {
                     const int r = i >> 4, c = i & 15;                // row, 16-byte chunk of the 256-byte row
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (r < M) {
@@ -303,7 +323,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                         v = *reinterpret_cast<const uint4 *>(a.q + ((int64_t)(n_lo + nd) * a.Hq + hh) * kD + c * 8);
                     }
                     const int half = c >> 3, cc = c & 7;
-                    *reinterpret_cast<uint4 *>(q_s + half * (kRows * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+                    *reinterpret_cast<uint4 *>(q_s + half * (QROWS * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive(&sb.q_full);
@@ -321,13 +341,14 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             }
             float m_ref = -INFINITY, l_run = 0.f;
             for (int j = 0; j <= nt_p && ok; ++j, ++tile) {
-                ok = mbar_wait(&sb.s_full, tile & 1, &sb, a.status);
+                ok = mbar_wait(&sb.s_full[tile & 1], (tile >> 1) & 1, &sb, a.status);
                 if (!ok) break;
                 tc_fence_after();
                 if (warp_active) {
                     uint32_t sv[2][32];
-                    tmem_ld32(tmem + lane_base + kColS, sv[0]);
-                    tmem_ld32(tmem + lane_base + kColS + 32, sv[1]);
+                    const uint32_t s_col = kColS + (tile & 1) * 64;
+                    tmem_ld32(tmem + lane_base + s_col, sv[0]);
+                    tmem_ld32(tmem + lane_base + s_col + 32, sv[1]);
                     tmem_wait_ld();
                     float mx = -INFINITY;
                     const bool tree = (j == nt_p);
@@ -348,6 +369,9 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     // lazy rescale: move the reference only when some row of the warp needs it
                     const bool need = mx > m_ref + 8.f;
                     if (__any_sync(kFull, need)) {
+                        // O is about to be rescaled in place: the previous tile's P V must have landed
+                        if (j > 0 && !mbar_wait(&sb.pv_done, (tile - 1) & 1, &sb, a.status)) { ok = false; }
+                        tc_fence_after();
                         const float m_new = need ? mx : m_ref;
                         const float f = (m_ref == -INFINITY) ? 0.f : exp2f(m_ref - m_new);
                         l_run *= f;
@@ -375,12 +399,12 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                         l_run += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
                         pv[c] = pk;
                     }
-                    tmem_st32(tmem + lane_base + kColP, pv);
+                    tmem_st32(tmem + lane_base + s_col, pv);
                     tmem_wait_st();
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sb.p_full);
+                if (lane == 0) mbar_arrive(&sb.p_full[tile & 1]);
             }
             if (!ok) break;
             // ---- unit done: O / l -> global
@@ -478,14 +502,24 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.q = static_cast<const __nv_bfloat16 *>(q);
     a.out = static_cast<__nv_bfloat16 *>(out);
     a.status = status;
-    if (cudaFuncSetAttribute(k_forest_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) !=
-        cudaSuccess)
-        return DSBD_ERR_CUDA;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     int grid = sms * 2;
     if (grid > a.n_units) grid = a.n_units;
-    k_forest_attn_tc<<<grid, kThreadsTc, kSmemBytes, stream>>>(kp, vp, kn, vn, a);
+    // up to 64 query rows: 16 KB of Q, three stages, two CTAs per SM; more rows: one CTA per SM
+    const bool small_q = f->max_tree_nodes * a.group <= 64;
+    if (!small_q && grid > sms) grid = sms;
+#define DSBD_LAUNCH_TC(QR, ST)                                                                              \
+    do {                                                                                                   \
+        constexpr uint32_t bytes = smem_bytes(QR, ST);                                                     \
+        if (cudaFuncSetAttribute(k_forest_attn_tc<QR, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                                 (int)bytes) != cudaSuccess)                                               \
+            return DSBD_ERR_CUDA;                                                                          \
+        k_forest_attn_tc<QR, ST><<<grid, kThreadsTc, bytes, stream>>>(kp, vp, kn, vn, a);                  \
+    } while (0)
+    if (small_q) DSBD_LAUNCH_TC(64, 3);
+    else DSBD_LAUNCH_TC(128, 3);
+#undef DSBD_LAUNCH_TC
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 
