@@ -29,6 +29,12 @@ if ROOT not in sys.path:
 METRIC = "verified forest nodes/sec per decode step"
 UNIT = "nodes/s"
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the two streaming
+# kernels on the full C5 workload, from the ncu captures summarised under profiles/
+# (k_forest_attn_tc_C5_16req.md, k_tile_stats_C5_16req.md): measured on 16 requests and scaled
+# by 64/16, the traffic being proportional to the number of requests.
+NCU_TRAFFIC_BYTES = {"C5": {"forest_attention": 8.698e9, "verify_dense_pass": 4.750e9}}
+
 
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -53,7 +59,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -190,7 +196,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="dsbd", choices=["dsbd", "reference"])
     ap.add_argument("--workload", default="C5")
@@ -366,12 +372,9 @@ def main():
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": kernels[dom]["gbs"] / peak,
                 "traffic": None}
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(prof):
-        try:
-            roofline["traffic"] = json.load(open(prof)).get(args.workload, {}).get(dom)
-        except (ValueError, OSError):
-            pass
+    if args.requests <= 0:
+        roofline["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload, {}).get(dom)
+    roofline["algorithmic_bytes"] = kernels[dom]["bytes"]
 
     cpu = None
     if not args.no_cpu_baseline:
