@@ -94,6 +94,29 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def rank_spec(spec, rank):
+    """Requests are independent, so a multi-GPU run gives every rank its own batch of the same
+    shape (weak scaling, no collective on the data path): same configuration, different seed."""
+    out = dict(spec)
+    out["seed"] = spec["seed"] + 1000 * rank
+    return out
+
+
+def max_over_ranks(ms, world, device):
+    """Step time of the job = the slowest rank's device time."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(nodes_per_rank, world, ms_per_step):
+    """Whole-job throughput: nodes verified by all ranks per second."""
+    return nodes_per_rank * world / (ms_per_step * 1e-3)
+
+
 def _cpu_baseline(data_host, spec, threads, budget_s=20.0):
     """The oracle, as it stands, on a bounded sample of the workload: verification of a few
     requests and attention of a few trees; returns nodes/s of the whole step extrapolated
@@ -227,7 +250,7 @@ def main():
     spec = inputs.config(args.workload)
     if args.requests > 0:
         spec["R"] = args.requests
-    spec["seed"] = spec["seed"] + 1000 * rank            # every rank verifies its own requests
+    spec = rank_spec(spec, rank)                         # every rank verifies its own requests
     data = inputs.generate(spec, dev)
     forest, prm, poff = data["forest"], dict(data["params"]), data["prefix_off"]
     f = dsbd.Forest(forest, dev)
@@ -290,11 +313,7 @@ def main():
     barrier()
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    total_ms = ev[0].elapsed_time(ev[1])
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), world, dev)
     attn_ms = float(np.mean([a.elapsed_time(b) for a, b in e_attn]))
     ver_ms = float(np.mean([a.elapsed_time(b) for a, b in e_ver]))
     assert int(status.item()) == 0, "device status %d" % int(status.item())
@@ -345,10 +364,8 @@ def main():
             e2e_step(s + 1)
         s1.record(stream)
         barrier()
-        te = torch.tensor([s0.elapsed_time(s1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": f.N * world * args.e2e_steps / (float(te.item()) * 1e-3), "unit": UNIT,
+        te = max_over_ranks(s0.elapsed_time(s1), world, dev)
+        e2e = {"value": job_value(f.N, world, te / args.e2e_steps), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps}
         del host
 
@@ -381,7 +398,7 @@ def main():
         cpu = _cpu_baseline(_host_views(data, spec), spec, os.cpu_count() or 1)
 
     ms_per_step = total_ms / args.steps
-    line = {"metric": METRIC, "value": f.N * world / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+    line = {"metric": METRIC, "value": job_value(f.N, world, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 attention / f32 logits", "data": "synthetic",
             "config": {"workload": args.workload, "requests": f.R, "beams": f.B, "nodes": f.N,

@@ -216,6 +216,10 @@ struct VerifyArgs {
     double *tile_sums;        // [R][2][max_m][max_live*T]
     unsigned long long *hist; // [R][2 banks][kBins+1] fixed-point ratio histograms (p<<32 | q)
     unsigned long long *dbg;  // phase time stamps (DSBD_PHASE_TIMING builds only)
+    // verify mode computes the row and tree statistics of its own request first
+    double *lse_w, *score_w;
+    int32_t *depth_w;
+    const float *root_logp, *root_logq;
     int max_m, max_live;
     // outputs
     dsbd_verify_out_t out;
@@ -245,6 +249,7 @@ struct Shared {
     double col_a[kMaxLive + 1], col_b[kMaxLive + 1];
     double tail[kMaxLive + 2];
     int bank, need_exact, res_j, run_j, chain_pos;
+    uint32_t wtot_p[kWarps], wtot_q[kWarps];
     double rho[kMaxLive], uu[kMaxLive];     // per live draft: p_beam/q_beam and its uniform
 };
 
@@ -480,47 +485,56 @@ constexpr double kUnfix = 1.0 / 2147483648.0;
 constexpr double kGapTol = 2.5e-7;            // bracket width above which F(s) is recomputed exactly
 
 __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, uint32_t *hp,
-                               uint32_t *hq, int cta_rank, int n_cta) {
+                               uint32_t *hq, double *sums1, int cta_rank, int n_cta) {
     const int lane = threadIdx.x & 31;
     const int warp = cta_rank * kWarps + (threadIdx.x >> 5);
     const int nwarps = n_cta * kWarps;
-    const int items = sh.nA * a.T * 2;                   // half tiles of 512 tokens
+    const int items = sh.nA * a.T;
     uint32_t over_p = 0u, over_q = 0u;                   // cells beyond the last edge: always above s
     for (int item = warp; item < items; item += nwarps) {
-        const int tile = item >> 1, half = item & 1;
-        const int i = tile / a.T, t = tile - i * a.T;
+        const int i = item / a.T, t = item - i * a.T;
         const int row = sh.A[i];
         const float *rp = a.zp + (int64_t)row * a.stride;
         const float *rq = a.zq + (int64_t)row * a.stride;
         const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
-        float4 vp[4], vq[4];
-        const int e0 = t * kTile + half * (kTile / 2);
-        load_half_tile(rp, e0, a.V, al, lane, vp);
-        load_half_tile(rq, e0, a.V, al, lane, vq);
         const float bp = sh.bp[i], bq = sh.bq[i];
+        float res1 = 0.f;                                // sum of (p - q)+ over the tile: residual mass at s = 1
 #pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const float zp4[4] = {vp[it].x, vp[it].y, vp[it].z, vp[it].w};
-            const float zq4[4] = {vq[it].x, vq[it].y, vq[it].z, vq[it].w};
+        for (int half = 0; half < 2; ++half) {
+            float4 vp[4], vq[4];
+            const int e0 = t * kTile + half * (kTile / 2);
+            load_half_tile(rp, e0, a.V, al, lane, vp);
+            load_half_tile(rq, e0, a.V, al, lane, vq);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float xp = fmaf(zp4[c], a.k2, bp), xq = fmaf(zq4[c], a.k2, bq);
-                const float dl = xp - xq;                       // log2(rho); NaN compares false
-                if (dl > 0.f) {
-                    const uint32_t fp = __float2uint_rn(exp2f(xp) * kFix);
-                    const uint32_t fq = __float2uint_rn(exp2f(xq) * kFix);
-                    const float bf = dl * binscale;
-                    if (bf < (float)kBins) {
-                        const int bin = (int)bf;
-                        atomicAdd(hp + bin, fp);
-                        atomicAdd(hq + bin, fq);
-                    } else {
-                        over_p += fp;
-                        over_q += fq;
+            for (int it = 0; it < 4; ++it) {
+                const float zp4[4] = {vp[it].x, vp[it].y, vp[it].z, vp[it].w};
+                const float zq4[4] = {vq[it].x, vq[it].y, vq[it].z, vq[it].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float xp = fmaf(zp4[c], a.k2, bp), xq = fmaf(zq4[c], a.k2, bq);
+                    const float dl = xp - xq;                       // log2(rho); NaN compares false
+                    if (dl > 0.f) {
+                        const float pm = exp2f(xp), qm = exp2f(xq);
+                        res1 += fmaxf(pm - qm, 0.f);
+                        const uint32_t fp = __float2uint_rn(pm * kFix);
+                        const uint32_t fq = __float2uint_rn(qm * kFix);
+                        const float bf = dl * binscale;
+                        if (bf < (float)kBins) {
+                            const int bin = (int)bf;
+                            atomicAdd(hp + bin, fp);
+                            atomicAdd(hq + bin, fq);
+                        } else {
+                            over_p += fp;
+                            over_q += fq;
+                        }
                     }
                 }
             }
         }
+        // tile sums of the residual after ONE rejection (s_1 = 1): what a completion draw at run
+        // position 2 searches, so that this common case needs no second pass over the rows
+        const double tot = warp_sum((double)res1);
+        if (lane == 0) sums1[item] = tot;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -540,17 +554,24 @@ __device__ int draw_cell(const VerifyArgs &a, const Shared &sh, double u, bool u
         target = u * z_res;
         tile = locate_tile([&](int i) { return __ldcg(res_sums + i); }, sh.nA * a.T, target, lane, &before);
     } else {
+        // p_beam: first the live parent (its row holds exactly its beam weight), then the tile
         double z = 0.0;
         for (int i = 0; i < sh.nA; ++i) z += sh.wp[i];
         target = u * z;
-        const int T = a.T;
-        tile = locate_tile([&](int i) {
-            const int ia = i / T;
-            const int row = sh.A[ia];
-            const TileStat ts = a.stats[(int64_t)row * T + (i - ia * T)];
+        double row_before = 0.0;
+        const int ia = locate_tile([&](int i) { return sh.wp[i]; }, sh.nA, target, lane, &row_before);
+        if (ia < 0) return -1;
+        const int T = a.T, row = sh.A[ia];
+        const double wpa = sh.wp[ia], lse_row = a.lse[row];
+        double in_row = 0.0;
+        const int t = locate_tile([&](int i) {
+            const TileStat ts = a.stats[(int64_t)row * T + i];
             if (!(ts.sum > 0.f)) return 0.0;
-            return sh.wp[ia] * (double)ts.sum * exp((double)ts.mx * a.inv_tau - a.lse[row]);
-        }, sh.nA * a.T, target, lane, &before);
+            return wpa * (double)ts.sum * exp((double)ts.mx * a.inv_tau - lse_row);
+        }, T, target - row_before, lane, &in_row);
+        if (t < 0) return -1;
+        tile = ia * T + t;
+        before = row_before + in_row;
     }
     if (tile < 0) return -1;
     const int ia = tile / a.T;
@@ -577,7 +598,7 @@ k_verify(VerifyArgs a) {
     __shared__ Shared sh;
     __shared__ double sp_live[kMaxLive], sq_live[kMaxLive];
     __shared__ int8_t st[kMaxLive * kMaxLive];     // status of the request's nodes, local index
-    __shared__ uint32_t hp[kBins + 2], hq[kBins + 2];   // p and q mass per ratio bin, fixed point
+    __shared__ __align__(16) uint32_t hp[kBins + 2], hq[kBins + 2];   // p and q mass per ratio bin, fixed point
 
     const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
     const int n_lo = a.beam_node_off[b_lo], n_hi = a.beam_node_off[b_hi];
@@ -591,8 +612,123 @@ k_verify(VerifyArgs a) {
     int n_out = 0;
     int ts_n = 0; (void)ts_n;
 
-    // ---- set-up ----
     TS(1);
+    if (!a.select_mode) {
+        // ---- log-sum-exp of every row of the request from the dense pass's tile statistics ----
+        const int n_req = n_hi - n_lo;
+        const int cw = cta_rank * kWarps + warp, ncw = n_cta * kWarps;
+        for (int task = cw; task < 2 * n_req; task += ncw) {
+            const int model = task / n_req, row = n_lo + (task - model * n_req);
+            const TileStat *ts = a.stats + ((int64_t)model * a.N + row) * a.T;
+            double mx = -INFINITY;
+            for (int t = lane; t < a.T; t += 32) mx = fmax(mx, (double)ts[t].mx);
+            mx = warp_max(mx);
+            double acc = 0.0;
+            if (mx > -INFINITY)
+                for (int t = lane; t < a.T; t += 32)
+                    if (ts[t].sum > 0.f) acc += (double)ts[t].sum * exp(((double)ts[t].mx - mx) * a.inv_tau);
+            acc = warp_sum(acc);
+            if (lane == 0) {
+                const double v = (mx > -INFINITY) ? mx * a.inv_tau + log(acc) : -INFINITY;
+                a.lse_w[(int64_t)model * a.N + row] = v;
+                float *o = model ? a.out.lse_q : a.out.lse_p;
+                if (o) o[row] = (float)v;
+            }
+        }
+        __threadfence();
+        cluster.sync();
+        // ---- log-prob of every draft token given its parent (all nodes at once) ----
+        for (int i = cta_rank * kThreads + threadIdx.x; i < n_req; i += n_cta * kThreads) {
+            const int n = n_lo + i, par = a.parent[n];
+            double lp = 0.0, lq = 0.0;
+            if (par >= 0) {
+                const int tok = a.token[n];
+                if (par < n_lo || par >= n) {
+                    report(a.status, DSBD_DEV_BAD_FOREST);
+                    lp = lq = -INFINITY;
+                } else if (tok < 0 || tok >= a.V) {
+                    report(a.status, DSBD_DEV_BAD_TOKEN);
+                    lp = lq = -INFINITY;
+                } else {
+                    lp = (double)a.zp[(int64_t)par * a.stride + tok] * a.inv_tau - a.lse_w[par];
+                    lq = (double)a.zq[(int64_t)par * a.stride + tok] * a.inv_tau - a.lse_w[a.N + par];
+                }
+            }
+            a.score_w[n] = lp;
+            a.score_w[a.N + n] = lq;
+        }
+        __threadfence();
+        cluster.sync();
+        // ---- cumulative beam scores and depths (rank 0 of the cluster) ----
+        if (writer) {
+            if (n_req <= 1024) {
+                // stage the per-node log-probs in shared memory (the histogram arrays are idle
+                // here), then every node sums its own path to the root
+                double *slp = reinterpret_cast<double *>(hp), *slq = reinterpret_cast<double *>(hq);
+                for (int i = threadIdx.x; i < n_req; i += kThreads) {
+                    slp[i] = a.score_w[n_lo + i];
+                    slq[i] = a.score_w[a.N + n_lo + i];
+                }
+                __syncthreads();
+                for (int b = b_lo + (int)threadIdx.x; b < b_hi; b += kThreads) {
+                    const int root = a.beam_node_off[b];
+                    if (a.parent[root] != -1) report(a.status, DSBD_DEV_BAD_FOREST);
+                    slp[root - n_lo] = (double)a.root_logp[b];
+                    slq[root - n_lo] = (double)a.root_logq[b];
+                }
+                __syncthreads();
+                for (int i = threadIdx.x; i < n_req; i += kThreads) {
+                    double sp = 0.0, sq = 0.0;
+                    int dep = 0, cur = i;
+                    while (true) {
+                        sp += slp[cur];
+                        sq += slq[cur];
+                        const int par = a.parent[n_lo + cur];
+                        if (par < n_lo || par >= n_lo + cur) break;      // root (-1) or malformed
+                        cur = par - n_lo;
+                        if (++dep > a.gamma) { report(a.status, DSBD_DEV_BAD_FOREST); break; }
+                    }
+                    a.score_w[n_lo + i] = sp;
+                    a.score_w[a.N + n_lo + i] = sq;
+                    a.depth_w[n_lo + i] = dep;
+                    if (a.out.node_logp) a.out.node_logp[n_lo + i] = (float)sp;
+                    if (a.out.node_logq) a.out.node_logq[n_lo + i] = (float)sq;
+                }
+                __syncthreads();
+            } else {
+                for (int b = b_lo + (int)threadIdx.x; b < b_hi; b += kThreads) {
+                    const int lo = a.beam_node_off[b], hi = a.beam_node_off[b + 1];
+                    for (int n = lo; n < hi; ++n) {
+                        const int par = a.parent[n];
+                        double sp, sq;
+                        int dep = 0;
+                        if (n == lo) {
+                            sp = (double)a.root_logp[b];
+                            sq = (double)a.root_logq[b];
+                            if (par != -1) report(a.status, DSBD_DEV_BAD_FOREST);
+                        } else if (par < lo || par >= n) {
+                            sp = sq = -INFINITY;
+                            dep = a.gamma + 1;
+                        } else {
+                            sp = a.score_w[par] + a.score_w[n];
+                            sq = a.score_w[a.N + par] + a.score_w[a.N + n];
+                            dep = a.depth_w[par] + 1;
+                            if (dep > a.gamma) report(a.status, DSBD_DEV_BAD_FOREST);
+                        }
+                        a.score_w[n] = sp;
+                        a.score_w[a.N + n] = sq;
+                        a.depth_w[n] = dep;
+                        if (a.out.node_logp) a.out.node_logp[n] = (float)sp;
+                        if (a.out.node_logq) a.out.node_logq[n] = (float)sq;
+                    }
+                }
+            }
+        }
+        __threadfence();
+        cluster.sync();
+    }
+
+    // ---- set-up ----
     for (int i = cta_rank * kThreads + threadIdx.x; i < 2 * hist_len; i += n_cta * kThreads) ghist[i] = 0ull;
     if (warp == 0) {
         if (lane == 0) {
@@ -714,7 +850,8 @@ k_verify(VerifyArgs a) {
             const double top = log2((double)(m > 2 ? m : 2));          // s_j <= j <= m
             const float binscale = (float)((double)kBins / top);
             unsigned long long *gh = ghist + sh.bank * hist_len;
-            histogram_pass(a, sh, binscale, hp, hq, cta_rank, n_cta);
+            histogram_pass(a, sh, binscale, hp, hq, sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride, cta_rank,
+                           n_cta);
             __syncthreads();
             TS(4);
             for (int i = threadIdx.x; i <= kBins; i += blockDim.x)
@@ -731,24 +868,27 @@ k_verify(VerifyArgs a) {
             cluster.sync();                            // everyone has read the bank: it can be cleared
             for (int i = cta_rank * kThreads + threadIdx.x; i < hist_len; i += n_cta * kThreads) gh[i] = 0ull;
             TS(6);
-            // in-place suffix sums: hp[k] = p mass of the bins >= k (warp 0, 129 bins per lane)
-            if (warp == 0) {
-                constexpr int per = (kBins + 1 + 31) / 32;
-                const int lo = lane * per, hi = min(lo + per, kBins + 1);
+            // in-place suffix sums: hp[k] = p mass of the bins >= k (17 bins per thread)
+            {
+                constexpr int per = (kBins + 1 + kThreads - 1) / kThreads;
+                const int lo = min((int)threadIdx.x * per, kBins + 1), hi = min(lo + per, kBins + 1);
                 uint32_t mp_ = 0u, mq_ = 0u;
                 for (int i = lo; i < hi; ++i) { mp_ += hp[i]; mq_ += hq[i]; }
-                uint32_t ap = mp_, aq = mq_;              // inclusive scan from the top lane down
+                uint32_t ap = mp_, aq = mq_;              // suffix scan inside the warp, top lane down
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const uint32_t tp = __shfl_down_sync(kFull, ap, o), tq = __shfl_down_sync(kFull, aq, o);
                     if (lane + o < 32) { ap += tp; aq += tq; }
                 }
-                uint32_t rp_ = ap - mp_, rq_ = aq - mq_;  // mass of the lanes above
+                if (lane == 0) { sh.wtot_p[warp] = ap; sh.wtot_q[warp] = aq; }
+                __syncthreads();
+                uint32_t rp_ = ap - mp_, rq_ = aq - mq_;  // mass of the lanes above in this warp
+                for (int w = warp + 1; w < kWarps; ++w) { rp_ += sh.wtot_p[w]; rq_ += sh.wtot_q[w]; }
                 for (int i = hi - 1; i >= lo; --i) {
                     rp_ += hp[i]; rq_ += hq[i];
                     hp[i] = rp_; hq[i] = rq_;
                 }
-                if (lane == 0) { hp[kBins + 1] = 0u; hq[kBins + 1] = 0u; }
+                if (threadIdx.x == 0) { hp[kBins + 1] = 0u; hq[kBins + 1] = 0u; }
             }
             __syncthreads();
 
@@ -880,7 +1020,7 @@ k_verify(VerifyArgs a) {
         TS(9);
         // ---- a residual draw locates its tile through tile sums of max(p_beam - s_{j-1} q_beam, 0) ----
         double *res_sums = sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride;   // slot 0 of the bank
-        if (!a.select_mode && !sh.err && sh.res_j > 1) {
+        if (!a.select_mode && !sh.err && sh.res_j > 2) {          // run position 2 is served by the histogram pass
             residual_pass(a, sh, (float)sh.s_arr[sh.res_j - 1], res_sums, cta_rank, n_cta);
             __threadfence();
             cluster.sync();
@@ -921,17 +1061,22 @@ k_verify(VerifyArgs a) {
                     sh.done = 1;
                     if (writer) a.out.l_last[r] = l;
                 }
-            } else if (lane == 0) {
+            } else {
                 // the accepted drafts, ascending node id, are the next layer's input beams
                 int nA = 0;
-                for (int n = 0; n < n_req_nodes; ++n)
-                    if (a.depth[n_lo + n] == l && st[n] == DSBD_NODE_ACCEPTED) {
-                        sh.A[nA] = n_lo + n;
-                        sp_live[nA] = a.score[n_lo + n];
-                        sq_live[nA] = a.score[a.N + n_lo + n];
-                        ++nA;
+                for (int base = 0; base < n_req_nodes; base += 32) {
+                    const int n = base + lane;
+                    const bool in = n < n_req_nodes && a.depth[n_lo + n] == l && st[n] == DSBD_NODE_ACCEPTED;
+                    const unsigned mask = __ballot_sync(kFull, in);
+                    const int pos = nA + __popc(mask & ((1u << lane) - 1));
+                    if (in && pos < kMaxLive) {
+                        sh.A[pos] = n_lo + n;
+                        sp_live[pos] = a.score[n_lo + n];
+                        sq_live[pos] = a.score[a.N + n_lo + n];
                     }
-                sh.nA = nA;
+                    nA += __popc(mask);
+                }
+                if (lane == 0) sh.nA = nA;
             }
             if (lane == 0 && err) sh.err = err;
         }
@@ -1014,7 +1159,8 @@ int cluster_size_for(int tiles, int R) {
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     int cs = 1;
-    if (tiles >= 64) cs = 8;
+    if (tiles >= 256) cs = 16;
+    else if (tiles >= 64) cs = 8;
     else if (tiles >= 32) cs = 4;
     else if (tiles >= 16) cs = 2;
     while (cs > 1 && (long long)R * cs > 4ll * sms) cs >>= 1;
@@ -1023,6 +1169,8 @@ int cluster_size_for(int tiles, int R) {
 
 int launch_verify(const VerifyArgs &args, int R, int tiles, cudaStream_t stream) {
     const int cs = cluster_size_for(tiles, R);
+    if (cs > 8 && cudaFuncSetAttribute(k_verify, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+        return DSBD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(R * cs));
     cfg.blockDim = dim3(kThreads);
@@ -1085,14 +1233,6 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
     const int64_t items = (int64_t)2 * f->N * L.T;
     k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_p, logits_q, row_stride, p->V, L.T,
                                                             f->N, f->N, nullptr, nullptr, k2, stats);
-    {
-        const int64_t warps = (int64_t)2 * f->N;
-        k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
-            stats, L.T, f->N, f->N, nullptr, nullptr, inv_tau, lse, out->lse_p, out->lse_q);
-    }
-    k_tree_scores<<<(f->B + 127) / 128, 128, 0, stream>>>(
-        f->B, f->beam_node_off, f->parent, f->token, logits_p, logits_q, row_stride, p->V, f->max_depth,
-        inv_tau, root_logp, root_logq, lse, f->N, score, depth, out->node_logp, out->node_logq, status);
     if (cudaGetLastError() != cudaSuccess) return DSBD_ERR_CUDA;
 
     VerifyArgs a = {};
@@ -1112,6 +1252,8 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
     a.dbg = reinterpret_cast<unsigned long long *>(ws + L.total) - (size_t)f->R * 256;
 #endif
     a.out = *out; a.status = status; a.select_mode = 0;
+    a.lse_w = lse; a.score_w = score; a.depth_w = depth;
+    a.root_logp = root_logp; a.root_logq = root_logq;
     return launch_verify(a, f->R, L.max_live * L.T, stream);
 }
 

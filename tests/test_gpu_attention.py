@@ -90,6 +90,20 @@ def test_ragged_prefixes_and_tree_shapes(dtype, Hq, Hkv, d):
     attention_close(to_host_f32(out), ref, bf16=dtype == torch.bfloat16)
 
 
+@pytest.mark.parametrize("Hq,Hkv,max_nodes", [(8, 2, 32), (16, 2, 16), (4, 4, 64), (32, 8, 9)])
+def test_tensor_core_kernel_row_counts(Hq, Hkv, max_nodes):
+    """bf16, d = 128: the tcgen05 kernel with 64-row and with 128-row query tiles (nodes x group
+    up to 128), ragged prefixes around its 64-token tiles."""
+    rng = np.random.default_rng(Hq * 7 + max_nodes)
+    rand_tree = lambda n: [-1] + [int(rng.integers(0, i)) for i in range(1, n)]
+    trees = [rand_tree(max_nodes), [-1], rand_tree(max(2, max_nodes // 2)), rand_tree(max_nodes), rand_tree(3)]
+    L = [63, 64, 65, 700, 1]
+    forest, spec, t, poff = _custom(rng, trees, L, Hq, Hkv, 128, torch.bfloat16)
+    out = _gpu(forest, spec, t, poff)
+    nodes, ref = _oracle_beams(forest, spec, t, poff, list(range(len(trees))))
+    attention_close(to_host_f32(out), ref, bf16=True)
+
+
 def test_host_side_errors():
     rng = np.random.default_rng(0)
     forest, spec, t, poff = _custom(rng, [[-1, 0]], [8], 4, 4, 64, torch.bfloat16)
