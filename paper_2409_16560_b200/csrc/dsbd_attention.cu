@@ -223,7 +223,7 @@ int check(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
 
 extern "C" size_t dsbd_forest_attention_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     if (check(f, d) != DSBD_OK) return 0;
-    return 256;
+    return attention_tc_supported(f, d) ? attention_tc_workspace(f, d) : 256;
 }
 
 extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q,
@@ -245,7 +245,8 @@ extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_des
     // DSBD_ATTN_IMPL=simt forces the CUDA-core kernel (debugging aid)
     const char *impl = getenv("DSBD_ATTN_IMPL");
     if (!(impl && strcmp(impl, "simt") == 0) && attention_tc_supported(f, d))
-        return launch_attention_tc(f, d, q, k_new, v_new, k_prefix, v_prefix, prefix_off, out, status, stream);
+        return launch_attention_tc(f, d, q, k_new, v_new, k_prefix, v_prefix, prefix_off, out, workspace,
+                                   workspace_bytes, status, stream);
 
     AttnArgs a = {};
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;

@@ -49,8 +49,17 @@ constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;
 constexpr long long kWaitCycles = 2000000000ll;   // about a second
 
+// One work item: the query rows of unit (b, g) against the prefix tokens [t0, t1) of its beam,
+// plus the tree tile when `last`.  A unit split into several items leaves partial results
+// (reference maximum, row sum, unnormalised O) that a second kernel merges.
+struct AttnItem { int b, g, t0, t1, last, nparts, slot, pad; };
+
 struct TcArgs {
     int B, N, Hq, Hkv, group, n_units;
+    int max_rows;                     // max over trees of nodes * group
+    const AttnItem *items;            // nullptr: one item per unit, in unit order
+    const int *n_items;               // device count of items (with items)
+    float *partial;                   // [slot][max_rows][130]: m_ref, l, O[128]
     float scale_log2;
     const int32_t *beam_node_off, *parent;
     const int64_t *prefix_off;
@@ -165,6 +174,16 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
            ((uint32_t)(M >> 4) << 24);
 }
 
+__device__ __forceinline__ int item_count(const TcArgs &a) { return a.items ? *a.n_items : a.n_units; }
+__device__ __forceinline__ AttnItem get_item(const TcArgs &a, int it) {
+    if (a.items) return a.items[it];
+    AttnItem x;
+    x.b = it / a.Hkv; x.g = it - x.b * a.Hkv;
+    x.t0 = 0; x.t1 = (int)(a.prefix_off[x.b + 1] - a.prefix_off[x.b]);
+    x.last = 1; x.nparts = 1; x.slot = 0; x.pad = 0;
+    return x;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t *>(&v);
@@ -210,13 +229,16 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
         if (lane == 0) {
             uint32_t tile = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
-                const int b = u / a.Hkv, g = u - b * a.Hkv;
+            const int n_items = item_count(a);
+            for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
+                const AttnItem item = get_item(a, u);
+                const int b = item.b, g = item.g;
                 const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
-                const int64_t row0 = a.prefix_off[b] * a.Hkv + (int64_t)g * L;
-                const int nt_p = (int)((L + kBN - 1) / kBN);
+                const int64_t row0 = a.prefix_off[b] * a.Hkv + (int64_t)g * L + item.t0;
+                const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
                 const int n_lo = a.beam_node_off[b];
-                for (int j = 0; j <= nt_p && ok; ++j, ++tile) {
+                const int nt = nt_p + item.last;
+                for (int j = 0; j < nt && ok; ++j, ++tile) {
                     const int s = tile % kStages;
                     const uint32_t par = (tile / kStages) & 1;
                     ok = mbar_wait(&sb.kv_empty[s], par ^ 1, &sb, a.status);
@@ -256,10 +278,10 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             uint32_t tile = 0, unit = 0;
             bool ok = true;
             const uint64_t qd = desc_k_major(smem_u32(q_s));
-            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++unit) {
-                const int b = u / a.Hkv;
-                const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
-                const int nt = (int)((L + kBN - 1) / kBN) + 1;
+            const int n_items = item_count(a);
+            for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x, ++unit) {
+                const AttnItem item = get_item(a, u);
+                const int nt = (item.t1 - item.t0 + kBN - 1) / kBN + item.last;
                 ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
                 // S(t) = Q K(t)^T into S buffer t & 1; issued one tile ahead of the P V product so
                 // that it runs while the softmax warps work on the previous tile
@@ -301,10 +323,13 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         uint32_t tile = 0, unit = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++unit) {
-            const int b = u / a.Hkv, g = u - b * a.Hkv;
-            const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
-            const int nt_p = (int)((L + kBN - 1) / kBN);
+        const int n_items = item_count(a);
+        for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x, ++unit) {
+            const AttnItem item = get_item(a, u);
+            const int b = item.b, g = item.g;
+            const int64_t L = item.t1;                         // tokens beyond t1 belong to other items
+            const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
+            const int nt = nt_p + item.last;
             const int n_lo = a.beam_node_off[b];
             const int n_tree = a.beam_node_off[b + 1] - n_lo;
             const int M = n_tree * a.group;
@@ -340,7 +365,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 }
             }
             float m_ref = -INFINITY, l_run = 0.f;
-            for (int j = 0; j <= nt_p && ok; ++j, ++tile) {
+            for (int j = 0; j < nt && ok; ++j, ++tile) {
                 ok = mbar_wait(&sb.s_full[tile & 1], (tile >> 1) & 1, &sb, a.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -356,7 +381,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     unsigned long long vis;
                     if (tree) vis = my_anc & (n_tree >= 64 ? ~0ull : ((1ull << n_tree) - 1));
                     else {
-                        const int64_t left = L - (int64_t)j * kBN;
+                        const int64_t left = L - item.t0 - (int64_t)j * kBN;
                         vis = left >= 64 ? ~0ull : ((1ull << left) - 1);
                     }
 #pragma unroll
@@ -412,22 +437,40 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             if (warp_active) {
-                const float inv = active ? 1.f / l_run : 0.f;
-                __nv_bfloat16 *dst = a.out + ((int64_t)(n_lo + node) * a.Hq + hq) * kD;
+                if (item.nparts == 1) {
+                    const float inv = active ? 1.f / l_run : 0.f;
+                    __nv_bfloat16 *dst = a.out + ((int64_t)(n_lo + node) * a.Hq + hq) * kD;
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t ov[32];
-                    tmem_ld32(tmem + lane_base + kColO + cc * 32, ov);
-                    tmem_wait_ld();
-                    if (active) {
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t ov[32];
+                        tmem_ld32(tmem + lane_base + kColO + cc * 32, ov);
+                        tmem_wait_ld();
+                        if (active) {
 #pragma unroll
-                        for (int c = 0; c < 32; c += 8) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
-                            w.y = pack_bf16(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
-                            w.z = pack_bf16(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
-                            w.w = pack_bf16(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(dst + cc * 32 + c) = w;
+                            for (int c = 0; c < 32; c += 8) {
+                                uint4 w;
+                                w.x = pack_bf16(__uint_as_float(ov[c]) * inv, __uint_as_float(ov[c + 1]) * inv);
+                                w.y = pack_bf16(__uint_as_float(ov[c + 2]) * inv, __uint_as_float(ov[c + 3]) * inv);
+                                w.z = pack_bf16(__uint_as_float(ov[c + 4]) * inv, __uint_as_float(ov[c + 5]) * inv);
+                                w.w = pack_bf16(__uint_as_float(ov[c + 6]) * inv, __uint_as_float(ov[c + 7]) * inv);
+                                *reinterpret_cast<uint4 *>(dst + cc * 32 + c) = w;
+                            }
+                        }
+                    }
+                } else {
+                    // partial result of this part of the unit: reference maximum, row sum, raw O
+                    float *dst = a.partial + ((int64_t)item.slot * a.max_rows + row) * 130;
+                    if (active) { dst[0] = m_ref; dst[1] = l_run; }
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t ov[32];
+                        tmem_ld32(tmem + lane_base + kColO + cc * 32, ov);
+                        tmem_wait_ld();
+                        if (active) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2)
+                                *reinterpret_cast<float2 *>(dst + 2 + cc * 32 + c) =
+                                    make_float2(__uint_as_float(ov[c]), __uint_as_float(ov[c + 1]));
                         }
                     }
                 }
@@ -440,6 +483,129 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
     if (warp == 5) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Work plan for ragged or small batches: every unit's prefix is cut into parts of at most
+// `chunk` tokens (equal parts, multiples of 64), and the items are ordered by decreasing tile
+// count, so that handing item i to CTA i mod grid spreads the work evenly.
+// ---------------------------------------------------------------------------------------
+struct UnitParts { int first_slot, nparts; };
+
+__device__ __forceinline__ void unit_parts(int64_t L, int chunk, int *np, int *plen) {
+    int n = (int)((L + chunk - 1) / chunk);
+    if (n < 1) n = 1;
+    const int64_t per = (L + n - 1) / n;
+    *np = n;
+    *plen = (int)((per + kBN - 1) / kBN) * kBN;
+}
+
+__global__ void __launch_bounds__(1024)
+k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, AttnItem *__restrict__ items,
+            int *__restrict__ n_items, UnitParts *__restrict__ units) {
+    __shared__ int bucket[1024];
+    __shared__ int scan[1024];
+    __shared__ int carry;
+    const int tid = threadIdx.x, n_units = B * Hkv;
+    bucket[tid] = 0;
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    // slots: exclusive scan of the part counts over the units, 1024 units at a time
+    for (int base = 0; base < n_units; base += 1024) {
+        const int u = base + tid;
+        int np = 0, plen = 0;
+        if (u < n_units) {
+            const int b = u / Hkv;
+            unit_parts(prefix_off[b + 1] - prefix_off[b], chunk, &np, &plen);
+        }
+        scan[tid] = np;
+        __syncthreads();
+        for (int o = 1; o < 1024; o <<= 1) {
+            const int v = tid >= o ? scan[tid - o] : 0;
+            __syncthreads();
+            scan[tid] += v;
+            __syncthreads();
+        }
+        if (u < n_units) {
+            units[u].first_slot = carry + scan[tid] - np;
+            units[u].nparts = np;
+            const int b = u / Hkv;
+            const int64_t L = prefix_off[b + 1] - prefix_off[b];
+            for (int p = 0; p < np; ++p) {
+                const int64_t t0 = (int64_t)p * plen;
+                const int64_t t1 = t0 + plen < L ? t0 + plen : L;
+                int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
+                atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
+            }
+        }
+        __syncthreads();
+        if (tid == 0) carry += scan[1023];
+        __syncthreads();
+    }
+    // start of every bucket in the output, largest tile count first
+    scan[tid] = bucket[1023 - tid];
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {
+        const int v = tid >= o ? scan[tid - o] : 0;
+        __syncthreads();
+        scan[tid] += v;
+        __syncthreads();
+    }
+    const int start = scan[tid] - bucket[1023 - tid];
+    __syncthreads();
+    bucket[1023 - tid] = start;                 // bucket[k] becomes the cursor of tile count k
+    if (tid == 0) *n_items = carry;
+    __syncthreads();
+    for (int u = tid; u < n_units; u += 1024) {
+        const int b = u / Hkv, g = u - b * Hkv;
+        const int64_t L = prefix_off[b + 1] - prefix_off[b];
+        int np, plen;
+        unit_parts(L, chunk, &np, &plen);
+        for (int p = 0; p < np; ++p) {
+            const int64_t t0 = (int64_t)p * plen;
+            const int64_t t1 = t0 + plen < L ? t0 + plen : L;
+            const int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
+            const int pos = atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
+            AttnItem it;
+            it.b = b; it.g = g; it.t0 = (int)t0; it.t1 = (int)t1; it.last = (p == np - 1);
+            it.nparts = np; it.slot = units[u].first_slot + p; it.pad = 0;
+            items[pos] = it;
+        }
+    }
+}
+
+// Merge the parts of every split unit: out = sum_c O_c 2^(m_c - m) / sum_c l_c 2^(m_c - m).
+__global__ void __launch_bounds__(128)
+k_attn_combine(TcArgs a, const UnitParts *__restrict__ units) {
+    const int u = blockIdx.x;
+    const UnitParts up = units[u];
+    if (up.nparts <= 1) return;
+    const int b = u / a.Hkv, g = u - b * a.Hkv;
+    const int n_lo = a.beam_node_off[b];
+    const int M = (a.beam_node_off[b + 1] - n_lo) * a.group;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int row = warp; row < M; row += 4) {
+        float m = -INFINITY;
+        for (int c = 0; c < up.nparts; ++c)
+            m = fmaxf(m, a.partial[((int64_t)(up.first_slot + c) * a.max_rows + row) * 130]);
+        float l = 0.f;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < up.nparts; ++c) {
+            const float *src = a.partial + ((int64_t)(up.first_slot + c) * a.max_rows + row) * 130;
+            const float w = src[0] == -INFINITY ? 0.f : exp2f(src[0] - m);
+            l += src[1] * w;
+            const float2 x = *reinterpret_cast<const float2 *>(src + 2 + lane * 4);
+            const float2 y = *reinterpret_cast<const float2 *>(src + 4 + lane * 4);
+            o.x += x.x * w; o.y += x.y * w; o.z += y.x * w; o.w += y.y * w;
+        }
+        const float inv = 1.f / l;
+        const int node = row / a.group, hq = g * a.group + (row - node * a.group);
+        __nv_bfloat16 *dst = a.out + ((int64_t)(n_lo + node) * a.Hq + hq) * kD + lane * 4;
+        uint2 w2;
+        w2.x = pack_bf16(o.x * inv, o.y * inv);
+        w2.y = pack_bf16(o.z * inv, o.w * inv);
+        *reinterpret_cast<uint2 *>(dst) = w2;
     }
 }
 
@@ -472,6 +638,45 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Launch shape shared by the workspace query and the launch.
+struct TcPlan {
+    int grid, chunk;          // chunk == 0: one item per unit, no plan kernel
+    int64_t items_max;
+    size_t off_items, off_units, off_partial, total;
+};
+
+TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+    TcPlan p = {};
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int group = d->Hq / d->Hkv;
+    const bool small_q = f->max_tree_nodes * group <= 64;
+    p.grid = small_q ? 2 * sms : sms;
+    const int64_t n_units = (int64_t)f->B * d->Hkv;
+    // Splitting a unit costs a pipeline drain, a Q reload and a partial result per part, so it
+    // pays only when there are fewer units than CTAs: then the prefix is cut so that about two
+    // items per CTA exist, in parts of at least 512 tokens.
+    int64_t c = (int64_t)d->total_prefix * d->Hkv / (2ll * p.grid);
+    if (c < 512) c = 512;
+    c = (c + kBN - 1) / kBN * kBN;
+    if (n_units >= p.grid || c >= d->max_prefix) {
+        p.chunk = 0;
+        p.items_max = n_units;
+        if (p.grid > n_units) p.grid = (int)n_units;
+        p.total = 256;
+        return p;
+    }
+    p.chunk = (int)c;
+    p.items_max = (int64_t)d->Hkv * (d->total_prefix / c + f->B);
+    size_t off = 256;
+    p.off_items = off;   off = align_up(off + sizeof(AttnItem) * (size_t)p.items_max, 256);
+    p.off_units = off;   off = align_up(off + sizeof(UnitParts) * (size_t)n_units, 256);
+    p.off_partial = off; off = align_up(off + sizeof(float) * 130 * (size_t)p.items_max * (size_t)(f->max_tree_nodes * group), 256);
+    p.total = off;
+    if (p.grid > p.items_max) p.grid = (int)p.items_max;
+    return p;
+}
+
 }  // namespace
 
 namespace dsbd {
@@ -485,30 +690,43 @@ bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     return encode_fn() != nullptr;
 }
 
+size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) { return make_plan(f, d).total; }
+
 int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
                         const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
-                        void *out, int32_t *status, cudaStream_t stream) {
+                        void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream) {
     CUtensorMap kp, vp, kn, vn;
     const uint64_t prows = (uint64_t)d->total_prefix * d->Hkv;
     if (!make_map(&kp, k_prefix, kD, prows, kD * 2) || !make_map(&vp, v_prefix, kD, prows, kD * 2) ||
         !make_map(&kn, k_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2) ||
         !make_map(&vn, v_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2))
         return DSBD_ERR_CUDA;
+    const TcPlan plan = make_plan(f, d);
+    if (workspace_bytes < plan.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    char *ws = static_cast<char *>(workspace);
     TcArgs a = {};
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;
     a.n_units = f->B * d->Hkv;
+    a.max_rows = f->max_tree_nodes * a.group;
     a.scale_log2 = d->scale * 1.4426950408889634f;
     a.beam_node_off = f->beam_node_off; a.parent = f->parent; a.prefix_off = prefix_off;
     a.q = static_cast<const __nv_bfloat16 *>(q);
     a.out = static_cast<__nv_bfloat16 *>(out);
     a.status = status;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    int grid = sms * 2;
-    if (grid > a.n_units) grid = a.n_units;
+    UnitParts *units = nullptr;
+    if (plan.chunk > 0) {
+        if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+        AttnItem *items = reinterpret_cast<AttnItem *>(ws + plan.off_items);
+        units = reinterpret_cast<UnitParts *>(ws + plan.off_units);
+        int *n_items = reinterpret_cast<int *>(ws);
+        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, plan.chunk, items, n_items, units);
+        a.items = items;
+        a.n_items = n_items;
+        a.partial = reinterpret_cast<float *>(ws + plan.off_partial);
+    }
+    const int grid = plan.grid;
     // up to 64 query rows: 16 KB of Q, three stages, two CTAs per SM; more rows: one CTA per SM
-    const bool small_q = f->max_tree_nodes * a.group <= 64;
-    if (!small_q && grid > sms) grid = sms;
+    const bool small_q = a.max_rows <= 64;
 #define DSBD_LAUNCH_TC(QR, ST)                                                                              \
     do {                                                                                                   \
         constexpr uint32_t bytes = smem_bytes(QR, ST);                                                     \
@@ -520,6 +738,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     if (small_q) DSBD_LAUNCH_TC(64, 3);
     else DSBD_LAUNCH_TC(128, 3);
 #undef DSBD_LAUNCH_TC
+    if (plan.chunk > 0) k_attn_combine<<<a.n_units, 128, 0, stream>>>(a, units);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 

@@ -104,6 +104,18 @@ def test_tensor_core_kernel_row_counts(Hq, Hkv, max_nodes):
     attention_close(to_host_f32(out), ref, bf16=True)
 
 
+@pytest.mark.parametrize("L", [[5000, 3000], [9000]])
+def test_few_units_long_prefix_is_split_and_merged(L):
+    """Fewer (beam, KV head) units than CTAs: the prefix of each unit is cut into parts that
+    different CTAs process, and their partial results are merged."""
+    rng = np.random.default_rng(len(L))
+    trees = [[-1, 0, 0, 1, 2, 2, 4][:7] for _ in L]
+    forest, spec, t, poff = _custom(rng, trees, L, 8, 2, 128, torch.bfloat16)
+    out = _gpu(forest, spec, t, poff)
+    nodes, ref = _oracle_beams(forest, spec, t, poff, list(range(len(trees))))
+    attention_close(to_host_f32(out), ref, bf16=True)
+
+
 def test_host_side_errors():
     rng = np.random.default_rng(0)
     forest, spec, t, poff = _custom(rng, [[-1, 0]], [8], 4, 4, 64, torch.bfloat16)
