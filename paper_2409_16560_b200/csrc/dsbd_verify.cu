@@ -6,19 +6,27 @@
 //                  1024-token tile the row maximum and sum of exponentials (warp-autonomous,
 //                  128-bit loads, warp-shuffle reductions).  HBM-bound; this is the pass the
 //                  algorithmic bytes 8*N*V belong to.
-//   k_row_finish   per row: log-sum-exp from the tile statistics.
-//   k_tree_scores  per tree: log-prob of every draft token given its parent, cumulative beam
-//                  scores, node depths.
-//   k_verify       one thread-block cluster per request walks the layers: live set, beam
-//                  weights, the residual masses c_{j+1} = F(s_j) (cluster-wide passes over the
-//                  live rows, reduced through a tile-sum table), the acceptance-count
-//                  recursion, the accept loop and the inverse-CDF draws.
+//   k_row_finish   per row: log-sum-exp from the tile statistics (dsbd_node_stats and
+//                  dsbd_select_width; dsbd_verify_step does this inside k_verify).
+//   k_verify       one thread-block cluster per request.  Prologue: log-sum-exp of the request's
+//                  rows, log-prob of every draft token, cumulative beam scores.  Then layer by
+//                  layer: live set and beam weights; ONE pass over the live rows that builds a
+//                  fixed-point histogram of the cells' ratios p_beam/q_beam, from which all the
+//                  residual masses c_{j+1} = F(s_j) of the layer follow without touching the
+//                  rows again; the acceptance-count recursion; the accept loop; the
+//                  inverse-CDF completion draws.
 //
 // The residual chain uses the closed form of the paper's recursion p_{k+1} = norm(max(p_k -
 // q_beam, 0)):  with F(s) = sum max(p_beam - s q_beam, 0), c_1 = 1, s_0 = 0, s_j = s_{j-1} + c_j
 // and c_{j+1} = F(s_j) one has p_j = max(p_beam - s_{j-1} q_beam, 0) / c_j, hence
 // alpha_j = 1 - c_{j+1}/c_j and the accept ratio of a draft x at run position j is
-// max(rho(x) - s_{j-1}, 0) / c_j with rho = p_beam(x)/q_beam(x).
+// max(rho(x) - s_{j-1}, 0) / c_j with rho = p_beam(x)/q_beam(x).  F(s) = P(rho > s) - s Q(rho > s)
+// only needs the p and q mass above a ratio threshold, which is what the histogram holds; the
+// one bin that s falls into is bracketed from its two sums and its edges, and when the bracket
+// is wider than 2.5e-7 that F(s_j) is recomputed exactly by a pass over the rows.
+//
+// Building with -DDSBD_PHASE_TIMING makes k_verify record %globaltimer stamps of its phases at
+// the end of the workspace (a tuning aid; off in normal builds).
 #include <cooperative_groups.h>
 #include <math.h>
 
@@ -144,50 +152,6 @@ __global__ void k_row_finish(const TileStat *__restrict__ stats, int T, int N, i
         lse[(int64_t)model * N + row] = v;
         if (model == 0 && lse_p_out) lse_p_out[row] = (float)v;
         if (model == 1 && lse_q_out) lse_q_out[row] = (float)v;
-    }
-}
-
-// Cumulative beam scores along every tree (one thread per tree) and node depths.
-__global__ void k_tree_scores(int B, const int32_t *__restrict__ beam_node_off,
-                              const int32_t *__restrict__ parent, const int32_t *__restrict__ token,
-                              const float *__restrict__ zp, const float *__restrict__ zq,
-                              int64_t stride, int V, int max_depth, double inv_tau,
-                              const float *__restrict__ root_logp, const float *__restrict__ root_logq,
-                              const double *__restrict__ lse, int N, double *__restrict__ score /*[2][N]*/,
-                              int32_t *__restrict__ depth, float *__restrict__ node_logp,
-                              float *__restrict__ node_logq, int32_t *status) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B) return;
-    const int lo = beam_node_off[b], hi = beam_node_off[b + 1];
-    for (int n = lo; n < hi; ++n) {
-        double sp, sq;
-        int dep = 0;
-        const int par = parent[n];
-        if (n == lo) {
-            sp = (double)root_logp[b];
-            sq = (double)root_logq[b];
-            if (par != -1) report(status, DSBD_DEV_BAD_FOREST);
-        } else if (par < lo || par >= n) {
-            report(status, DSBD_DEV_BAD_FOREST);
-            sp = sq = -INFINITY;
-            dep = max_depth + 1;
-        } else {
-            const int tok = token[n];
-            dep = depth[par] + 1;
-            if (dep > max_depth) report(status, DSBD_DEV_BAD_FOREST);
-            if (tok < 0 || tok >= V) {
-                report(status, DSBD_DEV_BAD_TOKEN);
-                sp = sq = -INFINITY;
-            } else {
-                sp = score[par] + ((double)zp[(int64_t)par * stride + tok] * inv_tau - lse[par]);
-                sq = score[N + par] + ((double)zq[(int64_t)par * stride + tok] * inv_tau - lse[N + par]);
-            }
-        }
-        score[n] = sp;
-        score[N + n] = sq;
-        depth[n] = dep;
-        if (node_logp) node_logp[n] = (float)sp;
-        if (node_logq) node_logq[n] = (float)sq;
     }
 }
 
