@@ -143,6 +143,28 @@ def test_ragged_vocab_unaligned_rows_masked_entries(V, pad, ninf, tree):
     check_exempt(exempt, decisions)
 
 
+@pytest.mark.parametrize("R,V,max_w,gamma", [(700, 300, 3, 2), (3, 2500, 64, 1), (40, 9000, 16, 3)])
+def test_many_requests_and_widest_layers(R, V, max_w, gamma):
+    """More requests than resident clusters (several waves, small clusters), and the limit of
+    64 beams / 64 live drafts per layer."""
+    rng = np.random.default_rng(R + V)
+    forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=R, V=V, gamma=gamma, max_w=max_w)
+    if max_w == 64:
+        prm["W_min_r"] = None
+        prm["W_min"] = 1
+    dz = lambda a: torch.as_tensor(a).cuda()
+    exempt = decisions = 0
+    for step in range(2):
+        prm["step"] = step
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+        assert status == 0
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64), threads=8)
+        e, d = compare_verify(ref, gpu, forest)
+        exempt += e
+        decisions += d
+    check_exempt(exempt, decisions)
+
+
 def test_roots_only_forest_goes_straight_to_the_extra_layer():
     rng = np.random.default_rng(3)
     V, B = 2000, 3
