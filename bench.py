@@ -317,6 +317,11 @@ def main():
     attn_ms = float(np.mean([a.elapsed_time(b) for a, b in e_attn]))
     ver_ms = float(np.mean([a.elapsed_time(b) for a, b in e_ver]))
     assert int(status.item()) == 0, "device status %d" % int(status.item())
+    st = vout["req_stats"].cpu().numpy().reshape(-1, 4).astype(float)
+    verify_stats = {"layers_per_request": float(st[:, 0].mean()), "accept_tests_per_request": float(st[:, 1].mean()),
+                    "exact_recomputations_per_request": float(st[:, 2].mean()),
+                    "extra_completion_passes_per_request": float(st[:, 3].mean()),
+                    "output_beams_per_request": float(vout["out_width"].float().mean().item())}
 
     # the dense logits pass alone (the kernel the verify roofline is quoted on)
     torch.cuda.synchronize()
@@ -412,7 +417,7 @@ def main():
                            (a_bytes + v_bytes) * 1e-9),
                        "parallelism": "replicas x%d" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+            "roofline": roofline, "kernels": kernels, "verify_stats_last_step": verify_stats, "cpu_baseline": cpu}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

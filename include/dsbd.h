@@ -153,6 +153,9 @@ typedef struct {
     float   *lse_p;         /* [N]  log-sum-exp of each tempered logits row                  */
     float   *lse_q;
     int32_t *req_error;     /* [R]  0 or a DSBD_DEV_* code                                   */
+    int32_t *req_stats;     /* [R*4] or NULL: per request {layers verified, accept tests made,
+                                    residual masses that had to be recomputed exactly by a pass
+                                    over the rows, extra passes made for completion draws}   */
 } dsbd_verify_out_t;
 
 /* One verification step (Algorithm 1 with the dynamic width of Eqs. for P, P~, alpha_j, W_L):

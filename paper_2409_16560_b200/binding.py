@@ -48,7 +48,7 @@ class VerifyParamsT(C.Structure):
 
 _OUT_FIELDS = ["l_last", "out_width", "out_off", "out_parent", "out_node", "out_root_beam",
                "out_token", "out_logp", "out_logq", "out_source", "node_status", "layer_width",
-               "node_logp", "node_logq", "lse_p", "lse_q", "req_error"]
+               "node_logp", "node_logq", "lse_p", "lse_q", "req_error", "req_stats"]
 
 
 class VerifyOutT(C.Structure):
@@ -270,6 +270,7 @@ def alloc_verify_out(forest, out_off_host, device):
         "lse_p": torch.zeros(N, dtype=f32, device=device),
         "lse_q": torch.zeros(N, dtype=f32, device=device),
         "req_error": torch.zeros(R, dtype=i32, device=device),
+        "req_stats": torch.zeros(R * 4, dtype=i32, device=device),
     }
     return o
 

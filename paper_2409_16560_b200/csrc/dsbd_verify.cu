@@ -213,6 +213,7 @@ struct Shared {
     double col_a[kMaxLive + 1], col_b[kMaxLive + 1];
     double tail[kMaxLive + 2];
     int bank, need_exact, res_j, run_j, chain_pos;
+    int n_layers, n_tests, n_exact, n_respass;
     uint32_t wtot_p[kWarps], wtot_q[kWarps];
     double rho[kMaxLive], uu[kMaxLive];     // per live draft: p_beam/q_beam and its uniform
 };
@@ -697,6 +698,7 @@ k_verify(VerifyArgs a) {
     if (warp == 0) {
         if (lane == 0) {
             sh.err = 0; sh.done = 0;
+            sh.n_layers = sh.n_tests = sh.n_exact = sh.n_respass = 0;
             if (a.select_mode) {
                 const int lo = a.live_off[r], hi = a.live_off[r + 1];
                 sh.nA = hi - lo;
@@ -894,6 +896,7 @@ k_verify(VerifyArgs a) {
                 __syncthreads();
                 if (!sh.need_exact) break;
                 const int j = sh.chain_pos;
+                if (threadIdx.x == 0) ++sh.n_exact;
                 double *sums = sums_base + ((int64_t)sh.bank * a.max_m + (j - 1)) * slot_stride;
                 residual_pass(a, sh, (float)sh.s_arr[j], sums, cta_rank, n_cta);
                 __threadfence();
@@ -951,6 +954,7 @@ k_verify(VerifyArgs a) {
                     else ratio = fmax(rho - sh.s_arr[j - 1], 0.0) / sh.c_arr[j];
                     if (ratio > 1.0) ratio = 1.0;
                     const double u = sh.uu[i];
+                    ++sh.n_tests;
                     if (u <= ratio) {
                         st[n - n_lo] = DSBD_NODE_ACCEPTED;
                         if (writer) a.out.node_status[n] = DSBD_NODE_ACCEPTED;
@@ -974,6 +978,7 @@ k_verify(VerifyArgs a) {
                     }
                 sh.W = W;
                 sh.count = count;
+                ++sh.n_layers;
                 sh.res_j = (count < W && j > 1) ? j : 0;   // residual draw at run position j needs tile sums
                 sh.run_j = j;
                 if (err) sh.err = err;
@@ -985,6 +990,7 @@ k_verify(VerifyArgs a) {
         // ---- a residual draw locates its tile through tile sums of max(p_beam - s_{j-1} q_beam, 0) ----
         double *res_sums = sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride;   // slot 0 of the bank
         if (!a.select_mode && !sh.err && sh.res_j > 2) {          // run position 2 is served by the histogram pass
+            if (threadIdx.x == 0) ++sh.n_respass;
             residual_pass(a, sh, (float)sh.s_arr[sh.res_j - 1], res_sums, cta_rank, n_cta);
             __threadfence();
             cluster.sync();
@@ -1070,6 +1076,12 @@ k_verify(VerifyArgs a) {
         if (!a.select_mode) {
             a.out.out_width[r] = n_out;
             if (a.out.req_error) a.out.req_error[r] = sh.err;
+            if (a.out.req_stats) {
+                a.out.req_stats[4 * r] = sh.n_layers;
+                a.out.req_stats[4 * r + 1] = sh.n_tests;
+                a.out.req_stats[4 * r + 2] = sh.n_exact;
+                a.out.req_stats[4 * r + 3] = sh.n_respass;
+            }
         }
         if (sh.err) report(a.status, sh.err);
     }

@@ -165,6 +165,31 @@ def test_many_requests_and_widest_layers(R, V, max_w, gamma):
     check_exempt(exempt, decisions)
 
 
+def test_peaky_distributions_use_the_exact_fallback():
+    """When the histogram bin that a residual threshold falls into holds a heavy cell its
+    bracket is too wide, and that residual mass is recomputed exactly by a pass over the rows.
+    The path must be exercised and stay in parity."""
+    rng = np.random.default_rng(11)
+    exempt = decisions = fallbacks = respass = 0
+    for trial in range(3):
+        # a small vocabulary: every cell is heavy compared with the bracket tolerance, so any
+        # threshold that shares its bin with a cell needs the exact evaluation
+        forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=200, V=64, gamma=3, max_w=6)
+        prm["step"] = trial
+        dz = lambda a: torch.as_tensor(a).cuda()
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+        assert status == 0
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64))
+        e, d = compare_verify(ref, gpu, forest)
+        exempt += e; decisions += d
+        st = gpu["req_stats"].reshape(-1, 4)
+        assert np.array_equal(st[:, 0], np.minimum(ref["l_last"], forest["max_depth"]))   # layers verified
+        assert st[:, 1].sum() == (ref["trace_kind"] == oracle.TR_ACCEPT).sum()            # accept tests
+        fallbacks += int(st[:, 2].sum()); respass += int(st[:, 3].sum())
+    check_exempt(exempt, decisions)
+    assert fallbacks > 0
+
+
 def test_roots_only_forest_goes_straight_to_the_extra_layer():
     rng = np.random.default_rng(3)
     V, B = 2000, 3
