@@ -402,10 +402,10 @@ def main():
     if not args.no_cpu_baseline:
         cpu = _cpu_baseline(_host_views(data, spec), spec, os.cpu_count() or 1)
 
-    # kernels of this library per step: the attention kernel (plus the plan and combine kernels
-    # when units are split, which shows as a workspace beyond the 256-byte minimum), the dense
-    # logits pass and the per-request verification kernel
-    launches_per_step = (3 if ws_a.numel() > 256 else 1) + 2
+    # kernels of this library per step: the attention kernel (plus its plan / combine kernels when
+    # the launch shape uses them), the dense logits pass and the per-request verification kernel
+    launches_per_step = dsbd.forest_attention_launches(f, spec["Hq"], spec["Hkv"], spec["d"], data["q"].dtype,
+                                                       scale, poff) + 2
     ms_per_step = total_ms / args.steps
     line = {"metric": METRIC, "value": job_value(f.N, world, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,

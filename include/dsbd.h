@@ -107,6 +107,11 @@ int dsbd_forest_attention(const dsbd_forest_t *forest, const dsbd_attn_desc_t *d
 
 size_t dsbd_forest_attention_workspace(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc);
 
+/* How many kernels dsbd_forest_attention launches for this shape (1: the attention kernel; 2:
+ * plus a work plan that orders ragged units; 3: plus the merge of split units), 0 for invalid
+ * arguments.  For launch accounting; host-only. */
+int dsbd_forest_attention_launches(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc);
+
 /* Parameters of the verification (Section "Details", Algorithm 1, and Section
  * "Dynamic-Width Speculative Beam Decoding"). */
 typedef struct {

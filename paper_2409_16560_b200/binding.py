@@ -19,7 +19,7 @@ SRC_DRAFT, SRC_RESIDUAL, SRC_FILL, SRC_EXTRA = 0, 1, 2, 3
 MAX_TREE_NODES = 64
 MAX_LIVE = 64
 
-EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_verify_step",
+EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
            "dsbd_status_string"]
 
@@ -75,6 +75,8 @@ def load():
     lib.dsbd_status_string.argtypes = [C.c_int]
     lib.dsbd_forest_attention_workspace.restype = C.c_size_t
     lib.dsbd_forest_attention_workspace.argtypes = [_vp, _vp]
+    lib.dsbd_forest_attention_launches.restype = C.c_int
+    lib.dsbd_forest_attention_launches.argtypes = [_vp, _vp]
     lib.dsbd_verify_workspace.restype = C.c_size_t
     lib.dsbd_verify_workspace.argtypes = [_vp, _vp]
     lib.dsbd_forest_attention.restype = C.c_int
@@ -180,6 +182,12 @@ def forest_attention_workspace(forest, Hq, Hkv, d, dtype, scale, prefix_off_host
     f = forest.struct()
     desc = _attn_desc(Hq, Hkv, d, dtype, scale, prefix_off_host)
     return int(load().dsbd_forest_attention_workspace(C.addressof(f), C.addressof(desc)))
+
+
+def forest_attention_launches(forest, Hq, Hkv, d, dtype, scale, prefix_off_host):
+    f = forest.struct()
+    desc = _attn_desc(Hq, Hkv, d, dtype, scale, prefix_off_host)
+    return int(load().dsbd_forest_attention_launches(C.addressof(f), C.addressof(desc)))
 
 
 def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_prefix, prefix_off,

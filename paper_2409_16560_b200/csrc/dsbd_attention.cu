@@ -226,6 +226,11 @@ extern "C" size_t dsbd_forest_attention_workspace(const dsbd_forest_t *f, const 
     return attention_tc_supported(f, d) ? attention_tc_workspace(f, d) : 256;
 }
 
+extern "C" int dsbd_forest_attention_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+    if (check(f, d) != DSBD_OK) return 0;
+    return attention_tc_supported(f, d) ? attention_tc_launches(f, d) : 1;
+}
+
 extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q,
                                      const void *k_new, const void *v_new, const void *k_prefix,
                                      const void *v_prefix, const int64_t *prefix_off, void *out,

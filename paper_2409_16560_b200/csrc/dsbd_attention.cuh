@@ -12,6 +12,9 @@ bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
 // Workspace bytes of the tensor-core path (work plan and partial results of split units).
 size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
 
+// Kernels one call launches: the attention kernel, plus the plan and the combine kernel when used.
+int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
+
 int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
                         const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
                         void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream);

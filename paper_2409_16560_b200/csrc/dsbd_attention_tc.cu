@@ -232,6 +232,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const int n_items = item_count(a);
             for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
                 const AttnItem item = get_item(a, u);
+                if (item.b < 0) continue;
                 const int b = item.b, g = item.g;
                 const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
                 const int64_t row0 = a.prefix_off[b] * a.Hkv + (int64_t)g * L + item.t0;
@@ -279,8 +280,9 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             bool ok = true;
             const uint64_t qd = desc_k_major(smem_u32(q_s));
             const int n_items = item_count(a);
-            for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x, ++unit) {
+            for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
                 const AttnItem item = get_item(a, u);
+                if (item.b < 0) continue;
                 const int nt = (item.t1 - item.t0 + kBN - 1) / kBN + item.last;
                 ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
                 // S(t) = Q K(t)^T into S buffer t & 1; issued one tile ahead of the P V product so
@@ -315,6 +317,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     tc_commit(&sb.pv_done);
                 }
                 if (ok) tc_commit(&sb.o_full);
+                ++unit;
             }
         }
     } else {
@@ -324,8 +327,9 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
         uint32_t tile = 0, unit = 0;
         bool ok = true;
         const int n_items = item_count(a);
-        for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x, ++unit) {
+        for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
             const AttnItem item = get_item(a, u);
+            if (item.b < 0) continue;
             const int b = item.b, g = item.g;
             const int64_t L = item.t1;                         // tokens beyond t1 belong to other items
             const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
@@ -476,6 +480,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 }
             }
             tc_fence_before();
+            ++unit;
         }
     }
     tc_fence_before();
@@ -502,8 +507,8 @@ __device__ __forceinline__ void unit_parts(int64_t L, int chunk, int *np, int *p
 }
 
 __global__ void __launch_bounds__(1024)
-k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, AttnItem *__restrict__ items,
-            int *__restrict__ n_items, UnitParts *__restrict__ units) {
+k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, int grid,
+            AttnItem *__restrict__ items, int *__restrict__ n_items, UnitParts *__restrict__ units) {
     __shared__ int bucket[1024];
     __shared__ int scan[1024];
     __shared__ int carry;
@@ -555,7 +560,13 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, A
     const int start = scan[tid] - bucket[1023 - tid];
     __syncthreads();
     bucket[1023 - tid] = start;                 // bucket[k] becomes the cursor of tile count k
-    if (tid == 0) *n_items = carry;
+    // The list is read in rounds of `grid` items, CTA k taking entry k of every round.  Odd rounds
+    // are stored back to front, so that the CTA with the longest item of one round gets the
+    // shortest of the next; the last round is padded with empty entries (b = -1).
+    const int total_items = carry;
+    const int padded = (total_items + grid - 1) / grid * grid;
+    for (int i = total_items - total_items % grid + tid; i < padded; i += 1024) items[i].b = -1;
+    if (tid == 0) *n_items = padded;
     __syncthreads();
     for (int u = tid; u < n_units; u += 1024) {
         const int b = u / Hkv, g = u - b * Hkv;
@@ -566,7 +577,9 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, A
             const int64_t t0 = (int64_t)p * plen;
             const int64_t t1 = t0 + plen < L ? t0 + plen : L;
             const int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
-            const int pos = atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
+            int pos = atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
+            const int round = pos / grid;
+            if (round & 1) pos = round * grid + (grid - 1 - (pos - round * grid));
             AttnItem it;
             it.b = b; it.g = g; it.t0 = (int)t0; it.t1 = (int)t1; it.last = (p == np - 1);
             it.nparts = np; it.slot = units[u].first_slot + p; it.pad = 0;
@@ -640,7 +653,8 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, ui
 
 // Launch shape shared by the workspace query and the launch.
 struct TcPlan {
-    int grid, chunk;          // chunk == 0: one item per unit, no plan kernel
+    int grid, chunk;          // chunk == 0: one item per unit in unit order, no plan kernel
+    bool split;               // units are cut into parts (partials + combine kernel)
     int64_t items_max;
     size_t off_items, off_units, off_partial, total;
 };
@@ -655,25 +669,32 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     const int64_t n_units = (int64_t)f->B * d->Hkv;
     // Splitting a unit costs a pipeline drain, a Q reload and a partial result per part, so it
     // pays only when there are fewer units than CTAs: then the prefix is cut so that about two
-    // items per CTA exist, in parts of at least 512 tokens.
+    // items per CTA exist, in parts of at least 512 tokens.  Ragged batches with enough units
+    // are only re-ordered (longest first, rounds alternating in direction).
     int64_t c = (int64_t)d->total_prefix * d->Hkv / (2ll * p.grid);
     if (c < 512) c = 512;
     c = (c + kBN - 1) / kBN * kBN;
-    if (n_units >= p.grid || c >= d->max_prefix) {
+    p.split = n_units < p.grid && c < d->max_prefix;
+    const bool ragged = (int64_t)d->max_prefix * f->B * 100 > (int64_t)d->total_prefix * 115;
+    if (!p.split && !(ragged && n_units > p.grid)) {
         p.chunk = 0;
         p.items_max = n_units;
         if (p.grid > n_units) p.grid = (int)n_units;
         p.total = 256;
         return p;
     }
+    if (!p.split) c = (int64_t)1 << 30;                  // one part per unit
     p.chunk = (int)c;
-    p.items_max = (int64_t)d->Hkv * (d->total_prefix / c + f->B);
+    p.items_max = (p.split ? (int64_t)d->Hkv * (d->total_prefix / c + f->B) : n_units) + p.grid;
+    if (p.grid > p.items_max - p.grid) p.grid = (int)(p.items_max - p.grid);
+    if (p.grid < 1) p.grid = 1;
     size_t off = 256;
     p.off_items = off;   off = align_up(off + sizeof(AttnItem) * (size_t)p.items_max, 256);
     p.off_units = off;   off = align_up(off + sizeof(UnitParts) * (size_t)n_units, 256);
-    p.off_partial = off; off = align_up(off + sizeof(float) * 130 * (size_t)p.items_max * (size_t)(f->max_tree_nodes * group), 256);
+    p.off_partial = off;
+    if (p.split)
+        off = align_up(off + sizeof(float) * 130 * (size_t)p.items_max * (size_t)(f->max_tree_nodes * group), 256);
     p.total = off;
-    if (p.grid > p.items_max) p.grid = (int)p.items_max;
     return p;
 }
 
@@ -691,6 +712,11 @@ bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
 }
 
 size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) { return make_plan(f, d).total; }
+
+int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+    const TcPlan p = make_plan(f, d);
+    return 1 + (p.chunk > 0 ? 1 : 0) + (p.split ? 1 : 0);
+}
 
 int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
                         const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
@@ -719,7 +745,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
         AttnItem *items = reinterpret_cast<AttnItem *>(ws + plan.off_items);
         units = reinterpret_cast<UnitParts *>(ws + plan.off_units);
         int *n_items = reinterpret_cast<int *>(ws);
-        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, plan.chunk, items, n_items, units);
+        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, plan.chunk, plan.grid, items, n_items, units);
         a.items = items;
         a.n_items = n_items;
         a.partial = reinterpret_cast<float *>(ws + plan.off_partial);
@@ -738,7 +764,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     if (small_q) DSBD_LAUNCH_TC(64, 3);
     else DSBD_LAUNCH_TC(128, 3);
 #undef DSBD_LAUNCH_TC
-    if (plan.chunk > 0) k_attn_combine<<<a.n_units, 128, 0, stream>>>(a, units);
+    if (plan.split) k_attn_combine<<<a.n_units, 128, 0, stream>>>(a, units);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 
