@@ -19,7 +19,7 @@ _lib = None
 
 NODE_UNREACHED, NODE_ACCEPTED, NODE_REJECTED, NODE_CUT, NODE_PRUNED = 0, 1, 2, 3, 4
 SRC_DRAFT, SRC_RESIDUAL, SRC_FILL, SRC_EXTRA = 0, 1, 2, 3
-TR_ACCEPT, TR_RESIDUAL, TR_FILL, TR_EXTRA, TR_WIDTH = 0, 1, 2, 3, 4
+TR_ACCEPT, TR_RESIDUAL, TR_FILL, TR_EXTRA, TR_WIDTH, TR_WARP = 0, 1, 2, 3, 4, 5
 
 _i32p = C.POINTER(C.c_int32)
 _i64p = C.POINTER(C.c_int64)
@@ -38,7 +38,8 @@ class _Params(C.Structure):
     _fields_ = [("V", C.c_int32), ("temperature", C.c_double), ("thresh", C.c_double),
                 ("W_min", C.c_int32), ("W_max", C.c_int32), ("W_nom", C.c_int32),
                 ("W_min_r", _i32p), ("W_max_r", _i32p), ("W_nom_r", _i32p),
-                ("seed", C.c_uint64), ("step", C.c_uint64), ("req_id", _i32p)]
+                ("seed", C.c_uint64), ("step", C.c_uint64), ("req_id", _i32p),
+                ("top_k", C.c_int32), ("top_p", C.c_double)]
 
 
 class _VerifyOut(C.Structure):
@@ -107,6 +108,8 @@ def _params(params, R, keep):
             setattr(p, name, _p(a, _i32p))
     p.seed = int(params.get("seed", 0))
     p.step = int(params.get("step", 0))
+    p.top_k = int(params.get("top_k", 0))
+    p.top_p = float(params.get("top_p", 1.0))
     return p
 
 
@@ -181,6 +184,15 @@ def default_out_off(forest, params):
     return np.concatenate([[0], np.cumsum(cap)]).astype(np.int32)
 
 
+def warp(w, top_k=0, top_p=1.0):
+    """T o w: the warped copy of the joint distribution w (any shape; cells in C order)."""
+    w = np.array(w, dtype=np.float64)
+    flat = np.ascontiguousarray(w.ravel())
+    lib().dsbd_oracle_warp(_p(flat, _f64p), C.c_int64(flat.size), C.c_int32(int(top_k)), C.c_double(float(top_p)),
+                           _f64p(), _f64p())
+    return flat.reshape(w.shape)
+
+
 def verify_step(forest, params, logits_p, logits_q, root_logp, root_logq, out_off=None,
                 inject_u=None, trace=True, dist=False, threads=1, row_stride=None):
     """One verification step for every request; returns a dict of numpy arrays."""
@@ -220,7 +232,7 @@ def verify_step(forest, params, logits_p, logits_q, root_logp, root_logq, out_of
     dlen = np.zeros(1, np.int64)
     if trace:
         nodes = N
-        cap = 4 * nodes + 8 * R * (gamma + 2) + int(out_off[-1]) + 64
+        cap = 4 * nodes + 12 * R * (gamma + 2) + int(out_off[-1]) + 64
         o.trace_cap = cap
         o.trace_len = _p(tlen, _i64p)
         for name in ("trace_req", "trace_layer", "trace_kind", "trace_index", "trace_near"):

@@ -303,6 +303,51 @@ static void beam_distribution(const float *z, int64_t stride, int32_t V, double 
     }
 }
 
+/* ------------------------------------------------------------------ warping ---------- */
+typedef struct { double v; int64_t i; } cell_t;
+static int cmp_cell_desc(const void *x, const void *y)
+{
+    const cell_t *a = (const cell_t *)x, *b = (const cell_t *)y;
+    if (a->v != b->v) return a->v > b->v ? -1 : 1;
+    return a->i < b->i ? -1 : (a->i > b->i ? 1 : 0);
+}
+
+/* T o w: sort the cells by probability, keep the first top_k, renormalise, then keep the
+ * shortest prefix whose mass reaches top_p, renormalise.  (The order top-k, then top-p on the
+ * renormalised vector is the usual one for chained warpers.) */
+void dsbd_oracle_warp(double *w, int64_t n, int32_t top_k, double top_p, double *gap_k, double *gap_p)
+{
+    if (gap_k) *gap_k = 1.0;
+    if (gap_p) *gap_p = 1.0;
+    const int use_k = top_k > 0 && top_k < n, use_p = top_p > 0.0 && top_p < 1.0;
+    if (!use_k && !use_p) return;
+    cell_t *c = (cell_t *)malloc(sizeof(cell_t) * (size_t)n);
+    for (int64_t i = 0; i < n; ++i) { c[i].v = w[i]; c[i].i = i; }
+    qsort(c, (size_t)n, sizeof(cell_t), cmp_cell_desc);
+    int64_t keep = n;
+    if (use_k) {
+        keep = top_k;
+        if (gap_k && c[keep - 1].v > 0.0) *gap_k = (c[keep - 1].v - c[keep].v) / c[keep - 1].v;
+    }
+    double z = 0.0;
+    for (int64_t j = 0; j < keep; ++j) z += c[j].v;
+    if (use_p && z > 0.0) {
+        double cum = 0.0;
+        int64_t j = 0;
+        for (; j < keep; ++j) {
+            cum += c[j].v / z;
+            if (gap_p) { double g = fabs(cum - top_p); if (g < *gap_p) *gap_p = g; }
+            if (cum >= top_p) { ++j; break; }
+        }
+        keep = j;
+        z = 0.0;
+        for (int64_t q = 0; q < keep; ++q) z += c[q].v;
+    }
+    for (int64_t i = 0; i < n; ++i) w[i] = 0.0;
+    if (z > 0.0) for (int64_t j = 0; j < keep; ++j) w[c[j].i] = c[j].v / z;
+    free(c);
+}
+
 static int cmp_rank(const void *x, const void *y)
 {
     const int64_t *a = (const int64_t *)x, *b = (const int64_t *)y;
@@ -409,6 +454,14 @@ static void verify_request(req_ctx *c, int32_t r, const int32_t *depth, const in
         double *p_cur = (double *)malloc(sizeof(double) * (size_t)cells);
         beam_distribution(c->zp, c->stride, V, tau, A, nA, o->node_logp, o->lse_p, p_beam);
         beam_distribution(c->zq, c->stride, V, tau, A, nA, o->node_logq, o->lse_q, q_beam);
+        if (prm->top_k > 0 || (prm->top_p > 0.0 && prm->top_p < 1.0)) {
+            /* p_beam = T o (p / P), q_beam = T o (q / Q)  (Section "Details") */
+            double gk, gp;
+            dsbd_oracle_warp(p_beam, cells, prm->top_k, prm->top_p, &gk, &gp);
+            trace_push(c, l, DSBD_O_TR_WARP, 0, 0.0, gk, gp, gk < NEAR_TIE || gp < NEAR_TIE);
+            dsbd_oracle_warp(q_beam, cells, prm->top_k, prm->top_p, &gk, &gp);
+            trace_push(c, l, DSBD_O_TR_WARP, 1, 0.0, gk, gp, gk < NEAR_TIE || gp < NEAR_TIE);
+        }
 
         /* width of this layer */
         double *alpha = (double *)malloc(sizeof(double) * (size_t)(m + 1));
@@ -503,6 +556,11 @@ static void verify_request(req_ctx *c, int32_t r, const int32_t *depth, const in
         const int64_t cells = (int64_t)nA * V;
         double *p_beam = (double *)malloc(sizeof(double) * (size_t)cells);
         beam_distribution(c->zp, c->stride, V, tau, A, nA, o->node_logp, o->lse_p, p_beam);
+        if (prm->top_k > 0 || (prm->top_p > 0.0 && prm->top_p < 1.0)) {
+            double gk, gp;
+            dsbd_oracle_warp(p_beam, cells, prm->top_k, prm->top_p, &gk, &gp);
+            trace_push(c, gamma + 1, DSBD_O_TR_WARP, 0, 0.0, gk, gp, gk < NEAR_TIE || gp < NEAR_TIE);
+        }
         o->layer_width[(int64_t)r * (gamma + 1) + gamma] = W_nom;
         for (int32_t k = 0; k < W_nom && !err; ++k) {
             const double u = next_uniform(c, inject, inject_stride, &inject_pos, rid,
@@ -615,6 +673,8 @@ int dsbd_oracle_select_width(const dsbd_oracle_forest *f, const dsbd_oracle_para
         double *q_beam = (double *)malloc(sizeof(double) * (size_t)(cells + 1));
         beam_distribution(logits_p, row_stride, V, tau, A, nA, node_logp, lse_p, p_beam);
         beam_distribution(logits_q, row_stride, V, tau, A, nA, node_logq, lse_q, q_beam);
+        dsbd_oracle_warp(p_beam, cells, prm->top_k, prm->top_p, NULL, NULL);
+        dsbd_oracle_warp(q_beam, cells, prm->top_k, prm->top_p, NULL, NULL);
         double *al = (double *)malloc(sizeof(double) * (size_t)(mr + 1));
         double *P = (double *)malloc(sizeof(double) * (size_t)(mr + 1) * (size_t)(mr + 1));
         double *G = (double *)malloc(sizeof(double) * (size_t)(mr + 2));

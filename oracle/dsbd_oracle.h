@@ -49,6 +49,9 @@ typedef struct {
     uint64_t seed, step;             /* Philox key and decode-step counter                   */
     const int32_t *req_id;           /* optional [R]: request number used in the Philox      */
                                      /* counter (NULL = 0..R-1); lets a test verify a subset */
+    int32_t top_k;                   /* warping T of the joint distributions: keep the top_k  */
+    double top_p;                    /* cells (0 = off), then the smallest set of the largest */
+                                     /* cells whose mass reaches top_p (<= 0 or >= 1 = off)   */
 } dsbd_oracle_params;
 
 /* node_status values */
@@ -68,7 +71,10 @@ enum {
 /* trace kinds */
 enum {
     DSBD_O_TR_ACCEPT = 0, DSBD_O_TR_RESIDUAL = 1, DSBD_O_TR_FILL = 2, DSBD_O_TR_EXTRA = 3,
-    DSBD_O_TR_WIDTH = 4
+    DSBD_O_TR_WIDTH = 4,
+    DSBD_O_TR_WARP = 5      /* one per warped distribution: a = relative gap between the last
+                               kept and the first dropped cell of the top-k cut, b = distance
+                               of the kept mass from top_p at the top-p cut; index 0 = p, 1 = q */
 };
 
 typedef struct {
@@ -138,6 +144,12 @@ void dsbd_oracle_alpha_chain(const double *p_beam, const double *q_beam, int64_t
  * K = 0..m+1 (G[m+1] = 0); returns W~ = max{K in 0..m : G(K) >= thresh}. */
 int32_t dsbd_oracle_width_dp(const double *alpha, int32_t m, double thresh, double *P,
                              double *G);
+
+/* The warping T applied to a joint distribution w over n cells, in place (Section "Decodings of
+ * LLMs": top-k keeps the k most probable entries, top-p the smallest set of most probable
+ * entries whose mass reaches p; both renormalise).  Ties are broken towards the lower cell
+ * index.  gap_k / gap_p (optional) receive the quantities of the DSBD_O_TR_WARP record. */
+void dsbd_oracle_warp(double *w, int64_t n, int32_t top_k, double top_p, double *gap_k, double *gap_p);
 
 /* One verification step (Algorithm 1 with the dynamic width) for every request.
  * inject_u: NULL, or [R*inject_stride] uniforms consumed in order by the random decisions of

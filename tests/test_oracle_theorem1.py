@@ -59,7 +59,7 @@ def _layer_law(model, layer_lists, probs, fixed_prefix, target, params, gamma):
         nxt = []
         for r, (i, pre, prob) in enumerate(states):
             lo, hi = starts[r], starts[r + 1]
-            recs = [t for t in range(lo, hi) if res["trace_kind"][t] != oracle.TR_WIDTH]
+            recs = [t for t in range(lo, hi) if res["trace_kind"][t] not in (oracle.TR_WIDTH, oracle.TR_WARP)]
             k = len(pre)
             if (k < len(recs) and res["trace_kind"][recs[k]] == oracle.TR_ACCEPT
                     and res["trace_layer"][recs[k]] == target):
@@ -111,6 +111,22 @@ def _layer_law(model, layer_lists, probs, fixed_prefix, target, params, gamma):
     return law, width
 
 
+def _warp_ref(w, top_k, top_p):
+    """The warping by its definition, written independently of the oracle: keep the top_k most
+    probable cells, renormalise; keep the shortest most-probable prefix whose mass reaches
+    top_p, renormalise.  Ties towards the lower cell index."""
+    w = np.asarray(w, dtype=np.float64).ravel()
+    order = np.lexsort((np.arange(w.size), -w))
+    keep = order[:top_k] if top_k else order
+    probs = w[keep] / w[keep].sum()
+    if top_p < 1.0:
+        n = int(np.searchsorted(np.cumsum(probs), top_p - 1e-15)) + 1
+        keep = keep[:n]
+    out = np.zeros_like(w)
+    out[keep] = w[keep] / w[keep].sum()
+    return out
+
+
 def _product_law(pb, W):
     out = np.array(1.0)
     for _ in range(W):
@@ -131,6 +147,26 @@ def test_first_layer_law_equals_beam_sampling(params):
     layer_lists = [[[(c // V, c % V) for c in t]] for t in tuples]
     probs = [float(np.prod(qb[list(t)])) for t in tuples]
     assert abs(sum(probs) - 1) < 1e-12
+    law, W = _layer_law(model, layer_lists, probs, [], 1, params, gamma=1)
+    assert abs(law.sum() - 1) < 1e-10
+    assert np.abs(law - _product_law(pb, W)).max() < 1e-12
+
+
+@pytest.mark.parametrize("top_k,top_p", [(5, 1.0), (0, 0.7), (6, 0.8), (1, 1.0)])
+def test_first_layer_law_with_warped_joints(top_k, top_p):
+    """With the warping T on both joints (drafts drawn from T o q_beam) the outputs follow the
+    product of T o p_beam."""
+    model = ToyModel(seed=5)
+    qb = _warp_ref(model.beam_dist("q", [(0,), (1,)]), top_k, top_p)
+    pb = _warp_ref(model.beam_dist("p", [(0,), (1,)]), top_k, top_p)
+    assert (pb > 0).sum() <= (top_k or 99) and abs(pb.sum() - 1) < 1e-12
+    assert np.abs(oracle.warp(model.beam_dist("p", [(0,), (1,)]), top_k, top_p).ravel() - pb).max() < 1e-15
+    support = np.nonzero(qb)[0]
+    tuples = list(itertools.product(support, repeat=3))
+    layer_lists = [[[(int(c) // V, int(c) % V) for c in t]] for t in tuples]
+    probs = [float(np.prod(qb[list(t)])) for t in tuples]
+    assert abs(sum(probs) - 1) < 1e-12
+    params = dict(W_min=2, W_max=2, W_nom=2, thresh=0.7, top_k=top_k, top_p=top_p)
     law, W = _layer_law(model, layer_lists, probs, [], 1, params, gamma=1)
     assert abs(law.sum() - 1) < 1e-10
     assert np.abs(law - _product_law(pb, W)).max() < 1e-12
