@@ -225,6 +225,8 @@ def main():
     ap.add_argument("--workload", default="C5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--top-k", type=int, default=0, help="warp the joint distributions: top-k (0 = off)")
+    ap.add_argument("--top-p", type=float, default=1.0, help="and top-p (needs --top-k); the paper uses 10 / 0.8")
     ap.add_argument("--requests", type=int, default=0,
                     help="override the number of requests of the workload (profiling on a smaller case)")
     args = ap.parse_args()
@@ -253,6 +255,7 @@ def main():
     spec = rank_spec(spec, rank)                         # every rank verifies its own requests
     data = inputs.generate(spec, dev)
     forest, prm, poff = data["forest"], dict(data["params"]), data["prefix_off"]
+    prm.update(top_k=args.top_k, top_p=args.top_p)
     f = dsbd.Forest(forest, dev)
     prm_dev = dict(prm, W_min_r=torch.as_tensor(prm["W_min_r"]).to(dev))
     out_off = dsbd.default_out_off(forest, prm)
@@ -413,7 +416,7 @@ def main():
             "config": {"workload": args.workload, "requests": f.R, "beams": f.B, "nodes": f.N,
                        "heads": "%dq/%dkv x %d" % (spec["Hq"], spec["Hkv"], spec["d"]), "vocab": spec["V"],
                        "prefix": list(spec["prefix"]), "temperature": spec["temperature"],
-                       "thresh": prm["thresh"], "l2": "inputs (%.1f GB) far exceed the 126 MB L2; no flush" % (
+                       "thresh": prm["thresh"], "top_k": args.top_k, "top_p": args.top_p, "l2": "inputs (%.1f GB) far exceed the 126 MB L2; no flush" % (
                            (a_bytes + v_bytes) * 1e-9),
                        "parallelism": "replicas x%d" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,

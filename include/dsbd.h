@@ -128,6 +128,14 @@ typedef struct {
     const int32_t *W_nom_r;
     uint64_t seed;                 /* Philox4x32-10 key                                      */
     uint64_t step;                 /* decode-step counter, mixed into the Philox counter     */
+    /* Warping T of the joint distributions p_beam, q_beam (Section "Decodings of LLMs" and the
+     * definitions of p_beam, q_beam in Section "Details"; the paper's experiments use top-k 10,
+     * top-p 0.8): keep the top_k most probable cells of the joint over (live parents x V) and
+     * renormalise, then keep the shortest most-probable prefix whose mass reaches top_p and
+     * renormalise; ties go to the lower (parent, token).  top_k = 0: no warping (then top_p must
+     * be 0 or >= 1).  This build supports 1 <= top_k <= 64; top_p outside (0,1) is "off". */
+    int32_t top_k;
+    float top_p;
 } dsbd_verify_params_t;
 
 /* node_status */

@@ -43,7 +43,7 @@ class VerifyParamsT(C.Structure):
     _fields_ = [("V", C.c_int32), ("temperature", C.c_float), ("thresh", C.c_float),
                 ("W_min", C.c_int32), ("W_max", C.c_int32), ("W_nom", C.c_int32),
                 ("W_min_r", _vp), ("W_max_r", _vp), ("W_nom_r", _vp),
-                ("seed", C.c_uint64), ("step", C.c_uint64)]
+                ("seed", C.c_uint64), ("step", C.c_uint64), ("top_k", C.c_int32), ("top_p", C.c_float)]
 
 
 _OUT_FIELDS = ["l_last", "out_width", "out_off", "out_parent", "out_node", "out_root_beam",
@@ -229,6 +229,8 @@ def _params(params, keep):
             setattr(p, name, _ptr(t))
     p.seed = int(params.get("seed", 0))
     p.step = int(params.get("step", 0))
+    p.top_k = int(params.get("top_k", 0))
+    p.top_p = float(params.get("top_p", 1.0))
     return p
 
 

@@ -169,6 +169,8 @@ struct VerifyArgs {
     int W_min, W_max, W_nom;
     const int32_t *W_min_r, *W_max_r, *W_nom_r;
     uint64_t seed, step;
+    int top_k;                // 0: unwarped joints
+    double top_p;             // outside (0,1): off
     // inputs
     const float *zp, *zq;
     int64_t stride;
@@ -545,6 +547,252 @@ __device__ int draw_cell(const VerifyArgs &a, const Shared &sh, double u, bool u
                         target - before, lane);
 }
 
+// ---------------------------------------------------------------------------------------
+// Warped joints (top-k / top-p).  The support of T o p_beam has at most top_k <= 64 cells, so
+// once it is known everything else of the layer is scalar work.  Finding it needs no pass over
+// the rows: the maximum of every 1024-token tile is known from the dense pass, the k largest
+// tile maxima are k distinct cells, hence the k-th largest cell of the joint is at least the
+// k-th largest tile bound and every cell of the top k lies in a tile whose bound reaches it.
+// Only those (about k) tiles are read.
+// ---------------------------------------------------------------------------------------
+constexpr int kMaxTopK = 64;
+constexpr int kMaxCand = 1024;
+struct WarpScratch {
+    double prob[2][kMaxTopK];     // warped probabilities, most probable first (0: p, 1: q)
+    double qat[kMaxTopK];         // q~ at the cells of the p support
+    int cell[2][kMaxTopK];        // live parent index * V + token
+    int order[kMaxTopK];          // the p support in canonical (cell-ascending) order
+    int n[2];
+    // scratch of build_support
+    float off[kMaxLive];          // log(beam weight) - lse of each live row
+    int sel[256];                 // tiles whose bound reaches the threshold
+    int n_sel, n_cand, err;
+    float theta;
+};
+
+// Support of the warped joint of one model; called by ALL threads of the CTA.
+// Returns 0 or a DSBD_DEV_* code (the same on every thread).
+__device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, double *cand_key, int *cand_cell,
+                             WarpScratch &ws) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int T = a.T, nt = sh.nA * T, k = a.top_k;
+    const TileStat *stats = a.stats + (int64_t)model * a.N * T;
+    const double *lw = model ? sh.lwq : sh.lwp;
+    const double *lse = a.lse + (int64_t)model * a.N;
+    const float *z = model ? a.zq : a.zp;
+    const float inv_tau_f = (float)a.inv_tau;
+    for (int i = threadIdx.x; i < sh.nA; i += blockDim.x) ws.off[i] = (float)(lw[i] - lse[sh.A[i]]);
+    if (threadIdx.x == 0) { ws.n_sel = 0; ws.n_cand = 0; ws.err = 0; ws.n[model] = 0; }
+    __syncthreads();
+    // float upper bound of log(joint probability) over tile i
+    auto bound = [&](int i) -> float {
+        const int ia = i / T;
+        return fmaf(stats[(int64_t)sh.A[ia] * T + (i - ia * T)].mx, inv_tau_f, ws.off[ia]);
+    };
+    if (warp == 0) {
+        // k-th largest distinct tile bound; with fewer than k distinct bounds every tile counts
+        float thr = INFINITY, top_bound = -INFINITY;
+        bool enough = true;
+        for (int kk = 0; kk < k; ++kk) {
+            float best = -INFINITY;
+            for (int i = lane; i < nt; i += 32) {
+                const float v = bound(i);
+                if (v < thr && v > best) best = v;
+            }
+            best = warp_max(best);
+            if (!(best > -INFINITY)) { enough = false; break; }
+            if (kk == 0) top_bound = best;
+            thr = best;
+        }
+        // the float keys carry an error of about 1e-5; the slack keeps the selection conservative
+        const float theta = enough ? thr - 5e-5f - 4e-6f * fabsf(thr) : -INFINITY;
+        int n_sel = 0;
+        if (top_bound > -INFINITY)
+            for (int base = 0; base < nt; base += 32) {
+                const int i = base + lane;
+                const bool hit = i < nt && bound(i) >= theta && bound(i) > -INFINITY;
+                const unsigned mask = __ballot_sync(kFull, hit);
+                if (hit) {
+                    const int pos = n_sel + __popc(mask & ((1u << lane) - 1));
+                    if (pos < 256) ws.sel[pos] = i;
+                }
+                n_sel += __popc(mask);
+            }
+        if (lane == 0) {
+            ws.theta = theta;
+            ws.n_sel = n_sel;
+            if (n_sel > 256) ws.err = DSBD_DEV_CAPACITY;       // hundreds of tiles tie at the cut
+        }
+    }
+    __syncthreads();
+    if (ws.err) return ws.err;
+    float theta = ws.theta;
+    const int n_sel = ws.n_sel;
+    // One sweep over the selected tiles by all warps: counts the cells whose key reaches th and,
+    // when asked, appends them to the candidate list (order is irrelevant: the final choice is
+    // by (key, cell)).
+    auto sweep = [&](float th, bool collect) {
+        if (threadIdx.x == 0) ws.n_cand = 0;
+        __syncthreads();
+        for (int sidx = warp; sidx < n_sel; sidx += kWarps) {
+            const int ti = ws.sel[sidx], ia = ti / T, t = ti - ia * T, row = sh.A[ia];
+            const float *rowp = z + (int64_t)row * a.stride;
+            const bool al = (reinterpret_cast<uintptr_t>(rowp) & 15) == 0;
+            float4 v[8];
+            load_tile(rowp, t * kTile, a.V, al, lane, v);
+            const float off_f = ws.off[ia];
+            const double off_d = lw[ia] - lse[row];
+            unsigned hits = 0;                               // bit (it*4+c) of this lane's 32 cells
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const float zz[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float kf = fmaf(zz[c], inv_tau_f, off_f);
+                    if (kf >= th && kf > -INFINITY) hits |= 1u << (it * 4 + c);
+                }
+            }
+            const int mine = __popc(hits);
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int tmp = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += tmp;
+            }
+            const int total = __shfl_sync(kFull, incl, 31);
+            int base_pos = 0;
+            if (lane == 0 && total) base_pos = atomicAdd(&ws.n_cand, total);
+            base_pos = __shfl_sync(kFull, base_pos, 0);
+            if (collect && mine) {
+                int pos = base_pos + incl - mine;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const float zz[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if (hits & (1u << (it * 4 + c))) {
+                            if (pos < kMaxCand) {
+                                cand_key[pos] = off_d + (double)zz[c] * a.inv_tau;
+                                cand_cell[pos] = ia * a.V + t * kTile + it * 128 + lane * 4 + c;
+                            }
+                            ++pos;
+                        }
+                }
+            }
+        }
+        __syncthreads();
+        return ws.n_cand;
+    };
+    int n_cand = sweep(theta, true);
+    if (n_cand > kMaxCand) {
+        // too many cells reach the conservative threshold (few tiles, large k, or near ties):
+        // bisect for a threshold with between k and kMaxCand cells above it
+        float lo_t = theta, hi_t = -INFINITY;
+        for (int sidx = 0; sidx < n_sel; ++sidx) hi_t = fmaxf(hi_t, bound(ws.sel[sidx]));
+        if (!(lo_t > -INFINITY)) lo_t = hi_t - 400.f;
+        bool found = false;
+        for (int itn = 0; itn < 60 && hi_t > lo_t; ++itn) {
+            const float mid = 0.5f * (lo_t + hi_t);
+            const int c = sweep(mid, false);
+            if (c > kMaxCand) lo_t = mid;
+            else if (c < k) hi_t = mid;
+            else { theta = mid; found = true; break; }
+        }
+        if (!found) return DSBD_DEV_CAPACITY;              // a huge tie at the cut
+        n_cand = sweep(theta, true);
+    }
+    // exact top k of the candidates (warp 0): k rounds of arg-max (key descending, cell ascending)
+    if (warp == 0) {
+        int n_sup = 0;
+        for (int kk = 0; kk < k; ++kk) {
+            double bk = -INFINITY;
+            int bc = 0x7fffffff, bi = -1;
+            for (int j = lane; j < n_cand; j += 32) {
+                const double key = cand_key[j];
+                const int cell = cand_cell[j];
+                if (key > bk || (key == bk && key > -INFINITY && cell < bc)) { bk = key; bc = cell; bi = j; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const double ok = __shfl_xor_sync(kFull, bk, o);
+                const int oc = __shfl_xor_sync(kFull, bc, o), oi = __shfl_xor_sync(kFull, bi, o);
+                if (ok > bk || (ok == bk && ok > -INFINITY && oc < bc)) { bk = ok; bc = oc; bi = oi; }
+            }
+            if (bi < 0 || !(bk > -INFINITY)) break;
+            if (lane == 0) {
+                ws.prob[model][n_sup] = exp(bk);
+                ws.cell[model][n_sup] = bc;
+                cand_key[bi] = -INFINITY;
+            }
+            ++n_sup;
+            __syncwarp();
+        }
+        // renormalise over the top k, then the top-p cut and its renormalisation (sorted order)
+        if (lane == 0) {
+            double zsum = 0.0;
+            for (int j = 0; j < n_sup; ++j) zsum += ws.prob[model][j];
+            int keep = n_sup;
+            if (a.top_p > 0.0 && a.top_p < 1.0 && zsum > 0.0) {
+                double cum = 0.0;
+                int j = 0;
+                for (; j < n_sup; ++j) {
+                    cum += ws.prob[model][j] / zsum;
+                    if (cum >= a.top_p) { ++j; break; }
+                }
+                keep = j;
+                zsum = 0.0;
+                for (int q = 0; q < keep; ++q) zsum += ws.prob[model][q];
+            }
+            for (int j = 0; j < keep; ++j) ws.prob[model][j] = zsum > 0.0 ? ws.prob[model][j] / zsum : 0.0;
+            ws.n[model] = keep;
+        }
+    }
+    __syncthreads();
+    return 0;
+}
+
+__device__ __forceinline__ double support_lookup(const WarpScratch &ws, int model, int cell) {
+    for (int j = 0; j < ws.n[model]; ++j)
+        if (ws.cell[model][j] == cell) return ws.prob[model][j];
+    return 0.0;
+}
+
+// Inverse-CDF draw over the p support in canonical order; mass max(p~ - s q~, 0) (s = 0: p~).
+// By one thread.  Returns the index into the p support or -1.
+__device__ int draw_support(const WarpScratch &ws, double u, double s) {
+    const int n = ws.n[0];
+    double zsum = 0.0;
+    for (int o = 0; o < n; ++o) {
+        const int i = ws.order[o];
+        zsum += fmax(ws.prob[0][i] - s * ws.qat[i], 0.0);
+    }
+    if (!(zsum > 0.0)) return -1;
+    const double target = u * zsum;
+    double cum = 0.0;
+    int last = -1;
+    for (int o = 0; o < n; ++o) {
+        const int i = ws.order[o];
+        const double w = fmax(ws.prob[0][i] - s * ws.qat[i], 0.0);
+        cum += w;
+        if (w > 0.0) { last = i; if (cum >= target) return i; }
+    }
+    return last;
+}
+
+// After build_support(p) [and q]: q~ at the p cells and the canonical order of the p support.
+__device__ void finish_supports(WarpScratch &ws, bool have_q, int lane) {
+    for (int i = lane; i < ws.n[0]; i += 32) ws.qat[i] = have_q ? support_lookup(ws, 1, ws.cell[0][i]) : 0.0;
+    if (lane == 0) {
+        const int n = ws.n[0];
+        for (int i = 0; i < n; ++i) {
+            int j = i - 1;
+            while (j >= 0 && ws.cell[0][ws.order[j]] > ws.cell[0][i]) { ws.order[j + 1] = ws.order[j]; --j; }
+            ws.order[j + 1] = i;
+        }
+    }
+    __syncwarp();
+}
+
 #ifdef DSBD_PHASE_TIMING
 #define TS(slot) do { if (threadIdx.x == 0 && writer) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); a.dbg[(int64_t)r * 256 + ts_n] = ((unsigned long long)(slot) << 48) | (t_ & 0xFFFFFFFFFFFFull); if (ts_n < 255) ++ts_n; } } while (0)
 #else
@@ -811,7 +1059,39 @@ k_verify(VerifyArgs a) {
         const int m = sh.m;
         TS(3);
 
-        if (m >= 1 && !sh.err) {
+        const bool warped = a.top_k > 0;
+        WarpScratch &wsup = *reinterpret_cast<WarpScratch *>(hq);       // the histogram arrays are idle when warped
+        if (warped) {
+            // ---- supports of T o p_beam and T o q_beam, then the whole chain on <= 64 cells ----
+            if (!sh.err) {
+                double *cand_key = reinterpret_cast<double *>(hp);
+                int *cand_cell = reinterpret_cast<int *>(hp + 2 * kMaxCand);
+                int e = build_support(a, sh, 0, cand_key, cand_cell, wsup);
+                if (!e) e = build_support(a, sh, 1, cand_key, cand_cell, wsup);
+                if (e) { if (threadIdx.x == 0) sh.err = e; }
+                else if (warp == 0) {
+                    finish_supports(wsup, true, lane);
+                    // rho of every live draft from the warped joints
+                    if (!a.select_mode)
+                        for (int i = lane; i < m; i += 32) {
+                            const int cell = sh.S_parent_idx[i] * a.V + a.token[sh.S[i]];
+                            const double pw = support_lookup(wsup, 0, cell), qw = support_lookup(wsup, 1, cell);
+                            sh.rho[i] = qw > 0.0 ? pw / qw : (pw > 0.0 ? INFINITY : 0.0);
+                        }
+                    // c_{j+1} = F(s_j) over the p support, lanes over cells
+                    for (int j = 1; j <= m; ++j) {
+                        const double s_j = sh.s_arr[j - 1] + sh.c_arr[j];
+                        double acc = 0.0;
+                        for (int i = lane; i < wsup.n[0]; i += 32) acc += fmax(wsup.prob[0][i] - s_j * wsup.qat[i], 0.0);
+                        acc = warp_sum(acc);
+                        if (lane == 0) { sh.s_arr[j] = s_j; sh.c_arr[j + 1] = acc; sh.chain_len = j; }
+                        __syncwarp();
+                        if (!(acc > 0.0)) break;
+                    }
+                }
+            }
+            __syncthreads();
+        } else if (m >= 1 && !sh.err) {
             // ---- one pass: ratio histogram of the layer over the live rows ----
             const double top = log2((double)(m > 2 ? m : 2));          // s_j <= j <= m
             const float binscale = (float)((double)kBins / top);
@@ -989,7 +1269,7 @@ k_verify(VerifyArgs a) {
         TS(9);
         // ---- a residual draw locates its tile through tile sums of max(p_beam - s_{j-1} q_beam, 0) ----
         double *res_sums = sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride;   // slot 0 of the bank
-        if (!a.select_mode && !sh.err && sh.res_j > 2) {          // run position 2 is served by the histogram pass
+        if (!a.select_mode && !sh.err && !warped && sh.res_j > 2) {   // run position 2 is served by the histogram pass
             if (threadIdx.x == 0) ++sh.n_respass;
             residual_pass(a, sh, (float)sh.s_arr[sh.res_j - 1], res_sums, cta_rank, n_cta);
             __threadfence();
@@ -1014,11 +1294,19 @@ k_verify(VerifyArgs a) {
                     const bool use_res = residual && j > 1;
                     const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l,
                                                       residual ? 1u : 2u, residual ? 0u : (uint32_t)fill);
-                    double z_res = 0.0;
-                    if (use_res) z_res = ordered_sum(res_sums, sh.nA * a.T, lane);
-                    int ia = 0;
-                    const int tok = draw_cell(a, sh, u, use_res, use_res ? (float)sh.s_arr[j - 1] : 0.f, z_res,
-                                              res_sums, lane, &ia);
+                    int ia = 0, tok;
+                    if (warped) {
+                        int pick = -1;
+                        if (lane == 0) pick = draw_support(wsup, u, use_res ? sh.s_arr[j - 1] : 0.0);
+                        pick = __shfl_sync(kFull, pick, 0);
+                        tok = -1;
+                        if (pick >= 0) { ia = wsup.cell[0][pick] / a.V; tok = wsup.cell[0][pick] - ia * a.V; }
+                    } else {
+                        double z_res = 0.0;
+                        if (use_res) z_res = ordered_sum(res_sums, sh.nA * a.T, lane);
+                        tok = draw_cell(a, sh, u, use_res, use_res ? (float)sh.s_arr[j - 1] : 0.f, z_res, res_sums,
+                                        lane, &ia);
+                    }
                     if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
                     if (lane == 0)
                         emit_output(a, r, &n_out, sh.A[ia], -1, tok, residual ? DSBD_SRC_RESIDUAL : DSBD_SRC_FILL,
@@ -1055,14 +1343,33 @@ k_verify(VerifyArgs a) {
 
     TS(11);
     // ---- every layer passed: W_nom beams from p_beam^(gamma+1) ----
-    if (!a.select_mode && warp == 0 && !sh.done && !sh.err) {
-        live_weights(a, sh, sp_live, sq_live, lane);
-        int err = 0;
+    const bool extra = !a.select_mode && !sh.done && !sh.err;
+    WarpScratch &wsx = *reinterpret_cast<WarpScratch *>(hq);
+    int extra_err = 0;
+    if (extra) {
+        if (warp == 0) live_weights(a, sh, sp_live, sq_live, lane);
+        __syncthreads();
+        if (a.top_k > 0) {
+            extra_err = build_support(a, sh, 0, reinterpret_cast<double *>(hp),
+                                      reinterpret_cast<int *>(hp + 2 * kMaxCand), wsx);
+            if (!extra_err && warp == 0) finish_supports(wsx, false, lane);
+        }
+    }
+    if (extra && warp == 0) {
+        int err = extra_err;
         if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
         for (int kk = 0; kk < W_nom && !err; ++kk) {
             const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1), 3u, (uint32_t)kk);
-            int ia = 0;
-            const int tok = draw_cell(a, sh, u, false, 0.f, 0.0, nullptr, lane, &ia);
+            int ia = 0, tok;
+            if (a.top_k > 0) {
+                int pick = -1;
+                if (lane == 0) pick = draw_support(wsx, u, 0.0);
+                pick = __shfl_sync(kFull, pick, 0);
+                tok = -1;
+                if (pick >= 0) { ia = wsx.cell[0][pick] / a.V; tok = wsx.cell[0][pick] - ia * a.V; }
+            } else {
+                tok = draw_cell(a, sh, u, false, 0.f, 0.0, nullptr, lane, &ia);
+            }
             if (tok < 0) { err = DSBD_DEV_EXHAUSTED; break; }
             if (lane == 0) emit_output(a, r, &n_out, sh.A[ia], -1, tok, DSBD_SRC_EXTRA, writer, &err);
             n_out = __shfl_sync(kFull, n_out, 0);
@@ -1126,6 +1433,9 @@ int check_forest(const dsbd_forest_t *f) {
 int check_params(const dsbd_verify_params_t *p) {
     if (!p || p->V <= 0 || !(p->temperature > 0.f)) return DSBD_ERR_INVALID_ARG;
     if (p->W_min < 1 && !p->W_min_r) return DSBD_ERR_INVALID_ARG;
+    if (p->top_k < 0) return DSBD_ERR_INVALID_ARG;
+    if (p->top_k > 64) return DSBD_ERR_UNSUPPORTED;
+    if (p->top_k == 0 && p->top_p > 0.f && p->top_p < 1.f) return DSBD_ERR_UNSUPPORTED;   // top-p needs a top-k bound
     return DSBD_OK;
 }
 
@@ -1219,6 +1529,7 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
     a.W_min = p->W_min; a.W_max = p->W_max; a.W_nom = p->W_nom;
     a.W_min_r = p->W_min_r; a.W_max_r = p->W_max_r; a.W_nom_r = p->W_nom_r;
     a.seed = p->seed; a.step = p->step;
+    a.top_k = p->top_k; a.top_p = (double)p->top_p;
     a.zp = logits_p; a.zq = logits_q; a.stride = row_stride;
     a.stats = stats; a.lse = lse; a.score = score; a.depth = depth;
     a.tile_sums = reinterpret_cast<double *>(ws + L.sums);
@@ -1365,6 +1676,7 @@ extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_param
     a.W_min = p->W_min; a.W_max = p->W_max; a.W_nom = p->W_nom;
     a.W_min_r = p->W_min_r; a.W_max_r = p->W_max_r; a.W_nom_r = p->W_nom_r;
     a.seed = p->seed; a.step = p->step;
+    a.top_k = p->top_k; a.top_p = (double)p->top_p;
     a.zp = logits_p; a.zq = logits_q; a.stride = row_stride;
     a.stats = stats; a.lse = lse; a.score = nullptr; a.depth = nullptr;
     a.tile_sums = reinterpret_cast<double *>(ws + L.sums);

@@ -190,6 +190,39 @@ def test_peaky_distributions_use_the_exact_fallback():
     assert fallbacks > 0
 
 
+@pytest.mark.parametrize("name,steps", [("C1", range(30)), ("C2", range(30)), ("C3", range(4)), ("C4", range(3))])
+def test_configs_with_the_papers_warping(name, steps):
+    """top-k 10 / top-p 0.8 on the joint distributions, the setting of the paper's experiments."""
+    data = inputs.generate(inputs.config(name), "cuda", parts=("verify",))
+    data["params"].update(top_k=10, top_p=0.8)
+    _both(data, steps)
+
+
+@pytest.mark.parametrize("top_k,top_p", [(1, 1.0), (3, 0.5), (64, 1.0), (64, 0.95), (7, 0.05)])
+def test_warping_edge_settings(top_k, top_p):
+    rng = np.random.default_rng(top_k)
+    exempt = decisions = 0
+    for trial in range(4):
+        forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=6, V=2100, gamma=3, max_w=5,
+                                                              tree="binary" if trial % 2 else "chain")
+        # make some drafts land inside the warped support: the best tokens of the small model
+        best = np.argsort(-zq[:, :2100], axis=1)[:, :3]
+        for n in range(forest["N"]):
+            if forest["parent"][n] >= 0 and rng.uniform() < 0.7:
+                forest["token"][n] = best[forest["parent"][n], rng.integers(0, 3)]
+        prm.update(top_k=top_k, top_p=top_p, step=trial)
+        dz = lambda a: torch.as_tensor(a).cuda()
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+        # drafts outside the support of the warped q_beam are events of probability zero; when
+        # one is rejected where no residual mass is left, both sides report it (code 2)
+        assert status in (0, 2)
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64))
+        e, d = compare_verify(ref, gpu, forest, allow_exhausted=True)
+        exempt += e; decisions += d
+        assert (ref["error"] == 0).sum() >= 1
+    check_exempt(exempt, decisions)
+
+
 def test_roots_only_forest_goes_straight_to_the_extra_layer():
     rng = np.random.default_rng(3)
     V, B = 2000, 3
