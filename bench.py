@@ -196,7 +196,8 @@ def run_reference(args):
     spec = inputs.config(args.workload)
     # a slice of the workload is enough for the sample: fewer requests, same shapes
     small = dict(spec, R=min(spec["R"], 2))
-    data = inputs.generate(small, "cpu")
+    data = inputs.generate(small, "cpu", draft_top_k=args.top_k, draft_top_p=args.top_p)
+    data["params"].update(top_k=args.top_k, top_p=args.top_p)
     views = _host_views(data, small)
     views["max_reqs"], views["max_beams"] = 1, 1
     threads = os.cpu_count() or 1
@@ -253,7 +254,8 @@ def main():
     if args.requests > 0:
         spec["R"] = args.requests
     spec = rank_spec(spec, rank)                         # every rank verifies its own requests
-    data = inputs.generate(spec, dev)
+    data = inputs.generate(spec, dev, draft_top_k=args.top_k, draft_top_p=args.top_p)
+    data["params"].update(top_k=args.top_k, top_p=args.top_p)
     forest, prm, poff = data["forest"], dict(data["params"]), data["prefix_off"]
     prm.update(top_k=args.top_k, top_p=args.top_p)
     f = dsbd.Forest(forest, dev)

@@ -40,8 +40,7 @@ enum {
 /* device-side codes written to *status / req_error */
 enum {
     DSBD_DEV_BAD_TOKEN = 1,      /* draft token outside [0, V)                               */
-    DSBD_DEV_EXHAUSTED = 2,      /* a draw from a distribution without mass, or a rejection
-                                    that had probability zero                                */
+    DSBD_DEV_EXHAUSTED = 2,      /* a draw from a distribution without mass                  */
     DSBD_DEV_CAPACITY = 3,       /* more output beams than the request's out_off range holds */
     DSBD_DEV_BAD_FOREST = 4,     /* parent index outside its tree, too many live beams/drafts */
     DSBD_DEV_TIMEOUT = 5         /* a bounded wait gave up                                   */

@@ -502,16 +502,17 @@ static void verify_request(req_ctx *c, int32_t r, const int32_t *depth, const in
                 double z = 0.0;
                 for (int64_t k = 0; k < cells; ++k) {
                     double d = p_cur[k] - q_beam[k];
-                    p_cur[k] = d > 0.0 ? d : 0.0;
-                    z += p_cur[k];
+                    z += d > 0.0 ? d : 0.0;
                 }
                 if (z > 0.0) {
-                    for (int64_t k = 0; k < cells; ++k) p_cur[k] /= z;
-                } else {
-                    /* a rejection that had probability zero: p' == q_beam */
-                    err = DSBD_O_ERR_EXHAUSTED;
-                    memcpy(p_cur, p_beam, sizeof(double) * (size_t)cells);
+                    for (int64_t k = 0; k < cells; ++k) {
+                        double d = p_cur[k] - q_beam[k];
+                        p_cur[k] = (d > 0.0 ? d : 0.0) / z;
+                    }
                 }
+                /* else p' == q_beam: only a draft outside the support of q_beam can be rejected
+                 * there (an event of probability zero when the drafts are samples of q_beam);
+                 * it carries nothing to subtract and p' stays as it is */
             }
         }
         for (int32_t i = 0; i < m; ++i)

@@ -1243,12 +1243,9 @@ k_verify(VerifyArgs a) {
                     } else {
                         st[n - n_lo] = DSBD_NODE_REJECTED;
                         if (writer) a.out.node_status[n] = DSBD_NODE_REJECTED;
-                        if (j <= sh.chain_len && sh.c_arr[j + 1] > 0.0) {
-                            ++j;
-                        } else {
-                            err = DSBD_DEV_EXHAUSTED;     // a rejection of probability zero
-                            j = 1;
-                        }
+                        // an empty residual means p' == q_beam: the rejected draft lay outside the
+                        // support of q_beam, there is nothing to subtract and p' stays
+                        if (j <= sh.chain_len && sh.c_arr[j + 1] > 0.0) ++j;
                     }
                 }
                 for (int i = 0; i < m; ++i)

@@ -80,8 +80,12 @@ def build_forest(spec, rng):
     return forest, widths, prefix_off
 
 
-def generate(spec, device, parts=("attention", "verify")):
+def generate(spec, device, parts=("attention", "verify"), draft_top_k=0, draft_top_p=1.0):
     """All tensors of one decode step on `device`, from one seeded torch generator.
+
+    draft_top_k / draft_top_p: when set, every draft token is drawn by ordinary per-row top-k /
+    top-p sampling from the small model's next-token distribution (the usual sampler of a
+    draft model run with warping), so the drafts are high-probability tokens.
 
     Returns a dict: forest (numpy arrays), widths, prefix_off (numpy int64), params (python
     scalars + per-request width arrays as numpy), and the torch tensors q, k_new, v_new,
@@ -137,7 +141,16 @@ def generate(spec, device, parts=("attention", "verify")):
         for s in range(0, nonroot.numel(), rows):
             idx = nonroot[s:s + rows]
             probs = torch.softmax(zq[parent[idx].long()] / tau, dim=1)
-            token[idx] = torch.multinomial(probs, 1, generator=gen).squeeze(1)
+            if draft_top_k > 0:
+                top, ids = torch.topk(probs, min(int(draft_top_k), V), dim=1)
+                if 0.0 < draft_top_p < 1.0:
+                    top = top / top.sum(1, keepdim=True)
+                    before = torch.cumsum(top, 1) - top
+                    top = torch.where(before < draft_top_p, top, torch.zeros_like(top))
+                pick = torch.multinomial(top, 1, generator=gen)
+                token[idx] = ids.gather(1, pick).squeeze(1)
+            else:
+                token[idx] = torch.multinomial(probs, 1, generator=gen).squeeze(1)
         forest["token"] = token.to(torch.int32).cpu().numpy()
         W_cfg = spec["W"][1] if isinstance(spec["W"], tuple) else spec["W"]
         out["params"] = dict(V=V, temperature=tau, thresh=0.7, W_min=1, W_max=W_cfg, W_nom=W_cfg,

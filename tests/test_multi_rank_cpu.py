@@ -53,7 +53,7 @@ def test_two_gloo_ranks_share_only_the_clock():
 def test_reference_arm_prints_one_json_line(capsys):
     import json
     import types
-    args = types.SimpleNamespace(workload="C1", warmup=0, steps=1, gpus=1)
+    args = types.SimpleNamespace(workload="C1", warmup=0, steps=1, gpus=1, top_k=0, top_p=1.0)
     bench.run_reference(args)
     line = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == bench.UNIT and line["value"] > 0
