@@ -242,6 +242,47 @@ int dsbd_select_width(const dsbd_forest_t *forest, const dsbd_verify_params_t *p
                       void *workspace, size_t workspace_bytes, int32_t *status,
                       dsbd_stream_t stream);
 
+/* KV-cache update at the end of a decode step (Section "Forest-based Parallel Decoding": after
+ * the iteration the key-value caches are updated according to the output beams, an output beam
+ * keeping the cache of the input beam it descends from; Section "Reducing Memory Cost": keeping
+ * only the output beam of lowest perplexity leaves one cache per request).
+ *
+ * An output beam in slot s (parent node n = out_parent[s], input beam b = out_root_beam[s])
+ * gets the cache  [cache of b] ++ [keys/values of the nodes on the path root(b) .. n], which is
+ * exactly what n attended to; its new token becomes the root of the next draft tree.  Kept
+ * beams are numbered request by request, inside a request in slot order, and their caches are
+ * written packed in the layout dsbd_forest_attention reads: new beam j as [Hkv, L'_j, d]
+ * starting at element new_prefix_off[j]*Hkv*d of k_dst / v_dst, L'_j = L_b + depth(n) + 1.
+ * keep_best: per request only the slot of lowest perplexity exp(-out_logp/(L'+1)) is kept (the
+ * lower slot on a tie).
+ *
+ * Device inputs: the forest; out_off [R+1], out_width [R], out_parent, out_root_beam, out_logp
+ * as dsbd_verify_step wrote them (out_logp is read only with keep_best); k_new, v_new, k_prefix,
+ * v_prefix, prefix_off as given to dsbd_forest_attention (desc gives Hkv, d, dtype).
+ * Device outputs: k_dst, v_dst (dst_capacity tokens each, 16-byte aligned, must not overlap the
+ * inputs); new_req_beam_off [R+1]; new_prefix_off [n_slots+1] (entries past the number of kept
+ * beams repeat the total); new_beam_slot [n_slots] (the output slot each new beam came from, -1
+ * past the end).  n_slots is the host's copy of out_off[R].
+ * *status: DSBD_DEV_CAPACITY when the kept caches need more than dst_capacity tokens,
+ * DSBD_DEV_BAD_FOREST when a slot names a beam outside its request or a node outside that
+ * beam's tree; nothing is copied then. */
+typedef struct {
+    int32_t n_slots;
+    int32_t keep_best;
+    int64_t dst_capacity;
+} dsbd_commit_params_t;
+
+int dsbd_kv_commit(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
+                   const dsbd_commit_params_t *params,
+                   const int32_t *out_off, const int32_t *out_width, const int32_t *out_parent,
+                   const int32_t *out_root_beam, const float *out_logp,
+                   const void *k_new, const void *v_new, const void *k_prefix, const void *v_prefix,
+                   const int64_t *prefix_off, void *k_dst, void *v_dst,
+                   int32_t *new_req_beam_off, int64_t *new_prefix_off, int32_t *new_beam_slot,
+                   void *workspace, size_t workspace_bytes, int32_t *status, dsbd_stream_t stream);
+
+size_t dsbd_kv_commit_workspace(const dsbd_forest_t *forest, const dsbd_commit_params_t *params);
+
 const char *dsbd_status_string(int code);
 
 #ifdef __cplusplus

@@ -21,7 +21,7 @@ MAX_LIVE = 64
 
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
-           "dsbd_status_string"]
+           "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_status_string"]
 
 _vp = C.c_void_p
 
@@ -91,6 +91,10 @@ def load():
     lib.dsbd_select_width.restype = C.c_int
     lib.dsbd_select_width.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, _vp,
                                       _vp, _vp, C.c_int32, _vp, C.c_size_t, _vp, _vp]
+    lib.dsbd_kv_commit_workspace.restype = C.c_size_t
+    lib.dsbd_kv_commit_workspace.argtypes = [_vp, _vp]
+    lib.dsbd_kv_commit.restype = C.c_int
+    lib.dsbd_kv_commit.argtypes = [_vp] * 19 + [C.c_size_t, _vp, _vp]
     _lib = lib
     return lib
 
@@ -210,6 +214,45 @@ def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_pre
     if rc != OK:
         raise DsbdError("dsbd_forest_attention", rc)
     return out, status
+
+
+class CommitParamsT(C.Structure):
+    _fields_ = [("n_slots", C.c_int32), ("keep_best", C.c_int32), ("dst_capacity", C.c_int64)]
+
+
+def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out_logp, k_new, v_new,
+              k_prefix, v_prefix, prefix_off, prefix_off_host, n_slots, dst_capacity, keep_best=False,
+              k_dst=None, v_dst=None, workspace=None, status=None, stream=None):
+    """dsbd_kv_commit; returns a dict with k_dst, v_dst, new_req_beam_off, new_prefix_off,
+    new_beam_slot and the status tensor (all on the device, nothing is synchronised)."""
+    _require_cuda(out_off, out_width, out_parent, out_root_beam, k_new, v_new, k_prefix, v_prefix, prefix_off)
+    dev = k_new.device
+    f = forest.struct()
+    desc = _attn_desc(Hkv, Hkv, d, k_new.dtype, 1.0, prefix_off_host)
+    p = CommitParamsT()
+    p.n_slots, p.keep_best, p.dst_capacity = int(n_slots), int(bool(keep_best)), int(dst_capacity)
+    if k_dst is None:
+        k_dst = torch.empty(int(dst_capacity) * Hkv * d, dtype=k_new.dtype, device=dev)
+    if v_dst is None:
+        v_dst = torch.empty(int(dst_capacity) * Hkv * d, dtype=k_new.dtype, device=dev)
+    need = int(load().dsbd_kv_commit_workspace(C.addressof(f), C.addressof(p)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    new_req_beam_off = torch.empty(forest.R + 1, dtype=torch.int32, device=dev)
+    new_prefix_off = torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev)
+    new_beam_slot = torch.empty(int(n_slots), dtype=torch.int32, device=dev)
+    rc = load().dsbd_kv_commit(C.addressof(f), C.addressof(desc), C.addressof(p), _ptr(out_off), _ptr(out_width),
+                               _ptr(out_parent), _ptr(out_root_beam), _ptr(out_logp) if out_logp is not None else None,
+                               _ptr(k_new), _ptr(v_new), _ptr(k_prefix), _ptr(v_prefix), _ptr(prefix_off),
+                               _ptr(k_dst), _ptr(v_dst), _ptr(new_req_beam_off), _ptr(new_prefix_off),
+                               _ptr(new_beam_slot), _ptr(workspace), workspace.numel(), _ptr(status),
+                               _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_kv_commit", rc)
+    return dict(k_dst=k_dst, v_dst=v_dst, new_req_beam_off=new_req_beam_off, new_prefix_off=new_prefix_off,
+                new_beam_slot=new_beam_slot, status=status, workspace=workspace)
 
 
 def _params(params, keep):

@@ -1,0 +1,314 @@
+// KV-cache update at the end of a decode step (Section "Forest-based Parallel Decoding": the
+// caches are updated according to the output beams; Section "Reducing Memory Cost": keep only
+// the output beam of lowest perplexity).
+//
+//   k_commit_plan   one CTA: which output slots survive, their new cache lengths, the packed
+//                   offsets of the new caches, the nodes on each kept beam's path, and the list
+//                   of copy chunks.
+//   k_commit_copy   a streaming copy: every (new beam, kv head, K|V) is a byte stream -- the
+//                   input beam's cache, then one row per path node -- cut into 32 KB chunks;
+//                   CTAs walk the chunk list with 128-bit loads kept out of L1 and streaming
+//                   stores.  HBM-bound: read + write of every kept cache once.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dsbd_common.cuh"
+
+namespace {
+using namespace dsbd;
+
+constexpr int kPlanThreads = 1024;
+constexpr int kCopyThreads = 256;
+constexpr int kChunkBytes = 32768;                  // 8 x 16 B per thread
+constexpr int kUnits = kChunkBytes / 16 / kCopyThreads;
+
+struct Plan {
+    int32_t n_beams;          // kept output beams
+    int32_t error;
+    int64_t n_chunks;         // chunks of one (kv head, K|V) stream summed over the beams
+    int64_t total_tokens;
+};
+
+struct CommitArgs {
+    int R, B, N, gamma, Hkv, n_slots, keep_best;
+    int row_bytes;                                  // d * element size
+    int64_t capacity;
+    const int32_t *req_beam_off, *beam_node_off, *parent;
+    const int32_t *out_off, *out_width, *out_parent, *out_root_beam;
+    const float *out_logp;
+    const int64_t *prefix_off;
+    const unsigned char *k_new, *v_new, *k_prefix, *v_prefix;
+    unsigned char *k_dst, *v_dst;
+    int32_t *new_req_beam_off, *new_beam_slot;
+    int64_t *new_prefix_off;
+    // workspace
+    Plan *plan;
+    int32_t *req_count;       // [R]     kept beams of the request, then its first new beam
+    int32_t *src_beam;        // [n_slots]
+    int32_t *path;            // [n_slots][gamma+1] nodes root .. parent
+    int32_t *path_len;        // [n_slots]
+    int64_t *chunk_off;       // [n_slots+1]
+    int32_t *status;
+};
+
+// exclusive scan of v[0..n) in place by one CTA; returns the total in every thread
+template <typename T>
+__device__ T block_exclusive_scan(T *v, int n, T *warp_tot /*[32]*/) {
+    const int per = (n + blockDim.x - 1) / blockDim.x;
+    const int lo = min((int)threadIdx.x * per, n), hi = min(lo + per, n);
+    T local = 0;
+    for (int i = lo; i < hi; ++i) local += v[i];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    T incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const T t = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    T base = 0, total = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+        if (w < warp) base += warp_tot[w];
+        total += warp_tot[w];
+    }
+    T run = base + incl - local;
+    for (int i = lo; i < hi; ++i) { const T x = v[i]; v[i] = run; run += x; }
+    __syncthreads();
+    return total;
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+k_commit_plan(CommitArgs a) {
+    __shared__ int64_t tot64[32];
+    __shared__ int32_t tot32[32];
+    __shared__ int bad;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    // kept slots per request
+    for (int r = threadIdx.x; r < a.R; r += blockDim.x) {
+        const int w = a.out_width[r];
+        a.req_count[r] = w <= 0 ? 0 : (a.keep_best ? 1 : w);
+    }
+    __syncthreads();
+    const int n_beams = block_exclusive_scan<int32_t>(a.req_count, a.R, tot32);
+    if (n_beams > a.n_slots) { if (threadIdx.x == 0) bad = DSBD_DEV_CAPACITY; }
+    __syncthreads();
+    const bool fits = !bad;
+    // per request: its kept slots -> source beam, path, new length
+    for (int r = threadIdx.x; r < a.R && fits; r += blockDim.x) {
+        const int first = a.req_count[r];
+        a.new_req_beam_off[r] = first;
+        const int s0 = a.out_off[r], w = a.out_width[r];
+        if (w <= 0) continue;
+        int s_lo = s0, s_hi = s0 + w;
+        const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
+        if (a.keep_best) {
+            // lowest perplexity exp(-logp / length) = lowest -logp / length; first slot on a tie
+            int best = -1;
+            double best_key = 0.0;
+            for (int s = s_lo; s < s_hi; ++s) {
+                const int b = a.out_root_beam[s];
+                int n = a.out_parent[s];
+                if (b < b_lo || b >= b_hi || n < a.beam_node_off[b] || n >= a.beam_node_off[b + 1]) { bad = DSBD_DEV_BAD_FOREST; break; }
+                int depth = 0;
+                while (a.parent[n] >= 0 && depth <= a.gamma) { n = a.parent[n]; ++depth; }
+                const double length = (double)(a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 2;
+                const double key = -(double)a.out_logp[s] / length;
+                if (best < 0 || key < best_key) { best = s; best_key = key; }
+            }
+            if (best < 0) continue;
+            s_lo = best; s_hi = best + 1;
+        }
+        for (int s = s_lo; s < s_hi; ++s) {
+            const int j = first + (s - s_lo);
+            const int b = a.out_root_beam[s];
+            int n = a.out_parent[s];
+            if (b < b_lo || b >= b_hi || n < a.beam_node_off[b] || n >= a.beam_node_off[b + 1]) { bad = DSBD_DEV_BAD_FOREST; break; }
+            int depth = 0;
+            for (int c = n; a.parent[c] >= 0 && depth <= a.gamma; c = a.parent[c]) ++depth;
+            if (depth > a.gamma) { bad = DSBD_DEV_BAD_FOREST; break; }
+            int32_t *pj = a.path + (int64_t)j * (a.gamma + 1);
+            for (int c = n, i = depth; i >= 0; --i, c = a.parent[c]) pj[i] = c;
+            a.path_len[j] = depth + 1;
+            a.src_beam[j] = b;
+            a.new_beam_slot[j] = s;
+            const int64_t len = (a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 1;
+            a.new_prefix_off[j] = len;
+            a.chunk_off[j] = (len * a.row_bytes + kChunkBytes - 1) / kChunkBytes;
+        }
+    }
+    __syncthreads();
+    const bool ok = !bad;
+    const int nb = ok ? n_beams : 0;
+    if (threadIdx.x == 0) a.new_req_beam_off[a.R] = nb;
+    for (int r = threadIdx.x; r < a.R && !ok; r += blockDim.x) a.new_req_beam_off[r] = 0;
+    for (int j = nb + threadIdx.x; j < a.n_slots; j += blockDim.x) {
+        a.new_beam_slot[j] = -1;
+        a.new_prefix_off[j] = 0;
+        a.chunk_off[j] = 0;
+    }
+    __syncthreads();
+    const int64_t total = block_exclusive_scan<int64_t>(a.new_prefix_off, a.n_slots, tot64);
+    const int64_t chunks = block_exclusive_scan<int64_t>(a.chunk_off, a.n_slots, tot64);
+    if (threadIdx.x == 0) {
+        a.new_prefix_off[a.n_slots] = total;
+        a.chunk_off[a.n_slots] = chunks;
+        int err = bad;
+        if (!err && total > a.capacity) err = DSBD_DEV_CAPACITY;
+        a.plan->n_beams = nb;
+        a.plan->error = err;
+        a.plan->total_tokens = total;
+        a.plan->n_chunks = err ? 0 : chunks;
+        if (err) report(a.status, err);
+    }
+}
+
+__device__ __forceinline__ uint4 ld_stream16(const unsigned char *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream16(unsigned char *p, const uint4 &v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// Item = (chunk of the per-beam chunk list, kv head, K|V).  All offsets are multiples of 16
+// bytes because a row (d elements) is.
+__global__ void __launch_bounds__(kCopyThreads)
+k_commit_copy(CommitArgs a) {
+    __shared__ int s_j;
+    const int64_t n_chunks = a.plan->n_chunks;
+    const int n_beams = a.plan->n_beams;
+    const int64_t items = n_chunks * a.Hkv * 2;
+    const int rb = a.row_bytes;
+    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+        const int kv = (int)(item & 1);
+        const int64_t rest = item >> 1;
+        const int g = (int)(rest % a.Hkv);
+        const int64_t c = rest / a.Hkv;
+        if (threadIdx.x == 0) {
+            int lo = 0, hi = n_beams - 1;              // last j with chunk_off[j] <= c
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (a.chunk_off[mid] <= c) lo = mid; else hi = mid - 1;
+            }
+            s_j = lo;
+        }
+        __syncthreads();
+        const int j = s_j;
+        const int b = a.src_beam[j];
+        const int64_t L_old = a.prefix_off[b + 1] - a.prefix_off[b];
+        const int plen = a.path_len[j];
+        const int64_t L_new = L_old + plen;
+        const int64_t stream_bytes = L_new * rb, old_bytes = L_old * rb;
+        const int64_t start = (c - a.chunk_off[j]) * (int64_t)kChunkBytes;
+        const unsigned char *src_old = (kv ? a.v_prefix : a.k_prefix) + (a.prefix_off[b] * a.Hkv + (int64_t)g * L_old) * rb;
+        const unsigned char *src_new = kv ? a.v_new : a.k_new;
+        unsigned char *dst = (kv ? a.v_dst : a.k_dst) + ((a.new_prefix_off[j]) * a.Hkv + (int64_t)g * L_new) * rb;
+        const int32_t *path = a.path + (int64_t)j * (a.gamma + 1);
+        uint4 v[kUnits];
+        int64_t off[kUnits];
+#pragma unroll
+        for (int u = 0; u < kUnits; ++u) {
+            off[u] = start + ((int64_t)u * kCopyThreads + threadIdx.x) * 16;
+            if (off[u] < old_bytes) {
+                v[u] = ld_stream16(src_old + off[u]);
+            } else if (off[u] < stream_bytes) {
+                const int64_t o = off[u] - old_bytes;
+                const int t = (int)(o / rb);
+                const int within = (int)(o - (int64_t)t * rb);
+                v[u] = ld_stream16(src_new + ((int64_t)path[t] * a.Hkv + g) * rb + within);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnits; ++u)
+            if (off[u] < stream_bytes) st_stream16(dst + off[u], v[u]);
+        __syncthreads();
+    }
+}
+
+struct Layout {
+    size_t plan, req_count, src_beam, path, path_len, chunk_off, total;
+};
+
+Layout make_layout(const dsbd_forest_t *f, const dsbd_commit_params_t *p) {
+    Layout L;
+    size_t off = 0;
+    L.plan = off;      off = align_up(off + sizeof(Plan), 256);
+    L.req_count = off; off = align_up(off + sizeof(int32_t) * (size_t)f->R, 256);
+    L.src_beam = off;  off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots, 256);
+    L.path = off;      off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots * ((size_t)f->max_depth + 1), 256);
+    L.path_len = off;  off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots, 256);
+    L.chunk_off = off; off = align_up(off + sizeof(int64_t) * ((size_t)p->n_slots + 1), 256);
+    L.total = off;
+    return L;
+}
+
+bool args_ok(const dsbd_forest_t *f, const dsbd_commit_params_t *p) {
+    return f && p && f->R > 0 && f->B > 0 && f->N > 0 && f->max_depth >= 0 && f->req_beam_off &&
+           f->beam_node_off && f->parent && p->n_slots > 0 && p->dst_capacity >= 0;
+}
+
+}  // namespace
+
+extern "C" size_t dsbd_kv_commit_workspace(const dsbd_forest_t *forest, const dsbd_commit_params_t *params) {
+    if (!args_ok(forest, params)) return 0;
+    return make_layout(forest, params).total;
+}
+
+extern "C" int dsbd_kv_commit(const dsbd_forest_t *f, const dsbd_attn_desc_t *desc, const dsbd_commit_params_t *p,
+                              const int32_t *out_off, const int32_t *out_width, const int32_t *out_parent,
+                              const int32_t *out_root_beam, const float *out_logp, const void *k_new,
+                              const void *v_new, const void *k_prefix, const void *v_prefix,
+                              const int64_t *prefix_off, void *k_dst, void *v_dst, int32_t *new_req_beam_off,
+                              int64_t *new_prefix_off, int32_t *new_beam_slot, void *workspace,
+                              size_t workspace_bytes, int32_t *status, dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    if (!args_ok(f, p) || !desc) return DSBD_ERR_INVALID_ARG;
+    if (!out_off || !out_width || !out_parent || !out_root_beam || !k_new || !v_new || !k_prefix || !v_prefix ||
+        !prefix_off || !k_dst || !v_dst || !new_req_beam_off || !new_prefix_off || !new_beam_slot || !workspace ||
+        !status)
+        return DSBD_ERR_INVALID_ARG;
+    if (p->keep_best && !out_logp) return DSBD_ERR_INVALID_ARG;
+    if (desc->Hkv <= 0 || desc->d <= 0) return DSBD_ERR_INVALID_ARG;
+    if (desc->dtype != DSBD_DTYPE_BF16 && desc->dtype != DSBD_DTYPE_F32) return DSBD_ERR_UNSUPPORTED;
+    const int row_bytes = desc->d * (desc->dtype == DSBD_DTYPE_BF16 ? 2 : 4);
+    if (row_bytes % 16) return DSBD_ERR_UNSUPPORTED;
+    const uintptr_t ptrs = reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
+                           reinterpret_cast<uintptr_t>(k_prefix) | reinterpret_cast<uintptr_t>(v_prefix) |
+                           reinterpret_cast<uintptr_t>(k_dst) | reinterpret_cast<uintptr_t>(v_dst);
+    if (ptrs & 15) return DSBD_ERR_UNSUPPORTED;
+    const Layout L = make_layout(f, p);
+    if (workspace_bytes < L.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+
+    CommitArgs a = {};
+    a.R = f->R; a.B = f->B; a.N = f->N; a.gamma = f->max_depth; a.Hkv = desc->Hkv;
+    a.n_slots = p->n_slots; a.keep_best = p->keep_best ? 1 : 0; a.row_bytes = row_bytes;
+    a.capacity = p->dst_capacity;
+    a.req_beam_off = f->req_beam_off; a.beam_node_off = f->beam_node_off; a.parent = f->parent;
+    a.out_off = out_off; a.out_width = out_width; a.out_parent = out_parent; a.out_root_beam = out_root_beam;
+    a.out_logp = out_logp; a.prefix_off = prefix_off;
+    a.k_new = static_cast<const unsigned char *>(k_new); a.v_new = static_cast<const unsigned char *>(v_new);
+    a.k_prefix = static_cast<const unsigned char *>(k_prefix);
+    a.v_prefix = static_cast<const unsigned char *>(v_prefix);
+    a.k_dst = static_cast<unsigned char *>(k_dst); a.v_dst = static_cast<unsigned char *>(v_dst);
+    a.new_req_beam_off = new_req_beam_off; a.new_prefix_off = new_prefix_off; a.new_beam_slot = new_beam_slot;
+    a.plan = reinterpret_cast<Plan *>(ws + L.plan);
+    a.req_count = reinterpret_cast<int32_t *>(ws + L.req_count);
+    a.src_beam = reinterpret_cast<int32_t *>(ws + L.src_beam);
+    a.path = reinterpret_cast<int32_t *>(ws + L.path);
+    a.path_len = reinterpret_cast<int32_t *>(ws + L.path_len);
+    a.chunk_off = reinterpret_cast<int64_t *>(ws + L.chunk_off);
+    a.status = status;
+
+    k_commit_plan<<<1, kPlanThreads, 0, stream>>>(a);
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    k_commit_copy<<<sms * 8, kCopyThreads, 0, stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
