@@ -341,6 +341,38 @@ def main():
     torch.cuda.synchronize()
     dense_ms = d0.elapsed_time(d1) / n_dense
 
+    # the KV-cache update of the step's output beams (reported beside the step, not part of it)
+    esz = data["k_new"].element_size()
+    n_slots = int(out_off[-1])
+    ow = vout["out_width"].cpu().numpy().astype(np.int64)
+    L_req = np.diff(poff)[np.asarray(forest["req_beam_off"][:-1])]          # beams of a request share a length
+    cap = int((ow * (L_req + forest["max_depth"] + 1)).sum()) + 1
+    out_off_dev = torch.as_tensor(np.asarray(out_off, dtype=np.int32)).to(dev)
+    k_dst = torch.empty(cap * spec["Hkv"] * spec["d"], dtype=data["k_new"].dtype, device=dev)
+    v_dst = torch.empty_like(k_dst)
+    commit = None
+
+    def kv_commit():
+        return dsbd.kv_commit(f, spec["Hkv"], spec["d"], out_off_dev, vout["out_width"], vout["out_parent"],
+                              vout["out_root_beam"], vout["out_logp"], data["k_new"], data["v_new"],
+                              data["k_prefix"], data["v_prefix"], poff_dev, poff, n_slots=n_slots,
+                              dst_capacity=cap, k_dst=k_dst, v_dst=v_dst,
+                              workspace=commit["workspace"] if commit else None, status=status, stream=stream)
+    for _ in range(3):
+        commit = kv_commit()
+    c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True)
+    n_commit = max(args.steps // 4, 5)
+    c0.record(stream)
+    for _ in range(n_commit):
+        kv_commit()
+    c1.record(stream)
+    torch.cuda.synchronize()
+    commit_ms = c0.elapsed_time(c1) / n_commit
+    commit_tokens = int(commit["new_prefix_off"][-1].item())
+    commit_bytes = commit_tokens * spec["Hkv"] * spec["d"] * esz * 2 * 2      # K and V, read and write
+    assert int(status.item()) == 0, "device status %d" % int(status.item())
+    del k_dst, v_dst
+
     # end to end through the C ABI with host buffers
     e2e = None
     if args.e2e_steps > 0:
@@ -391,6 +423,7 @@ def main():
         "forest_attention": {"bytes": a_bytes, "ms": attn_ms, "gbs": a_bytes / attn_ms * 1e-6},
         "verify_dense_pass": {"bytes": v_bytes, "ms": dense_ms, "gbs": v_bytes / dense_ms * 1e-6},
         "verify_step_total": {"bytes": v_bytes, "ms": ver_ms, "gbs": v_bytes / ver_ms * 1e-6},
+        "kv_commit": {"bytes": commit_bytes, "ms": commit_ms, "gbs": commit_bytes / commit_ms * 1e-6},
     }
     for k in kernels.values():
         k["frac_of_%s_peak" % peak_kind] = k["gbs"] / peak

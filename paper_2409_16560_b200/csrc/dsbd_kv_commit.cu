@@ -6,7 +6,7 @@
 //                   offsets of the new caches, the nodes on each kept beam's path, and the list
 //                   of copy chunks.
 //   k_commit_copy   a streaming copy: every (new beam, kv head, K|V) is a byte stream -- the
-//                   input beam's cache, then one row per path node -- cut into 32 KB chunks;
+//                   input beam's cache, then one row per path node -- cut into 128 KB chunks;
 //                   CTAs walk the chunk list with 128-bit loads kept out of L1 and streaming
 //                   stores.  HBM-bound: read + write of every kept cache once.
 #include <cuda_runtime.h>
@@ -19,8 +19,10 @@ using namespace dsbd;
 
 constexpr int kPlanThreads = 1024;
 constexpr int kCopyThreads = 256;
-constexpr int kChunkBytes = 32768;                  // 8 x 16 B per thread
-constexpr int kUnits = kChunkBytes / 16 / kCopyThreads;
+constexpr int kRoundBytes = 32768;                  // 8 x 16 B per thread in flight
+constexpr int kRounds = 4;
+constexpr int kChunkBytes = kRoundBytes * kRounds;  // one work item
+constexpr int kUnits = kRoundBytes / 16 / kCopyThreads;
 
 struct Plan {
     int32_t n_beams;          // kept output beams
@@ -209,23 +211,27 @@ k_commit_copy(CommitArgs a) {
         const unsigned char *src_new = kv ? a.v_new : a.k_new;
         unsigned char *dst = (kv ? a.v_dst : a.k_dst) + ((a.new_prefix_off[j]) * a.Hkv + (int64_t)g * L_new) * rb;
         const int32_t *path = a.path + (int64_t)j * (a.gamma + 1);
-        uint4 v[kUnits];
-        int64_t off[kUnits];
+        for (int round = 0; round < kRounds; ++round) {
+            const int64_t r0 = start + (int64_t)round * kRoundBytes;
+            if (r0 >= stream_bytes) break;
+            uint4 v[kUnits];
+            int64_t off[kUnits];
 #pragma unroll
-        for (int u = 0; u < kUnits; ++u) {
-            off[u] = start + ((int64_t)u * kCopyThreads + threadIdx.x) * 16;
-            if (off[u] < old_bytes) {
-                v[u] = ld_stream16(src_old + off[u]);
-            } else if (off[u] < stream_bytes) {
-                const int64_t o = off[u] - old_bytes;
-                const int t = (int)(o / rb);
-                const int within = (int)(o - (int64_t)t * rb);
-                v[u] = ld_stream16(src_new + ((int64_t)path[t] * a.Hkv + g) * rb + within);
+            for (int u = 0; u < kUnits; ++u) {
+                off[u] = r0 + ((int64_t)u * kCopyThreads + threadIdx.x) * 16;
+                if (off[u] < old_bytes) {
+                    v[u] = ld_stream16(src_old + off[u]);
+                } else if (off[u] < stream_bytes) {
+                    const int64_t o = off[u] - old_bytes;
+                    const int t = (int)(o / rb);
+                    const int within = (int)(o - (int64_t)t * rb);
+                    v[u] = ld_stream16(src_new + ((int64_t)path[t] * a.Hkv + g) * rb + within);
+                }
             }
-        }
 #pragma unroll
-        for (int u = 0; u < kUnits; ++u)
-            if (off[u] < stream_bytes) st_stream16(dst + off[u], v[u]);
+            for (int u = 0; u < kUnits; ++u)
+                if (off[u] < stream_bytes) st_stream16(dst + off[u], v[u]);
+        }
         __syncthreads();
     }
 }
