@@ -294,3 +294,36 @@ def select_width(forest, params, logits_p, logits_q, node_logp, node_logq, live_
     if rc:
         raise ValueError("oracle select_width: error %d" % rc)
     return width, alpha[:, :mmax], tail
+
+
+def draft_layer(req_beam_off, params, layer, W_S, logits_q, beam_logq, out_off=None, inject_u=None):
+    """One beam-sampling step of the small model: W_S (int or [R] array) iid draws per request
+    from q_beam over its current beams x V.  params: V, temperature, seed, step, top_k, top_p,
+    req_id.  Returns dict(out_off, out_parent, out_token, out_logq, cdf_lo, cdf_hi, error)."""
+    rbo = _arr(req_beam_off, np.int32)
+    R = len(rbo) - 1
+    keep = []
+    p = _params(params, R, keep)
+    W_r = np.full(R, int(W_S), np.int32) if np.isscalar(W_S) else _arr(W_S, np.int32)
+    if out_off is None:
+        out_off = np.concatenate([[0], np.cumsum(W_r)])
+    out_off = _arr(out_off, np.int32)
+    z = _arr(logits_q, np.float32)
+    assert z.ndim == 2 and z.shape[0] == rbo[-1]
+    s = _arr(beam_logq, np.float64)
+    slots = int(out_off[-1])
+    res = dict(out_off=out_off, out_parent=np.full(slots, -1, np.int32), out_token=np.full(slots, -1, np.int32),
+               out_logq=np.zeros(slots), cdf_lo=np.zeros(slots), cdf_hi=np.zeros(slots),
+               error=np.zeros(R, np.int32))
+    inj, stride = None, 0
+    if inject_u is not None:
+        inj = _arr(inject_u, np.float64).reshape(R, -1)
+        stride = inj.shape[1]
+    rc = lib().dsbd_oracle_draft_layer(
+        C.c_int32(R), _p(rbo, _i32p), C.byref(p), C.c_int32(int(layer)), _p(W_r, _i32p), C.c_int32(0),
+        _p(z, _f32p), C.c_int64(z.shape[1]), _p(s, _f64p), _p(inj, _f64p), C.c_int64(stride),
+        _p(out_off, _i32p), _p(res["out_parent"], _i32p), _p(res["out_token"], _i32p),
+        _p(res["out_logq"], _f64p), _p(res["cdf_lo"], _f64p), _p(res["cdf_hi"], _f64p), _p(res["error"], _i32p))
+    if rc:
+        raise RuntimeError("dsbd_oracle_draft_layer: %d" % rc)
+    return res

@@ -693,3 +693,60 @@ int dsbd_oracle_select_width(const dsbd_oracle_forest *f, const dsbd_oracle_para
     free(lse_p); free(lse_q);
     return 0;
 }
+
+/* ------------------------------------------------------------------ draft stage ------ */
+/* One step of the small model's beam sampling (Section "Overview": beam sampling of width W_S
+ * for gamma steps; Section "Details": every draft beam is a sample of
+ * q_beam = T o (q / Q) over (current beams x V)).  Request r owns the current beams
+ * req_beam_off[r] .. req_beam_off[r+1]) with cumulative scores beam_logq and logits rows
+ * logits_q; it draws W_S iid cells by inverse CDF in canonical order, draw k with the uniform
+ * of (request, layer 2^29 + layer, purpose 3, index k).  Outputs per draw: the beam it extends
+ * (global index), the token, the new cumulative score; optional cdf_lo / cdf_hi (the cell's CDF
+ * interval, for near-tie accounting). */
+int dsbd_oracle_draft_layer(int32_t R, const int32_t *req_beam_off, const dsbd_oracle_params *prm,
+                            int32_t layer, const int32_t *W_S_r, int32_t W_S,
+                            const float *logits_q, int64_t row_stride, const double *beam_logq,
+                            const double *inject_u, int64_t inject_stride,
+                            const int32_t *out_off, int32_t *out_parent, int32_t *out_token,
+                            double *out_logq, double *cdf_lo, double *cdf_hi, int32_t *error)
+{
+    if (prm->V <= 0 || !(prm->temperature > 0.0) || row_stride < prm->V) return DSBD_O_ERR_BAD_FOREST;
+    const int32_t V = prm->V;
+    const double tau = prm->temperature;
+    for (int32_t r = 0; r < R; ++r) {
+        const int32_t b0 = req_beam_off[r], nA = req_beam_off[r + 1] - b0;
+        const int32_t W = W_S_r ? W_S_r[r] : W_S;
+        const uint32_t rid = prm->req_id ? (uint32_t)prm->req_id[r] : (uint32_t)r;
+        error[r] = 0;
+        if (nA <= 0) { if (W > 0) error[r] = DSBD_O_ERR_EXHAUSTED; continue; }
+        if (out_off[r + 1] - out_off[r] < W) { error[r] = DSBD_O_ERR_CAPACITY; continue; }
+        const int64_t cells = (int64_t)nA * V;
+        int32_t *A = (int32_t *)malloc(sizeof(int32_t) * (size_t)nA);
+        double *lse = (double *)malloc(sizeof(double) * (size_t)(b0 + nA));
+        double *q_beam = (double *)malloc(sizeof(double) * (size_t)cells);
+        for (int32_t i = 0; i < nA; ++i) {
+            A[i] = b0 + i;
+            lse[b0 + i] = row_lse(logits_q + (int64_t)(b0 + i) * row_stride, V, tau);
+        }
+        beam_distribution(logits_q, row_stride, V, tau, A, nA, beam_logq, lse, q_beam);
+        if (prm->top_k > 0 || (prm->top_p > 0.0 && prm->top_p < 1.0))
+            dsbd_oracle_warp(q_beam, cells, prm->top_k, prm->top_p, NULL, NULL);
+        for (int32_t k = 0; k < W; ++k) {
+            double u;
+            if (inject_u) u = k < inject_stride ? inject_u[(int64_t)r * inject_stride + k] : 0.5;
+            else u = dsbd_oracle_uniform(prm->seed, prm->step, rid, (1u << 29) + (uint32_t)layer, 3u, (uint32_t)k);
+            double lo = 0, hi = 0, z = 0;
+            const int64_t cell = draw_cell(q_beam, cells, u, &lo, &hi, &z);
+            if (cell < 0) { error[r] = DSBD_O_ERR_EXHAUSTED; break; }
+            const int32_t a = A[cell / V], tok = (int32_t)(cell % V);
+            const int64_t s = out_off[r] + k;
+            out_parent[s] = a;
+            out_token[s] = tok;
+            out_logq[s] = beam_logq[a] + ((double)logits_q[(int64_t)a * row_stride + tok] / tau - lse[a]);
+            if (cdf_lo) cdf_lo[s] = lo;
+            if (cdf_hi) cdf_hi[s] = hi;
+        }
+        free(A); free(lse); free(q_beam);
+    }
+    return 0;
+}

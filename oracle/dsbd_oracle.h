@@ -170,6 +170,19 @@ int dsbd_oracle_select_width(const dsbd_oracle_forest *f, const dsbd_oracle_para
                              const int32_t *m, int32_t *width, double *alpha, double *tail,
                              int32_t alpha_stride);
 
+/* One step of the small model's beam sampling (Sections "Overview" and "Details"): request r
+ * draws W_S (W_S_r[r] when given) iid cells from q_beam = T o (q / Q) over its current beams
+ * req_beam_off[r] .. req_beam_off[r+1]) x V, draw k with the uniform of (request, layer
+ * 2^29 + layer, purpose 3, index k) or inject_u[r*inject_stride + k].  Per draw, in slot
+ * out_off[r] + k: the beam it extends (global index), the token, the new cumulative score, and
+ * optionally the cell's CDF interval.  error: [R]. */
+int dsbd_oracle_draft_layer(int32_t R, const int32_t *req_beam_off, const dsbd_oracle_params *prm,
+                            int32_t layer, const int32_t *W_S_r, int32_t W_S,
+                            const float *logits_q, int64_t row_stride, const double *beam_logq,
+                            const double *inject_u, int64_t inject_stride,
+                            const int32_t *out_off, int32_t *out_parent, int32_t *out_token,
+                            double *out_logq, double *cdf_lo, double *cdf_hi, int32_t *error);
+
 #ifdef __cplusplus
 }
 #endif
