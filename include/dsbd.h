@@ -242,6 +242,41 @@ int dsbd_select_width(const dsbd_forest_t *forest, const dsbd_verify_params_t *p
                       void *workspace, size_t workspace_bytes, int32_t *status,
                       dsbd_stream_t stream);
 
+/* One step of the draft stage (Section "Overview": the small model performs beam sampling of
+ * width W_S for gamma steps; Section "Details": every draft beam is a sample of
+ * q_beam = T o (q / Q) over (current beams x V)).  Request r owns the current beams
+ * req_beam_off[r] .. req_beam_off[r+1]) -- the input beams for the first draft layer, the W_S
+ * beams of the previous layer afterwards -- with cumulative scores beam_logq [n_beams] and
+ * next-token logits logits_q [n_beams rows, row_stride].  It draws W_S (W_S_r[r] when given) iid
+ * cells by inverse CDF in canonical order (beam ascending, token ascending); draw k uses the
+ * Philox uniform of (request r, layer number 2^29 + layer, purpose 3, index k), so the stream is
+ * disjoint from the verification's.  Draw k lands in slot out_off[r] + k: out_parent (global
+ * index of the beam it extends), out_token, out_logq (new cumulative score); k is the node's
+ * draft_rank.  temperature, top_k and top_p act as in dsbd_verify_params_t.
+ * All pointers device except params; req_error [R] optional.  Host facts: n_slots = out_off[R],
+ * max_req_beams <= DSBD_MAX_LIVE.  *status / req_error: DSBD_DEV_CAPACITY when a slot range is
+ * shorter than W_S, DSBD_DEV_EXHAUSTED for a request without beams. */
+typedef struct {
+    int32_t V;
+    float temperature;
+    int32_t W_S;
+    const int32_t *W_S_r;          /* optional [R], device                                   */
+    uint64_t seed, step;
+    int32_t layer;                 /* draft layer 1..gamma this call samples                  */
+    int32_t top_k;
+    float top_p;
+    int32_t n_slots;
+    int32_t max_req_beams;
+} dsbd_draft_params_t;
+
+int dsbd_draft_layer(int32_t R, int32_t n_beams, const int32_t *req_beam_off,
+                     const dsbd_draft_params_t *params, const float *logits_q, int64_t row_stride,
+                     const float *beam_logq, const int32_t *out_off, int32_t *out_parent,
+                     int32_t *out_token, float *out_logq, int32_t *req_error, void *workspace,
+                     size_t workspace_bytes, int32_t *status, dsbd_stream_t stream);
+
+size_t dsbd_draft_workspace(int32_t R, int32_t n_beams, const dsbd_draft_params_t *params);
+
 /* KV-cache update at the end of a decode step (Section "Forest-based Parallel Decoding": after
  * the iteration the key-value caches are updated according to the output beams, an output beam
  * keeping the cache of the input beam it descends from; Section "Reducing Memory Cost": keeping

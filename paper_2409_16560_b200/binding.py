@@ -21,7 +21,8 @@ MAX_LIVE = 64
 
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
-           "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_status_string"]
+           "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_draft_layer", "dsbd_draft_workspace",
+           "dsbd_status_string"]
 
 _vp = C.c_void_p
 
@@ -95,6 +96,11 @@ def load():
     lib.dsbd_kv_commit_workspace.argtypes = [_vp, _vp]
     lib.dsbd_kv_commit.restype = C.c_int
     lib.dsbd_kv_commit.argtypes = [_vp] * 19 + [C.c_size_t, _vp, _vp]
+    lib.dsbd_draft_workspace.restype = C.c_size_t
+    lib.dsbd_draft_workspace.argtypes = [C.c_int32, C.c_int32, _vp]
+    lib.dsbd_draft_layer.restype = C.c_int
+    lib.dsbd_draft_layer.argtypes = [C.c_int32, C.c_int32, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, _vp,
+                                     _vp, C.c_size_t, _vp, _vp]
     _lib = lib
     return lib
 
@@ -214,6 +220,54 @@ def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_pre
     if rc != OK:
         raise DsbdError("dsbd_forest_attention", rc)
     return out, status
+
+
+class DraftParamsT(C.Structure):
+    _fields_ = [("V", C.c_int32), ("temperature", C.c_float), ("W_S", C.c_int32), ("W_S_r", _vp),
+                ("seed", C.c_uint64), ("step", C.c_uint64), ("layer", C.c_int32), ("top_k", C.c_int32),
+                ("top_p", C.c_float), ("n_slots", C.c_int32), ("max_req_beams", C.c_int32)]
+
+
+def draft_layer(req_beam_off, req_beam_off_host, params, layer, W_S, logits_q, beam_logq, out_off, n_slots,
+                row_stride=None, workspace=None, status=None, stream=None):
+    """dsbd_draft_layer.  req_beam_off, out_off: int32 device tensors; W_S: int or int32 device
+    tensor [R]; params: V, temperature, seed, step, top_k, top_p.  Returns dict(out_parent,
+    out_token, out_logq, req_error, status) on the device."""
+    _require_cuda(req_beam_off, logits_q, beam_logq, out_off)
+    assert logits_q.dtype == torch.float32 and beam_logq.dtype == torch.float32
+    dev = logits_q.device
+    rbo = np.asarray(req_beam_off_host)
+    R, n_beams = len(rbo) - 1, int(rbo[-1])
+    p = DraftParamsT()
+    p.V = int(params["V"])
+    p.temperature = float(params.get("temperature", 1.0))
+    if torch.is_tensor(W_S):
+        _require_cuda(W_S)
+        assert W_S.dtype == torch.int32
+        p.W_S, p.W_S_r = 0, _ptr(W_S)
+    else:
+        p.W_S = int(W_S)
+    p.seed, p.step, p.layer = int(params.get("seed", 0)), int(params.get("step", 0)), int(layer)
+    p.top_k, p.top_p = int(params.get("top_k", 0)), float(params.get("top_p", 1.0))
+    p.n_slots = int(n_slots)
+    p.max_req_beams = int(np.diff(rbo).max())
+    need = int(load().dsbd_draft_workspace(R, n_beams, C.addressof(p)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    res = dict(out_parent=torch.full((int(n_slots),), -1, dtype=torch.int32, device=dev),
+               out_token=torch.full((int(n_slots),), -1, dtype=torch.int32, device=dev),
+               out_logq=torch.zeros(int(n_slots), dtype=torch.float32, device=dev),
+               req_error=torch.zeros(R, dtype=torch.int32, device=dev), status=status, workspace=workspace)
+    stride = int(row_stride) if row_stride is not None else int(logits_q.stride(0))
+    rc = load().dsbd_draft_layer(R, n_beams, _ptr(req_beam_off), C.addressof(p), _ptr(logits_q), stride,
+                                 _ptr(beam_logq), _ptr(out_off), _ptr(res["out_parent"]), _ptr(res["out_token"]),
+                                 _ptr(res["out_logq"]), _ptr(res["req_error"]), _ptr(workspace), workspace.numel(),
+                                 _ptr(status), _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_draft_layer", rc)
+    return res
 
 
 class CommitParamsT(C.Structure):

@@ -88,12 +88,14 @@ __device__ __forceinline__ void load_half_tile(const float *__restrict__ row, in
 __global__ void __launch_bounds__(kThreads)
 k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t stride, int V,
              int T, int N, int n_rows, const int32_t *__restrict__ rows,
-             const int32_t *__restrict__ n_rows_dev, float k2, TileStat *__restrict__ stats) {
+             const int32_t *__restrict__ n_rows_dev, float k2, TileStat *__restrict__ stats,
+             int one_model = 0) {
+    // one_model: zq is the same tensor as zp; read it once and store the statistics for both
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     if (n_rows_dev) n_rows = *n_rows_dev;
-    const int64_t total = (int64_t)2 * n_rows * T;
+    const int64_t total = (int64_t)(one_model ? 1 : 2) * n_rows * T;
     for (int64_t item = warp; item < total; item += nwarps) {
         const int t = (int)(item % T);
         const int64_t rm = item / T;
@@ -122,6 +124,7 @@ k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t
         if (lane == 0) {
             TileStat s; s.mx = mx; s.sum = sum;
             stats[((int64_t)model * N + row) * T + t] = s;
+            if (one_model) stats[((int64_t)N + row) * T + t] = s;
         }
     }
 }
@@ -187,6 +190,7 @@ struct VerifyArgs {
     int32_t *depth_w;
     const float *root_logp, *root_logq;
     int max_m, max_live;
+    uint32_t extra_layer_bias;   // added to the layer number in the Philox counter of the extra layer
     // outputs
     dsbd_verify_out_t out;
     int32_t *status;
@@ -1356,7 +1360,8 @@ k_verify(VerifyArgs a) {
         int err = extra_err;
         if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
         for (int kk = 0; kk < W_nom && !err; ++kk) {
-            const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1), 3u, (uint32_t)kk);
+            const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1) + a.extra_layer_bias, 3u,
+                                              (uint32_t)kk);
             int ia = 0, tok;
             if (a.top_k > 0) {
                 int pick = -1;
@@ -1567,6 +1572,131 @@ extern "C" int dsbd_node_stats(const dsbd_forest_t *f, const dsbd_verify_params_
     k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
         stats, L.T, f->N, f->N, nullptr, nullptr, inv_tau, lse, lse_p, lse_q);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------
+// dsbd_draft_layer: a beam-sampling step of the small model is the "extra layer" of the
+// verification kernel on a forest that has only roots (the current beams), with the small
+// model's logits standing for both models: W_S inverse-CDF draws from T o q_beam.
+// ---------------------------------------------------------------------------------------
+namespace {
+__global__ void k_draft_init(int n_beams, int32_t *beam_node_off, int32_t *parent) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i <= n_beams) beam_node_off[i] = i;
+    if (i < n_beams) parent[i] = -1;
+}
+
+struct DraftLayout {
+    Layout v;
+    size_t beam_node_off, parent, l_last, out_width, layer_width, node_status, out_node, out_root_beam,
+        out_source, out_logp, total;
+};
+
+dsbd_forest_t draft_forest(int R, int n_beams, const dsbd_draft_params_t *p) {
+    dsbd_forest_t f = {};
+    f.R = R; f.B = n_beams; f.N = n_beams; f.max_depth = 0;
+    f.max_tree_nodes = 1; f.max_req_beams = p->max_req_beams; f.max_layer_nodes = 0;
+    return f;
+}
+
+bool draft_args_ok(int R, int n_beams, const dsbd_draft_params_t *p) {
+    return p && R > 0 && n_beams > 0 && p->V > 0 && p->temperature > 0.f && p->n_slots > 0 &&
+           p->max_req_beams > 0 && (p->W_S >= 0 || p->W_S_r) && p->layer >= 0 && p->top_k >= 0;
+}
+
+DraftLayout make_draft_layout(int R, int n_beams, const dsbd_draft_params_t *p) {
+    DraftLayout D;
+    const dsbd_forest_t f = draft_forest(R, n_beams, p);
+    D.v = make_layout(&f, p->V);
+    size_t off = D.v.total;
+    auto take = [&](size_t bytes) { const size_t at = off; off = align_up(off + bytes, 256); return at; };
+    D.beam_node_off = take(sizeof(int32_t) * ((size_t)n_beams + 1));
+    D.parent = take(sizeof(int32_t) * (size_t)n_beams);
+    D.l_last = take(sizeof(int32_t) * (size_t)R);
+    D.out_width = take(sizeof(int32_t) * (size_t)R);
+    D.layer_width = take(sizeof(int32_t) * (size_t)R);
+    D.node_status = take((size_t)n_beams);
+    D.out_node = take(sizeof(int32_t) * (size_t)p->n_slots);
+    D.out_root_beam = take(sizeof(int32_t) * (size_t)p->n_slots);
+    D.out_source = take(sizeof(int32_t) * (size_t)p->n_slots);
+    D.out_logp = take(sizeof(float) * (size_t)p->n_slots);
+    D.total = off;
+    return D;
+}
+}  // namespace
+
+extern "C" size_t dsbd_draft_workspace(int32_t R, int32_t n_beams, const dsbd_draft_params_t *p) {
+    if (!draft_args_ok(R, n_beams, p)) return 0;
+    return make_draft_layout(R, n_beams, p).total;
+}
+
+extern "C" int dsbd_draft_layer(int32_t R, int32_t n_beams, const int32_t *req_beam_off,
+                                const dsbd_draft_params_t *p, const float *logits_q, int64_t row_stride,
+                                const float *beam_logq, const int32_t *out_off, int32_t *out_parent,
+                                int32_t *out_token, float *out_logq, int32_t *req_error, void *workspace,
+                                size_t workspace_bytes, int32_t *status, dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    if (!draft_args_ok(R, n_beams, p)) return DSBD_ERR_INVALID_ARG;
+    if (!req_beam_off || !logits_q || !beam_logq || !out_off || !out_parent || !out_token || !out_logq ||
+        !workspace || !status || row_stride < p->V)
+        return DSBD_ERR_INVALID_ARG;
+    if (p->max_req_beams > DSBD_MAX_LIVE || p->top_k > 64) return DSBD_ERR_UNSUPPORTED;
+    if (p->top_k == 0 && p->top_p > 0.f && p->top_p < 1.f) return DSBD_ERR_UNSUPPORTED;
+    const DraftLayout D = make_draft_layout(R, n_beams, p);
+    if (workspace_bytes < D.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+    const Layout &L = D.v;
+    TileStat *stats = reinterpret_cast<TileStat *>(ws + L.stats);
+    double *lse = reinterpret_cast<double *>(ws + L.lse);
+    double *score = reinterpret_cast<double *>(ws + L.score);
+    int32_t *depth = reinterpret_cast<int32_t *>(ws + L.depth);
+    int32_t *beam_node_off = reinterpret_cast<int32_t *>(ws + D.beam_node_off);
+    int32_t *parent = reinterpret_cast<int32_t *>(ws + D.parent);
+    const double inv_tau = 1.0 / (double)p->temperature;
+    const float k2 = (float)((double)kLog2e * inv_tau);
+
+    k_draft_init<<<(n_beams + 1 + 255) / 256, 256, 0, stream>>>(n_beams, beam_node_off, parent);
+    const int64_t items = (int64_t)n_beams * L.T;
+    k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_q, logits_q, row_stride, p->V, L.T, n_beams,
+                                                            n_beams, nullptr, nullptr, k2, stats, 1);
+    if (cudaGetLastError() != cudaSuccess) return DSBD_ERR_CUDA;
+
+    VerifyArgs a = {};
+    a.R = R; a.N = n_beams; a.gamma = 0;
+    a.req_beam_off = req_beam_off; a.beam_node_off = beam_node_off; a.parent = parent;
+    a.token = nullptr; a.draft_rank = nullptr;
+    a.V = p->V; a.T = L.T; a.k2 = k2; a.inv_tau = inv_tau; a.thresh = 0.5;
+    a.W_min = 1; a.W_max = 1; a.W_nom = p->W_S; a.W_nom_r = p->W_S_r;
+    a.seed = p->seed; a.step = p->step;
+    a.top_k = p->top_k; a.top_p = (double)p->top_p;
+    a.zp = logits_q; a.zq = logits_q; a.stride = row_stride;
+    a.stats = stats; a.lse = lse; a.score = score; a.depth = depth;
+    a.tile_sums = reinterpret_cast<double *>(ws + L.sums);
+    a.max_m = L.max_m; a.max_live = L.max_live;
+    a.hist = reinterpret_cast<unsigned long long *>(ws + L.hist);
+#ifdef DSBD_PHASE_TIMING
+    a.dbg = reinterpret_cast<unsigned long long *>(ws + L.total) - (size_t)R * 256;
+#endif
+    a.extra_layer_bias = (1u << 29) + (uint32_t)p->layer - 1u;     // layer number 2^29 + layer
+    a.out = dsbd_verify_out_t{};
+    a.out.l_last = reinterpret_cast<int32_t *>(ws + D.l_last);
+    a.out.out_width = reinterpret_cast<int32_t *>(ws + D.out_width);
+    a.out.out_off = out_off;
+    a.out.out_parent = out_parent;
+    a.out.out_node = reinterpret_cast<int32_t *>(ws + D.out_node);
+    a.out.out_root_beam = reinterpret_cast<int32_t *>(ws + D.out_root_beam);
+    a.out.out_token = out_token;
+    a.out.out_logp = reinterpret_cast<float *>(ws + D.out_logp);
+    a.out.out_logq = out_logq;
+    a.out.out_source = reinterpret_cast<int32_t *>(ws + D.out_source);
+    a.out.node_status = reinterpret_cast<int8_t *>(ws + D.node_status);
+    a.out.layer_width = reinterpret_cast<int32_t *>(ws + D.layer_width);
+    a.out.req_error = req_error;
+    a.status = status; a.select_mode = 0;
+    a.lse_w = lse; a.score_w = score; a.depth_w = depth;
+    a.root_logp = beam_logq; a.root_logq = beam_logq;
+    return launch_verify(a, R, L.max_live * L.T, stream);
 }
 
 // ---------------------------------------------------------------------------------------
