@@ -373,6 +373,30 @@ def main():
     assert int(status.item()) == 0, "device status %d" % int(status.item())
     del k_dst, v_dst
 
+    # one draft-stage sampling step of the same shape (W_S = beams of the request), reported
+    # beside the step: the small model's logits of the first B rows stand for a draft layer
+    rbo_host = np.asarray(forest["req_beam_off"], dtype=np.int32)
+    W_S_r = torch.as_tensor(np.diff(rbo_host).astype(np.int32)).to(dev)
+    rbo_dev = torch.as_tensor(rbo_host).to(dev)
+    zq_rows = data["logits_q"][:f.B]
+    draft = None
+
+    def draft_layer():
+        return dsbd.draft_layer(rbo_dev, rbo_host, prm, 1, W_S_r, zq_rows, data["root_logq"], rbo_dev, f.B,
+                                workspace=draft["workspace"] if draft else None, status=status, stream=stream)
+    for _ in range(3):
+        draft = draft_layer()
+    g0 = torch.cuda.Event(enable_timing=True); g1 = torch.cuda.Event(enable_timing=True)
+    n_draft = max(args.steps, 5)
+    g0.record(stream)
+    for _ in range(n_draft):
+        draft_layer()
+    g1.record(stream)
+    torch.cuda.synchronize()
+    draft_ms = g0.elapsed_time(g1) / n_draft
+    draft_bytes = 4 * f.B * spec["V"]
+    assert int(status.item()) == 0, "device status %d" % int(status.item())
+
     # end to end through the C ABI with host buffers
     e2e = None
     if args.e2e_steps > 0:
@@ -424,6 +448,7 @@ def main():
         "verify_dense_pass": {"bytes": v_bytes, "ms": dense_ms, "gbs": v_bytes / dense_ms * 1e-6},
         "verify_step_total": {"bytes": v_bytes, "ms": ver_ms, "gbs": v_bytes / ver_ms * 1e-6},
         "kv_commit": {"bytes": commit_bytes, "ms": commit_ms, "gbs": commit_bytes / commit_ms * 1e-6},
+        "draft_layer": {"bytes": draft_bytes, "ms": draft_ms, "gbs": draft_bytes / draft_ms * 1e-6},
     }
     for k in kernels.values():
         k["frac_of_%s_peak" % peak_kind] = k["gbs"] / peak
