@@ -111,6 +111,29 @@ size_t dsbd_forest_attention_workspace(const dsbd_forest_t *forest, const dsbd_a
  * arguments.  For launch accounting; host-only. */
 int dsbd_forest_attention_launches(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc);
 
+/* The same attention over PAGED caches.  The paper keeps one key-value cache per input beam and
+ * does not say how it is stored; here a cache may be a list of pages of DSBD_PAGE_TOKENS tokens
+ * in a pool, so that beams descending from one input beam share its pages and the cache update
+ * (dsbd_kv_commit_paged) copies no prefix.  k_pool, v_pool: [n_pages, Hkv, DSBD_PAGE_TOKENS, d];
+ * beam b owns the pages page_table[page_off[b] .. page_off[b+1]) in token order, ceil(L_b /
+ * DSBD_PAGE_TOKENS) of them, L_b = prefix_off[b+1] - prefix_off[b] (prefix_off only carries the
+ * lengths here; desc->total_prefix / max_prefix as before).  Rows of a last page past L_b are
+ * never used but must hold finite values.  Supported: bf16, d = 128 (the tensor-core kernel);
+ * otherwise UNSUPPORTED.  Workspace: dsbd_forest_attention_workspace. */
+enum { DSBD_PAGE_TOKENS = 64 };
+
+typedef struct {
+    const int32_t *page_table;     /* device                                                 */
+    const int64_t *page_off;       /* device [B+1]                                           */
+    int64_t n_pages;               /* host: pages in the pool                                */
+} dsbd_kv_pages_t;
+
+int dsbd_forest_attention_paged(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
+                                const void *q, const void *k_new, const void *v_new,
+                                const void *k_pool, const void *v_pool, const dsbd_kv_pages_t *pages,
+                                const int64_t *prefix_off, void *out, void *workspace,
+                                size_t workspace_bytes, int32_t *status, dsbd_stream_t stream);
+
 /* Parameters of the verification (Section "Details", Algorithm 1, and Section
  * "Dynamic-Width Speculative Beam Decoding"). */
 typedef struct {

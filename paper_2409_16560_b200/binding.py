@@ -22,6 +22,7 @@ MAX_LIVE = 64
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
            "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_draft_layer", "dsbd_draft_workspace",
+           "dsbd_forest_attention_paged",
            "dsbd_status_string"]
 
 _vp = C.c_void_p
@@ -96,6 +97,8 @@ def load():
     lib.dsbd_kv_commit_workspace.argtypes = [_vp, _vp]
     lib.dsbd_kv_commit.restype = C.c_int
     lib.dsbd_kv_commit.argtypes = [_vp] * 19 + [C.c_size_t, _vp, _vp]
+    lib.dsbd_forest_attention_paged.restype = C.c_int
+    lib.dsbd_forest_attention_paged.argtypes = [_vp] * 11 + [C.c_size_t, _vp, _vp]
     lib.dsbd_draft_workspace.restype = C.c_size_t
     lib.dsbd_draft_workspace.argtypes = [C.c_int32, C.c_int32, _vp]
     lib.dsbd_draft_layer.restype = C.c_int
@@ -219,6 +222,35 @@ def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_pre
                                       _ptr(workspace), workspace.numel(), _ptr(status), _stream(stream))
     if rc != OK:
         raise DsbdError("dsbd_forest_attention", rc)
+    return out, status
+
+
+class KvPagesT(C.Structure):
+    _fields_ = [("page_table", _vp), ("page_off", _vp), ("n_pages", C.c_int64)]
+
+
+def forest_attention_paged(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_pool, v_pool, page_table, page_off,
+                           prefix_off, prefix_off_host, out=None, workspace=None, status=None, stream=None):
+    """dsbd_forest_attention_paged; k_pool / v_pool: [n_pages, Hkv, 64, d]; returns (out, status)."""
+    _require_cuda(q, k_new, v_new, k_pool, v_pool, page_table, page_off, prefix_off)
+    assert page_table.dtype == torch.int32 and page_off.dtype == torch.int64
+    f = forest.struct()
+    desc = _attn_desc(Hq, Hkv, d, q.dtype, scale, prefix_off_host)
+    pages = KvPagesT()
+    pages.page_table, pages.page_off, pages.n_pages = _ptr(page_table), _ptr(page_off), int(k_pool.shape[0])
+    if out is None:
+        out = torch.empty_like(q)
+    need = int(load().dsbd_forest_attention_workspace(C.addressof(f), C.addressof(desc)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=q.device)
+    rc = load().dsbd_forest_attention_paged(C.addressof(f), C.addressof(desc), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                            _ptr(k_pool), _ptr(v_pool), C.addressof(pages), _ptr(prefix_off),
+                                            _ptr(out), _ptr(workspace), workspace.numel(), _ptr(status),
+                                            _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_forest_attention_paged", rc)
     return out, status
 
 

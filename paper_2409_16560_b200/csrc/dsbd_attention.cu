@@ -267,3 +267,24 @@ extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_des
     return d->d == 64 ? launch_simt<__nv_bfloat16, 64>(a, units, stream)
                       : launch_simt<__nv_bfloat16, 128>(a, units, stream);
 }
+
+extern "C" int dsbd_forest_attention_paged(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q,
+                                           const void *k_new, const void *v_new, const void *k_pool,
+                                           const void *v_pool, const dsbd_kv_pages_t *pages,
+                                           const int64_t *prefix_off, void *out, void *workspace,
+                                           size_t workspace_bytes, int32_t *status, dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    const int rc = check(f, d);
+    if (rc) return rc;
+    if (!q || !k_new || !v_new || !k_pool || !v_pool || !pages || !pages->page_table || !pages->page_off ||
+        pages->n_pages <= 0 || !prefix_off || !out || !status)
+        return DSBD_ERR_INVALID_ARG;
+    if (!attention_tc_supported(f, d, pages->n_pages)) return DSBD_ERR_UNSUPPORTED;
+    if (workspace_bytes < attention_tc_workspace(f, d) || !workspace) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) |
+                           reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(k_pool) |
+                           reinterpret_cast<uintptr_t>(v_pool) | reinterpret_cast<uintptr_t>(out);
+    if (bits & 15) return DSBD_ERR_UNSUPPORTED;
+    return launch_attention_tc(f, d, q, k_new, v_new, k_pool, v_pool, prefix_off, out, workspace, workspace_bytes,
+                               status, stream, pages);
+}

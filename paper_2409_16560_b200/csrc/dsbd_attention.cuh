@@ -6,8 +6,9 @@
 namespace dsbd {
 
 // True when the tcgen05 kernel covers this problem (bf16, d = 128, at most 128 query rows and
-// 64 nodes per tree, a non-empty KV prefix).
-bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
+// 64 nodes per tree, a non-empty KV prefix).  n_pages > 0: the caches are paged (k_prefix /
+// v_prefix are then the page pools).
+bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages = 0);
 
 // Workspace bytes of the tensor-core path (work plan and partial results of split units).
 size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
@@ -17,6 +18,7 @@ int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
 
 int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
                         const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
-                        void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream);
+                        void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream,
+                        const dsbd_kv_pages_t *pages = nullptr);
 
 }  // namespace dsbd

@@ -63,6 +63,8 @@ struct TcArgs {
     float scale_log2;
     const int32_t *beam_node_off, *parent;
     const int64_t *prefix_off;
+    const int32_t *page_table;        // paged caches: page ids of beam b at page_off[b] ..; nullptr: packed
+    const int64_t *page_off;
     const __nv_bfloat16 *q;
     __nv_bfloat16 *out;
     int32_t *status;
@@ -236,6 +238,9 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 const int b = item.b, g = item.g;
                 const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
                 const int64_t row0 = a.prefix_off[b] * a.Hkv + (int64_t)g * L + item.t0;
+                // paged: tile j of the item is page t0/64 + j of the beam, one 64-row box of the pool
+                const int32_t *pages = a.page_table ? a.page_table + a.page_off[b] + item.t0 / kBN : nullptr;
+                int page_next = (pages && item.t1 > item.t0) ? pages[0] : 0;
                 const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
                 const int n_lo = a.beam_node_off[b];
                 const int nt = nt_p + item.last;
@@ -247,7 +252,11 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     unsigned char *ks = stage_s + s * kStageBytes, *vs = ks + kTileBytes;
                     mbar_expect_tx(&sb.kv_full[s], kStageBytes);
                     if (j < nt_p) {
-                        const int y = (int)(row0 + (int64_t)j * kBN);
+                        int y = (int)(row0 + (int64_t)j * kBN);
+                        if (pages) {
+                            y = (page_next * a.Hkv + g) * kBN;
+                            if (j + 1 < nt_p) page_next = pages[j + 1];
+                        }
                         tma_load_2d(ks, &map_kp, 0, y, &sb.kv_full[s]);
                         tma_load_2d(ks + kTileBytes / 2, &map_kp, 64, y, &sb.kv_full[s]);
                         tma_load_2d(vs, &map_vp, 0, y, &sb.kv_full[s]);
@@ -702,12 +711,14 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
 
 namespace dsbd {
 
-bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages) {
     if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
     if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows) return false;
     if (f->max_tree_nodes > kBN) return false;
     if (d->total_prefix <= 0) return false;
-    if ((int64_t)d->total_prefix * d->Hkv >= (int64_t)1 << 31) return false;
+    // row coordinates of the K/V maps are 32-bit
+    const int64_t rows = n_pages > 0 ? n_pages * d->Hkv * kBN : (int64_t)d->total_prefix * d->Hkv;
+    if (rows >= (int64_t)1 << 31) return false;
     return encode_fn() != nullptr;
 }
 
@@ -720,9 +731,10 @@ int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
 
 int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
                         const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
-                        void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream) {
+                        void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream,
+                        const dsbd_kv_pages_t *pages) {
     CUtensorMap kp, vp, kn, vn;
-    const uint64_t prows = (uint64_t)d->total_prefix * d->Hkv;
+    const uint64_t prows = pages ? (uint64_t)pages->n_pages * d->Hkv * kBN : (uint64_t)d->total_prefix * d->Hkv;
     if (!make_map(&kp, k_prefix, kD, prows, kD * 2) || !make_map(&vp, v_prefix, kD, prows, kD * 2) ||
         !make_map(&kn, k_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2) ||
         !make_map(&vn, v_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2))
@@ -736,6 +748,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.max_rows = f->max_tree_nodes * a.group;
     a.scale_log2 = d->scale * 1.4426950408889634f;
     a.beam_node_off = f->beam_node_off; a.parent = f->parent; a.prefix_off = prefix_off;
+    if (pages) { a.page_table = pages->page_table; a.page_off = pages->page_off; }
     a.q = static_cast<const __nv_bfloat16 *>(q);
     a.out = static_cast<__nv_bfloat16 *>(out);
     a.status = status;
