@@ -341,6 +341,34 @@ int dsbd_kv_commit(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
 
 size_t dsbd_kv_commit_workspace(const dsbd_forest_t *forest, const dsbd_commit_params_t *params);
 
+/* The same update for PAGED caches (see dsbd_forest_attention_paged): nothing of a prefix is
+ * copied.  New beam j keeps the first L_b / DSBD_PAGE_TOKENS pages of its input beam b (shared),
+ * and gets ceil((L_b % DSBD_PAGE_TOKENS + path length) / DSBD_PAGE_TOKENS) fresh pages that
+ * receive b's partly filled last page, then the path's keys/values, then zeros.  Selection,
+ * numbering and keep_best as in dsbd_kv_commit.
+ * Allocator state (device, updated in place): free_stack [n_pages] and free_count [1]; the k-th
+ * fresh page of the call is free_stack[free_count - 1 - k], beams in order; afterwards the
+ * stack is rebuilt as every page that no new table names, ascending.  The pools are written
+ * only at fresh pages.  The old page_table / page_off / prefix_off are not modified.
+ * Outputs: new_req_beam_off [R+1], new_prefix_off [n_slots+1] (cumulative lengths), new_page_off
+ * [n_slots+1], new_page_table [params->dst_capacity entries], new_beam_slot [n_slots].
+ * *status: DSBD_DEV_CAPACITY when the tables need more than dst_capacity entries or the stack has
+ * too few free pages, DSBD_DEV_BAD_FOREST as in dsbd_kv_commit; then pools, tables and allocator
+ * stay as they were. */
+int dsbd_kv_commit_paged(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
+                         const dsbd_commit_params_t *params,
+                         const int32_t *out_off, const int32_t *out_width, const int32_t *out_parent,
+                         const int32_t *out_root_beam, const float *out_logp,
+                         const void *k_new, const void *v_new, void *k_pool, void *v_pool,
+                         const dsbd_kv_pages_t *pages, const int64_t *prefix_off,
+                         int32_t *free_stack, int32_t *free_count,
+                         int32_t *new_req_beam_off, int64_t *new_prefix_off, int64_t *new_page_off,
+                         int32_t *new_page_table, int32_t *new_beam_slot,
+                         void *workspace, size_t workspace_bytes, int32_t *status, dsbd_stream_t stream);
+
+size_t dsbd_kv_commit_paged_workspace(const dsbd_forest_t *forest, const dsbd_commit_params_t *params,
+                                      int64_t n_pages);
+
 const char *dsbd_status_string(int code);
 
 #ifdef __cplusplus

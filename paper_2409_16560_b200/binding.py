@@ -22,7 +22,7 @@ MAX_LIVE = 64
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
            "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_draft_layer", "dsbd_draft_workspace",
-           "dsbd_forest_attention_paged",
+           "dsbd_forest_attention_paged", "dsbd_kv_commit_paged", "dsbd_kv_commit_paged_workspace",
            "dsbd_status_string"]
 
 _vp = C.c_void_p
@@ -99,6 +99,10 @@ def load():
     lib.dsbd_kv_commit.argtypes = [_vp] * 19 + [C.c_size_t, _vp, _vp]
     lib.dsbd_forest_attention_paged.restype = C.c_int
     lib.dsbd_forest_attention_paged.argtypes = [_vp] * 11 + [C.c_size_t, _vp, _vp]
+    lib.dsbd_kv_commit_paged_workspace.restype = C.c_size_t
+    lib.dsbd_kv_commit_paged_workspace.argtypes = [_vp, _vp, C.c_int64]
+    lib.dsbd_kv_commit_paged.restype = C.c_int
+    lib.dsbd_kv_commit_paged.argtypes = [_vp] * 22 + [C.c_size_t, _vp, _vp]
     lib.dsbd_draft_workspace.restype = C.c_size_t
     lib.dsbd_draft_workspace.argtypes = [C.c_int32, C.c_int32, _vp]
     lib.dsbd_draft_layer.restype = C.c_int
@@ -339,6 +343,44 @@ def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out
         raise DsbdError("dsbd_kv_commit", rc)
     return dict(k_dst=k_dst, v_dst=v_dst, new_req_beam_off=new_req_beam_off, new_prefix_off=new_prefix_off,
                 new_beam_slot=new_beam_slot, status=status, workspace=workspace)
+
+
+def kv_commit_paged(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out_logp, k_new, v_new,
+                    k_pool, v_pool, page_table, page_off, prefix_off, prefix_off_host, free_stack, free_count,
+                    n_slots, table_capacity, keep_best=False, workspace=None, status=None, stream=None):
+    """dsbd_kv_commit_paged; the pools, free_stack and free_count are updated in place.  Returns a
+    dict with new_req_beam_off, new_prefix_off, new_page_off, new_page_table, new_beam_slot and the
+    status tensor (device tensors, nothing is synchronised)."""
+    _require_cuda(out_off, out_width, out_parent, out_root_beam, k_new, v_new, k_pool, v_pool, page_table,
+                  page_off, prefix_off, free_stack, free_count)
+    dev = k_new.device
+    f = forest.struct()
+    desc = _attn_desc(Hkv, Hkv, d, k_new.dtype, 1.0, prefix_off_host)
+    p = CommitParamsT()
+    p.n_slots, p.keep_best, p.dst_capacity = int(n_slots), int(bool(keep_best)), int(table_capacity)
+    pages = KvPagesT()
+    pages.page_table, pages.page_off, pages.n_pages = _ptr(page_table), _ptr(page_off), int(k_pool.shape[0])
+    need = int(load().dsbd_kv_commit_paged_workspace(C.addressof(f), C.addressof(p), pages.n_pages))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    res = dict(new_req_beam_off=torch.empty(forest.R + 1, dtype=torch.int32, device=dev),
+               new_prefix_off=torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev),
+               new_page_off=torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev),
+               new_page_table=torch.full((int(table_capacity),), -1, dtype=torch.int32, device=dev),
+               new_beam_slot=torch.empty(int(n_slots), dtype=torch.int32, device=dev),
+               status=status, workspace=workspace)
+    rc = load().dsbd_kv_commit_paged(
+        C.addressof(f), C.addressof(desc), C.addressof(p), _ptr(out_off), _ptr(out_width), _ptr(out_parent),
+        _ptr(out_root_beam), _ptr(out_logp) if out_logp is not None else None, _ptr(k_new), _ptr(v_new),
+        _ptr(k_pool), _ptr(v_pool), C.addressof(pages), _ptr(prefix_off), _ptr(free_stack), _ptr(free_count),
+        _ptr(res["new_req_beam_off"]), _ptr(res["new_prefix_off"]), _ptr(res["new_page_off"]),
+        _ptr(res["new_page_table"]), _ptr(res["new_beam_slot"]), _ptr(workspace), workspace.numel(), _ptr(status),
+        _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_kv_commit_paged", rc)
+    return res
 
 
 def _params(params, keep):

@@ -9,6 +9,13 @@
 //                   input beam's cache, then one row per path node -- cut into 128 KB chunks;
 //                   CTAs walk the chunk list with 128-bit loads kept out of L1 and streaming
 //                   stores.  HBM-bound: read + write of every kept cache once.
+//
+// Paged caches (pages of 64 tokens in a pool, see dsbd_forest_attention_paged) make the update
+// O(path) instead of O(prefix): a kept beam shares the full pages of its input beam and gets
+// fresh pages only for the input beam's last, partly filled page plus its path.
+//   k_commit_plan   (paged mode) also sizes the new page tables and the fresh pages
+//   k_commit_pages  writes the tables and fills the fresh pages
+//   k_commit_free   one CTA: rebuilds the free stack (every page no new table names)
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -18,6 +25,7 @@ namespace {
 using namespace dsbd;
 
 constexpr int kPlanThreads = 1024;
+constexpr int kPage = DSBD_PAGE_TOKENS;
 constexpr int kCopyThreads = 256;
 constexpr int kRoundBytes = 32768;                  // 8 x 16 B per thread in flight
 constexpr int kRounds = 4;
@@ -43,13 +51,22 @@ struct CommitArgs {
     unsigned char *k_dst, *v_dst;
     int32_t *new_req_beam_off, *new_beam_slot;
     int64_t *new_prefix_off;
+    // paged mode: k_prefix / v_prefix and k_dst / v_dst are the pools [n_pages, Hkv, 64, d]
+    int paged;
+    int64_t n_pages;
+    const int32_t *page_table;
+    const int64_t *page_off;
+    int32_t *new_page_table;
+    int64_t *new_page_off;
+    int32_t *free_stack, *free_count;
+    int32_t *used;            // [n_pages + 1] workspace
     // workspace
     Plan *plan;
     int32_t *req_count;       // [R]     kept beams of the request, then its first new beam
     int32_t *src_beam;        // [n_slots]
     int32_t *path;            // [n_slots][gamma+1] nodes root .. parent
     int32_t *path_len;        // [n_slots]
-    int64_t *chunk_off;       // [n_slots+1]
+    int64_t *chunk_off;       // [n_slots+1] copy chunks before each beam; paged: fresh pages before it
     int32_t *status;
 };
 
@@ -137,7 +154,14 @@ k_commit_plan(CommitArgs a) {
             a.new_beam_slot[j] = s;
             const int64_t len = (a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 1;
             a.new_prefix_off[j] = len;
-            a.chunk_off[j] = (len * a.row_bytes + kChunkBytes - 1) / kChunkBytes;
+            if (a.paged) {
+                const int64_t L_old = len - depth - 1;
+                const int64_t fresh = (L_old % kPage + depth + 1 + kPage - 1) / kPage;
+                a.chunk_off[j] = fresh;
+                a.new_page_off[j] = L_old / kPage + fresh;
+            } else {
+                a.chunk_off[j] = (len * a.row_bytes + kChunkBytes - 1) / kChunkBytes;
+            }
         }
     }
     __syncthreads();
@@ -149,15 +173,23 @@ k_commit_plan(CommitArgs a) {
         a.new_beam_slot[j] = -1;
         a.new_prefix_off[j] = 0;
         a.chunk_off[j] = 0;
+        if (a.paged) a.new_page_off[j] = 0;
     }
     __syncthreads();
     const int64_t total = block_exclusive_scan<int64_t>(a.new_prefix_off, a.n_slots, tot64);
     const int64_t chunks = block_exclusive_scan<int64_t>(a.chunk_off, a.n_slots, tot64);
+    int64_t table_len = 0;
+    if (a.paged) table_len = block_exclusive_scan<int64_t>(a.new_page_off, a.n_slots, tot64);
     if (threadIdx.x == 0) {
         a.new_prefix_off[a.n_slots] = total;
         a.chunk_off[a.n_slots] = chunks;
         int err = bad;
-        if (!err && total > a.capacity) err = DSBD_DEV_CAPACITY;
+        if (a.paged) {
+            a.new_page_off[a.n_slots] = table_len;
+            if (!err && (table_len > a.capacity || chunks > (int64_t)*a.free_count)) err = DSBD_DEV_CAPACITY;
+        } else if (!err && total > a.capacity) {
+            err = DSBD_DEV_CAPACITY;
+        }
         a.plan->n_beams = nb;
         a.plan->error = err;
         a.plan->total_tokens = total;
@@ -236,11 +268,72 @@ k_commit_copy(CommitArgs a) {
     }
 }
 
+// Paged update, CTA = (new beam j, kv head g, K|V): the (j, 0, K) CTA also writes the beam's page
+// table; every CTA fills its head's rows of the beam's fresh pages -- the rows of the input
+// beam's partial page, the path rows, then zeros (rows past a cache's length must stay finite
+// because the attention multiplies them by zero weights).
+__global__ void __launch_bounds__(kCopyThreads)
+k_commit_pages(CommitArgs a) {
+    if (a.plan->error) return;
+    const int j = blockIdx.x / (a.Hkv * 2);
+    if (j >= a.plan->n_beams) return;
+    const int g = (blockIdx.x / 2) % a.Hkv, kv = blockIdx.x & 1;
+    const int b = a.src_beam[j];
+    const int64_t L_old = a.prefix_off[b + 1] - a.prefix_off[b];
+    const int full = (int)(L_old / kPage), rem = (int)(L_old % kPage);
+    const int plen = a.path_len[j];
+    const int n_fresh = (int)(a.chunk_off[j + 1] - a.chunk_off[j]);
+    const int32_t *old_pages = a.page_table + a.page_off[b];
+    const int32_t *fresh = a.free_stack + (*a.free_count - 1 - a.chunk_off[j]);     // fresh page i = fresh[-i]
+    int32_t *table = a.new_page_table + a.new_page_off[j];
+    if (g == 0 && kv == 0) {
+        for (int i = threadIdx.x; i < full; i += blockDim.x) table[i] = old_pages[i];
+        for (int i = threadIdx.x; i < n_fresh; i += blockDim.x) table[full + i] = fresh[-i];
+    }
+    const int rb = a.row_bytes, upr = rb / 16;                   // 16-byte units per row
+    const unsigned char *pool_in = kv ? a.v_prefix : a.k_prefix;
+    unsigned char *pool_out = kv ? a.v_dst : a.k_dst;
+    const unsigned char *src_new = kv ? a.v_new : a.k_new;
+    const int32_t *path = a.path + (int64_t)j * (a.gamma + 1);
+    const int64_t part_row0 = rem ? ((int64_t)old_pages[full] * a.Hkv + g) * kPage : 0;
+    const int units = n_fresh * kPage * upr;
+    for (int u = threadIdx.x; u < units; u += blockDim.x) {
+        const int row = u / upr, within = (u - row * upr) * 16;  // row of the fresh pages' token range
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (row < rem) v = ld_stream16(pool_in + (part_row0 + row) * rb + within);
+        else if (row < rem + plen) v = ld_stream16(src_new + ((int64_t)path[row - rem] * a.Hkv + g) * rb + within);
+        const int pg = fresh[-(row / kPage)];
+        st_stream16(pool_out + (((int64_t)pg * a.Hkv + g) * kPage + (row % kPage)) * rb + within, v);
+    }
+}
+
+// The free stack after the update: every page that no new table names, ascending.
+__global__ void __launch_bounds__(kPlanThreads)
+k_commit_free(CommitArgs a) {
+    __shared__ int32_t tot32[32];
+    if (a.plan->error) return;
+    const int n = (int)a.n_pages;
+    for (int i = threadIdx.x; i <= n; i += blockDim.x) a.used[i] = 1;            // 1 = free
+    __syncthreads();
+    const int64_t entries = a.new_page_off[a.n_slots];
+    for (int64_t i = threadIdx.x; i < entries; i += blockDim.x) {
+        const int pg = a.new_page_table[i];
+        if (pg >= 0 && pg < n) a.used[pg] = 0;
+    }
+    __syncthreads();
+    const int total = block_exclusive_scan<int32_t>(a.used, n, tot32);           // position of each free page
+    if (threadIdx.x == 0) a.used[n] = total;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        if (a.used[i + 1] != a.used[i]) a.free_stack[a.used[i]] = i;
+    if (threadIdx.x == 0) *a.free_count = total;
+}
+
 struct Layout {
-    size_t plan, req_count, src_beam, path, path_len, chunk_off, total;
+    size_t plan, req_count, src_beam, path, path_len, chunk_off, used, total;
 };
 
-Layout make_layout(const dsbd_forest_t *f, const dsbd_commit_params_t *p) {
+Layout make_layout(const dsbd_forest_t *f, const dsbd_commit_params_t *p, int64_t n_pages = 0) {
     Layout L;
     size_t off = 0;
     L.plan = off;      off = align_up(off + sizeof(Plan), 256);
@@ -249,6 +342,7 @@ Layout make_layout(const dsbd_forest_t *f, const dsbd_commit_params_t *p) {
     L.path = off;      off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots * ((size_t)f->max_depth + 1), 256);
     L.path_len = off;  off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots, 256);
     L.chunk_off = off; off = align_up(off + sizeof(int64_t) * ((size_t)p->n_slots + 1), 256);
+    L.used = off;      off = align_up(off + sizeof(int32_t) * ((size_t)n_pages + 1), 256);
     L.total = off;
     return L;
 }
@@ -316,5 +410,71 @@ extern "C" int dsbd_kv_commit(const dsbd_forest_t *f, const dsbd_attn_desc_t *de
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     k_commit_copy<<<sms * 8, kCopyThreads, 0, stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
+}
+
+extern "C" size_t dsbd_kv_commit_paged_workspace(const dsbd_forest_t *forest, const dsbd_commit_params_t *params,
+                                                 int64_t n_pages) {
+    if (!args_ok(forest, params) || n_pages <= 0) return 0;
+    return make_layout(forest, params, n_pages).total;
+}
+
+extern "C" int dsbd_kv_commit_paged(const dsbd_forest_t *f, const dsbd_attn_desc_t *desc,
+                                    const dsbd_commit_params_t *p, const int32_t *out_off,
+                                    const int32_t *out_width, const int32_t *out_parent,
+                                    const int32_t *out_root_beam, const float *out_logp, const void *k_new,
+                                    const void *v_new, void *k_pool, void *v_pool, const dsbd_kv_pages_t *pages,
+                                    const int64_t *prefix_off, int32_t *free_stack, int32_t *free_count,
+                                    int32_t *new_req_beam_off, int64_t *new_prefix_off, int64_t *new_page_off,
+                                    int32_t *new_page_table, int32_t *new_beam_slot, void *workspace,
+                                    size_t workspace_bytes, int32_t *status, dsbd_stream_t stream_) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    if (!args_ok(f, p) || !desc || !pages) return DSBD_ERR_INVALID_ARG;
+    if (!out_off || !out_width || !out_parent || !out_root_beam || !k_new || !v_new || !k_pool || !v_pool ||
+        !pages->page_table || !pages->page_off || pages->n_pages <= 0 || !prefix_off || !free_stack || !free_count ||
+        !new_req_beam_off || !new_prefix_off || !new_page_off || !new_page_table || !new_beam_slot || !workspace ||
+        !status)
+        return DSBD_ERR_INVALID_ARG;
+    if (p->keep_best && !out_logp) return DSBD_ERR_INVALID_ARG;
+    if (desc->Hkv <= 0 || desc->d <= 0) return DSBD_ERR_INVALID_ARG;
+    if (desc->dtype != DSBD_DTYPE_BF16 && desc->dtype != DSBD_DTYPE_F32) return DSBD_ERR_UNSUPPORTED;
+    if (pages->n_pages >= (int64_t)1 << 31) return DSBD_ERR_UNSUPPORTED;
+    const int row_bytes = desc->d * (desc->dtype == DSBD_DTYPE_BF16 ? 2 : 4);
+    if (row_bytes % 16) return DSBD_ERR_UNSUPPORTED;
+    const uintptr_t ptrs = reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
+                           reinterpret_cast<uintptr_t>(k_pool) | reinterpret_cast<uintptr_t>(v_pool);
+    if (ptrs & 15) return DSBD_ERR_UNSUPPORTED;
+    const Layout L = make_layout(f, p, pages->n_pages);
+    if (workspace_bytes < L.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+    char *ws = static_cast<char *>(workspace);
+
+    CommitArgs a = {};
+    a.R = f->R; a.B = f->B; a.N = f->N; a.gamma = f->max_depth; a.Hkv = desc->Hkv;
+    a.n_slots = p->n_slots; a.keep_best = p->keep_best ? 1 : 0; a.row_bytes = row_bytes;
+    a.capacity = p->dst_capacity;
+    a.req_beam_off = f->req_beam_off; a.beam_node_off = f->beam_node_off; a.parent = f->parent;
+    a.out_off = out_off; a.out_width = out_width; a.out_parent = out_parent; a.out_root_beam = out_root_beam;
+    a.out_logp = out_logp; a.prefix_off = prefix_off;
+    a.k_new = static_cast<const unsigned char *>(k_new); a.v_new = static_cast<const unsigned char *>(v_new);
+    a.k_prefix = static_cast<const unsigned char *>(k_pool);
+    a.v_prefix = static_cast<const unsigned char *>(v_pool);
+    a.k_dst = static_cast<unsigned char *>(k_pool); a.v_dst = static_cast<unsigned char *>(v_pool);
+    a.new_req_beam_off = new_req_beam_off; a.new_prefix_off = new_prefix_off; a.new_beam_slot = new_beam_slot;
+    a.paged = 1; a.n_pages = pages->n_pages; a.page_table = pages->page_table; a.page_off = pages->page_off;
+    a.new_page_table = new_page_table; a.new_page_off = new_page_off;
+    a.free_stack = free_stack; a.free_count = free_count;
+    a.plan = reinterpret_cast<Plan *>(ws + L.plan);
+    a.req_count = reinterpret_cast<int32_t *>(ws + L.req_count);
+    a.src_beam = reinterpret_cast<int32_t *>(ws + L.src_beam);
+    a.path = reinterpret_cast<int32_t *>(ws + L.path);
+    a.path_len = reinterpret_cast<int32_t *>(ws + L.path_len);
+    a.chunk_off = reinterpret_cast<int64_t *>(ws + L.chunk_off);
+    a.used = reinterpret_cast<int32_t *>(ws + L.used);
+    a.status = status;
+
+    k_commit_plan<<<1, kPlanThreads, 0, stream>>>(a);
+    k_commit_pages<<<(unsigned)(p->n_slots * desc->Hkv * 2), kCopyThreads, 0, stream>>>(a);
+    k_commit_free<<<1, kPlanThreads, 0, stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }

@@ -78,3 +78,120 @@ def test_unsupported_shapes_are_refused():
         dsbd.forest_attention_paged(dsbd.Forest(forest, "cuda"), 4, 4, 64, 0.125, t["q"], t["k_new"], t["v_new"],
                                     pg["k_pool"], pg["v_pool"], pg["table"], pg["page_off"],
                                     torch.as_tensor(poff).cuda(), poff)
+
+
+def _forest_on(rng, req_beam_off, max_nodes):
+    B = int(req_beam_off[-1])
+    sizes = rng.integers(1, max_nodes + 1, size=B)
+    node_off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    parent = np.full(node_off[-1], -1, np.int32)
+    for b in range(B):
+        for i in range(1, sizes[b]):
+            parent[node_off[b] + i] = node_off[b] + rng.integers(0, i)
+    return dict(R=len(req_beam_off) - 1, B=B, N=int(node_off[-1]), max_depth=max_nodes,
+                req_beam_off=np.asarray(req_beam_off, np.int32), beam_node_off=node_off, parent=parent,
+                token=np.zeros(node_off[-1], np.int32))
+
+
+def _outputs(rng, forest, width):
+    rbo, bno = forest["req_beam_off"], forest["beam_node_off"]
+    R = forest["R"]
+    out_off = (np.arange(R + 1) * width).astype(np.int32)
+    out_width = rng.integers(1, width + 1, size=R).astype(np.int32)
+    out_parent = np.zeros(R * width, np.int32)
+    out_root = np.zeros(R * width, np.int32)
+    for r in range(R):
+        for k in range(width):
+            b = rng.integers(rbo[r], rbo[r + 1])
+            out_parent[r * width + k] = rng.integers(bno[b], bno[b + 1])
+            out_root[r * width + k] = b
+    return out_off, out_width, out_parent, out_root, (rng.normal(size=R * width) - 9).astype(np.float32)
+
+
+@pytest.mark.parametrize("dtype,Hkv,d", [(torch.bfloat16, 4, 128), (torch.float32, 2, 64)])
+def test_paged_commit_over_several_steps(dtype, Hkv, d):
+    """Six decode steps of cache updates on the device against the paged oracle on the host:
+    tables, offsets and allocator state bit for bit; the pools through what they mean (the
+    gathered caches); at the end the paged attention runs on the device's state."""
+    rng = np.random.default_rng(7)
+    rbo = np.array([0, 2, 3, 6, 7], np.int32)
+    L = [100, 100, 63, 700, 700, 700, 64]
+    poff = np.concatenate([[0], np.cumsum(L)]).astype(np.int64)
+    n_pages = 60
+    g = torch.Generator(device="cuda"); g.manual_seed(1)
+    mk = lambda *s: torch.randn(*s, generator=g, device="cuda").to(dtype)
+    kp, vp = mk(int(poff[-1]) * Hkv * d), mk(int(poff[-1]) * Hkv * d)
+    hk, hv, table, page_off, free, nfree = kvp.pack_into_pages(_bits(kp), _bits(vp), poff, Hkv, d, n_pages, rng)
+    dk, dv = _from_bits(hk, dtype).cuda(), _from_bits(hv, dtype).cuda()
+    d_table, d_page_off = torch.as_tensor(table).cuda(), torch.as_tensor(page_off).cuda()
+    d_free, d_nfree = torch.as_tensor(free).cuda(), torch.tensor([nfree], dtype=torch.int32, device="cuda")
+    i32 = lambda a: torch.as_tensor(np.asarray(a, np.int32)).cuda()
+    for step in range(6):
+        forest = _forest_on(rng, rbo, 6)
+        kn, vn = mk(forest["N"], Hkv, d), mk(forest["N"], Hkv, d)
+        outs = _outputs(rng, forest, 3)
+        keep_best = step == 3
+        ref = kvp.kv_commit_paged(forest, *outs, _bits(kn), _bits(vn), hk, hv, table, page_off, poff, free, nfree,
+                                  keep_best=keep_best)
+        assert ref["error"] == 0
+        res = dsbd.kv_commit_paged(dsbd.Forest(forest, "cuda"), Hkv, d, i32(outs[0]), i32(outs[1]), i32(outs[2]),
+                                   i32(outs[3]), torch.as_tensor(outs[4]).cuda(), kn, vn, dk, dv, d_table,
+                                   d_page_off, torch.as_tensor(poff).cuda(), poff, d_free, d_nfree,
+                                   n_slots=int(outs[0][-1]), table_capacity=len(ref["new_page_table"]) + 3,
+                                   keep_best=keep_best)
+        torch.cuda.synchronize()
+        assert int(res["status"].item()) == 0
+        nb = len(ref["new_beam_slot"])
+        assert np.array_equal(res["new_req_beam_off"].cpu().numpy(), ref["new_req_beam_off"])
+        assert np.array_equal(res["new_prefix_off"].cpu().numpy()[:nb + 1], ref["new_prefix_off"])
+        assert np.array_equal(res["new_page_off"].cpu().numpy()[:nb + 1], ref["new_page_off"])
+        nt = len(ref["new_page_table"])
+        assert np.array_equal(res["new_page_table"].cpu().numpy()[:nt], ref["new_page_table"])
+        assert np.array_equal(res["new_beam_slot"].cpu().numpy()[:nb], ref["new_beam_slot"])
+        assert int(d_nfree.item()) == ref["free_count"]
+        assert np.array_equal(d_free.cpu().numpy()[:ref["free_count"]], ref["free_stack"][:ref["free_count"]])
+        gk, gv = kvp.gather(_bits(dk).reshape(hk.shape), _bits(dv).reshape(hv.shape), ref["new_page_table"],
+                            ref["new_page_off"], ref["new_prefix_off"])
+        wk, wv = kvp.gather(ref["k_pool"], ref["v_pool"], ref["new_page_table"], ref["new_page_off"],
+                            ref["new_prefix_off"])
+        assert np.array_equal(gk, wk) and np.array_equal(gv, wv)
+        assert torch.isfinite(dk.float()).all() and torch.isfinite(dv.float()).all()
+        rbo, poff = ref["new_req_beam_off"], ref["new_prefix_off"]
+        hk, hv, table, page_off = ref["k_pool"], ref["v_pool"], ref["new_page_table"], ref["new_page_off"]
+        free, nfree = ref["free_stack"], ref["free_count"]
+        d_table = res["new_page_table"][:nt].contiguous()
+        d_page_off = res["new_page_off"][:nb + 1].contiguous()
+    if dtype == torch.bfloat16:
+        forest = _forest_on(rng, rbo, 6)
+        Hq = 2 * Hkv
+        t = dict(q=mk(forest["N"], Hq, d), k_new=mk(forest["N"], Hkv, d), v_new=mk(forest["N"], Hkv, d))
+        out, st = dsbd.forest_attention_paged(dsbd.Forest(forest, "cuda"), Hq, Hkv, d, inputs.default_scale(d),
+                                              t["q"], t["k_new"], t["v_new"], dk, dv, d_table, d_page_off,
+                                              torch.as_tensor(poff).cuda(), poff)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        wk, wv = kvp.gather(hk, hv, table, page_off, poff)
+        t["k_prefix"], t["v_prefix"] = _from_bits(wk, dtype).cuda(), _from_bits(wv, dtype).cuda()
+        nodes, ref = _oracle_beams(forest, dict(Hq=Hq, Hkv=Hkv, d=d), t, poff, list(range(forest["B"])))
+        attention_close(to_host_f32(out), ref, bf16=True)
+
+
+def test_paged_commit_without_free_pages_changes_nothing():
+    rng = np.random.default_rng(9)
+    Hkv, d = 2, 64
+    rbo, poff = np.array([0, 1], np.int32), np.array([0, 10], np.int64)
+    kp = torch.randn(10 * Hkv * d, device="cuda")
+    hk, hv, table, page_off, free, nfree = kvp.pack_into_pages(_bits(kp), _bits(kp), poff, Hkv, d, 2)
+    dk, dv = _from_bits(hk, torch.float32).cuda(), _from_bits(hv, torch.float32).cuda()
+    forest = _forest_on(rng, rbo, 2)
+    kn = torch.randn(forest["N"], Hkv, d, device="cuda")
+    i32 = lambda a: torch.as_tensor(np.asarray(a, np.int32)).cuda()
+    d_free, d_nfree = torch.as_tensor(free).cuda(), torch.tensor([nfree], dtype=torch.int32, device="cuda")
+    before = dk.clone()
+    res = dsbd.kv_commit_paged(dsbd.Forest(forest, "cuda"), Hkv, d, i32([0, 2]), i32([2]), i32([0, 0]), i32([0, 0]),
+                               None, kn, kn, dk, dv, torch.as_tensor(table).cuda(), torch.as_tensor(page_off).cuda(),
+                               torch.as_tensor(poff).cuda(), poff, d_free, d_nfree, n_slots=2, table_capacity=8)
+    torch.cuda.synchronize()
+    assert int(res["status"].item()) == 3
+    assert torch.equal(dk, before) and int(d_nfree.item()) == nfree
+    assert np.array_equal(d_free.cpu().numpy(), free)
