@@ -373,6 +373,55 @@ def main():
     assert int(status.item()) == 0, "device status %d" % int(status.item())
     del k_dst, v_dst
 
+    # the paged form of the caches: the same attention through page tables, and the cache update
+    # that copies no prefix (bf16, d = 128 only)
+    paged_ms = paged_commit_ms = None
+    if data["k_new"].dtype == torch.bfloat16 and spec["d"] == 128:
+        pg = inputs.paginate(data["k_prefix"], data["v_prefix"], poff, spec["Hkv"], spec["d"],
+                             extra_pages=2 * n_slots + 64, seed=int(spec["seed"]))
+        attn_out_pg = torch.empty_like(attn_out)
+
+        def attention_paged():
+            dsbd.forest_attention_paged(f, spec["Hq"], spec["Hkv"], spec["d"], scale, data["q"], data["k_new"],
+                                        data["v_new"], pg["k_pool"], pg["v_pool"], pg["page_table"],
+                                        pg["page_off"], poff_dev, poff, out=attn_out_pg, workspace=ws_a,
+                                        status=status, stream=stream)
+        for _ in range(3):
+            attention_paged()
+        p0 = torch.cuda.Event(enable_timing=True); p1 = torch.cuda.Event(enable_timing=True)
+        n_pg = max(args.steps // 2, 5)
+        p0.record(stream)
+        for _ in range(n_pg):
+            attention_paged()
+        p1.record(stream)
+        torch.cuda.synchronize()
+        paged_ms = p0.elapsed_time(p1) / n_pg
+        assert torch.equal(attn_out_pg, attn_out), "paged and packed attention differ"
+        table_cap = int(pg["page_table"].numel()) + 2 * n_slots
+        free0, count0 = pg["free_stack"].clone(), pg["free_count"].clone()
+        pc = None
+
+        def commit_paged():
+            # every call starts from the same allocator state (two small device copies)
+            pg["free_stack"].copy_(free0); pg["free_count"].copy_(count0)
+            return dsbd.kv_commit_paged(f, spec["Hkv"], spec["d"], out_off_dev, vout["out_width"], vout["out_parent"],
+                                        vout["out_root_beam"], vout["out_logp"], data["k_new"], data["v_new"],
+                                        pg["k_pool"], pg["v_pool"], pg["page_table"], pg["page_off"], poff_dev, poff,
+                                        pg["free_stack"], pg["free_count"], n_slots=n_slots,
+                                        table_capacity=table_cap, workspace=pc["workspace"] if pc else None,
+                                        status=status, stream=stream)
+        for _ in range(3):
+            pc = commit_paged()
+        q0 = torch.cuda.Event(enable_timing=True); q1 = torch.cuda.Event(enable_timing=True)
+        q0.record(stream)
+        for _ in range(n_commit):
+            commit_paged()
+        q1.record(stream)
+        torch.cuda.synchronize()
+        paged_commit_ms = q0.elapsed_time(q1) / n_commit
+        assert int(status.item()) == 0, "device status %d" % int(status.item())
+        del pg, attn_out_pg
+
     # one draft-stage sampling step of the same shape (W_S = beams of the request), reported
     # beside the step: the small model's logits of the first B rows stand for a draft layer
     rbo_host = np.asarray(forest["req_beam_off"], dtype=np.int32)
@@ -450,6 +499,11 @@ def main():
         "kv_commit": {"bytes": commit_bytes, "ms": commit_ms, "gbs": commit_bytes / commit_ms * 1e-6},
         "draft_layer": {"bytes": draft_bytes, "ms": draft_ms, "gbs": draft_bytes / draft_ms * 1e-6},
     }
+    if paged_ms is not None:
+        kernels["forest_attention_paged"] = {"bytes": a_bytes, "ms": paged_ms, "gbs": a_bytes / paged_ms * 1e-6}
+        # the paged update moves only partial pages and paths; the same kept-cache bytes as
+        # kv_commit are the work it replaces, so no bandwidth figure is given
+        kernels["kv_commit_paged"] = {"bytes": 0, "ms": paged_commit_ms, "gbs": 0.0}
     for k in kernels.values():
         k["frac_of_%s_peak" % peak_kind] = k["gbs"] / peak
         k["frac_of_8TBs_nominal"] = k["gbs"] / 8000.0

@@ -159,6 +159,44 @@ def generate(spec, device, parts=("attention", "verify"), draft_top_k=0, draft_t
     return out
 
 
+PAGE_TOKENS = 64
+
+
+def paginate(k_prefix, v_prefix, prefix_off, Hkv, d, extra_pages, seed=0):
+    """The packed caches cut into pages of 64 tokens with shuffled page ids (layout change only).
+    Returns dict(k_pool, v_pool [n_pages, Hkv, 64, d], page_table int32, page_off int64 [B+1],
+    free_stack int32 [n_pages], free_count int32 [1]); rows past a cache's length are zero."""
+    dev = k_prefix.device
+    L = np.diff(np.asarray(prefix_off))
+    need = [int(-(-int(l) // PAGE_TOKENS)) for l in L]
+    total = int(sum(need))
+    n_pages = total + int(extra_pages)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    ids = torch.randperm(n_pages, generator=gen)
+    k_pool = torch.zeros(n_pages, Hkv, PAGE_TOKENS, d, dtype=k_prefix.dtype, device=dev)
+    v_pool = torch.zeros_like(k_pool)
+    page_off = np.concatenate([[0], np.cumsum(need)]).astype(np.int64)
+    for b, l in enumerate(L):
+        l = int(l)
+        if l == 0:
+            continue
+        base = int(prefix_off[b]) * Hkv * d
+        pages = ids[int(page_off[b]):int(page_off[b + 1])].to(dev)
+        for src, pool in ((k_prefix, k_pool), (v_prefix, v_pool)):
+            x = src[base:base + Hkv * l * d].view(Hkv, l, d)
+            pad = need[b] * PAGE_TOKENS - l
+            if pad:
+                x = torch.cat([x, torch.zeros(Hkv, pad, d, dtype=x.dtype, device=dev)], dim=1)
+            pool[pages] = x.view(Hkv, need[b], PAGE_TOKENS, d).permute(1, 0, 2, 3)
+    free = torch.sort(ids[total:]).values.to(torch.int32)
+    free_stack = torch.zeros(n_pages, dtype=torch.int32)
+    free_stack[:free.numel()] = free
+    return dict(k_pool=k_pool, v_pool=v_pool, page_table=ids[:total].to(torch.int32).to(dev),
+                page_off=torch.as_tensor(page_off).to(dev), free_stack=free_stack.to(dev),
+                free_count=torch.tensor([free.numel()], dtype=torch.int32, device=dev))
+
+
 def attention_bytes(spec, forest, prefix_off):
     """Algorithmic HBM bytes of one forest-attention launch: the KV prefix of every beam once
     (K and V), plus Q, O and the new K/V of every node."""
