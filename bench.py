@@ -357,7 +357,8 @@ def main():
                               vout["out_root_beam"], vout["out_logp"], data["k_new"], data["v_new"],
                               data["k_prefix"], data["v_prefix"], poff_dev, poff, n_slots=n_slots,
                               dst_capacity=cap, k_dst=k_dst, v_dst=v_dst,
-                              workspace=commit["workspace"] if commit else None, status=status, stream=stream)
+                              workspace=commit["workspace"] if commit else None, status=status, stream=stream,
+                              out=commit)
     for _ in range(3):
         commit = kv_commit()
     c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True)
@@ -409,7 +410,7 @@ def main():
                                         pg["k_pool"], pg["v_pool"], pg["page_table"], pg["page_off"], poff_dev, poff,
                                         pg["free_stack"], pg["free_count"], n_slots=n_slots,
                                         table_capacity=table_cap, workspace=pc["workspace"] if pc else None,
-                                        status=status, stream=stream)
+                                        status=status, stream=stream, out=pc)
         for _ in range(3):
             pc = commit_paged()
         q0 = torch.cuda.Event(enable_timing=True); q1 = torch.cuda.Event(enable_timing=True)
@@ -432,7 +433,8 @@ def main():
 
     def draft_layer():
         return dsbd.draft_layer(rbo_dev, rbo_host, prm, 1, W_S_r, zq_rows, data["root_logq"], rbo_dev, f.B,
-                                workspace=draft["workspace"] if draft else None, status=status, stream=stream)
+                                workspace=draft["workspace"] if draft else None, status=status, stream=stream,
+                                out=draft)
     for _ in range(3):
         draft = draft_layer()
     g0 = torch.cuda.Event(enable_timing=True); g1 = torch.cuda.Event(enable_timing=True)

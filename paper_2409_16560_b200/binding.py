@@ -265,8 +265,8 @@ class DraftParamsT(C.Structure):
 
 
 def draft_layer(req_beam_off, req_beam_off_host, params, layer, W_S, logits_q, beam_logq, out_off, n_slots,
-                row_stride=None, workspace=None, status=None, stream=None):
-    """dsbd_draft_layer.  req_beam_off, out_off: int32 device tensors; W_S: int or int32 device
+                row_stride=None, workspace=None, status=None, stream=None, out=None):
+    """dsbd_draft_layer (out: the dict of an earlier call, to reuse its tensors).  req_beam_off, out_off: int32 device tensors; W_S: int or int32 device
     tensor [R]; params: V, temperature, seed, step, top_k, top_p.  Returns dict(out_parent,
     out_token, out_logq, req_error, status) on the device."""
     _require_cuda(req_beam_off, logits_q, beam_logq, out_off)
@@ -292,10 +292,12 @@ def draft_layer(req_beam_off, req_beam_off_host, params, layer, W_S, logits_q, b
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
-    res = dict(out_parent=torch.full((int(n_slots),), -1, dtype=torch.int32, device=dev),
-               out_token=torch.full((int(n_slots),), -1, dtype=torch.int32, device=dev),
-               out_logq=torch.zeros(int(n_slots), dtype=torch.float32, device=dev),
-               req_error=torch.zeros(R, dtype=torch.int32, device=dev), status=status, workspace=workspace)
+    res = out if out is not None else dict(
+        out_parent=torch.full((int(n_slots),), -1, dtype=torch.int32, device=dev),
+        out_token=torch.full((int(n_slots),), -1, dtype=torch.int32, device=dev),
+        out_logq=torch.zeros(int(n_slots), dtype=torch.float32, device=dev),
+        req_error=torch.zeros(R, dtype=torch.int32, device=dev))
+    res["status"], res["workspace"] = status, workspace
     stride = int(row_stride) if row_stride is not None else int(logits_q.stride(0))
     rc = load().dsbd_draft_layer(R, n_beams, _ptr(req_beam_off), C.addressof(p), _ptr(logits_q), stride,
                                  _ptr(beam_logq), _ptr(out_off), _ptr(res["out_parent"]), _ptr(res["out_token"]),
@@ -312,7 +314,7 @@ class CommitParamsT(C.Structure):
 
 def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out_logp, k_new, v_new,
               k_prefix, v_prefix, prefix_off, prefix_off_host, n_slots, dst_capacity, keep_best=False,
-              k_dst=None, v_dst=None, workspace=None, status=None, stream=None):
+              k_dst=None, v_dst=None, workspace=None, status=None, stream=None, out=None):
     """dsbd_kv_commit; returns a dict with k_dst, v_dst, new_req_beam_off, new_prefix_off,
     new_beam_slot and the status tensor (all on the device, nothing is synchronised)."""
     _require_cuda(out_off, out_width, out_parent, out_root_beam, k_new, v_new, k_prefix, v_prefix, prefix_off)
@@ -330,9 +332,13 @@ def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
-    new_req_beam_off = torch.empty(forest.R + 1, dtype=torch.int32, device=dev)
-    new_prefix_off = torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev)
-    new_beam_slot = torch.empty(int(n_slots), dtype=torch.int32, device=dev)
+    if out is not None:
+        new_req_beam_off, new_prefix_off, new_beam_slot = (out[k] for k in ("new_req_beam_off", "new_prefix_off",
+                                                                              "new_beam_slot"))
+    else:
+        new_req_beam_off = torch.empty(forest.R + 1, dtype=torch.int32, device=dev)
+        new_prefix_off = torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev)
+        new_beam_slot = torch.empty(int(n_slots), dtype=torch.int32, device=dev)
     rc = load().dsbd_kv_commit(C.addressof(f), C.addressof(desc), C.addressof(p), _ptr(out_off), _ptr(out_width),
                                _ptr(out_parent), _ptr(out_root_beam), _ptr(out_logp) if out_logp is not None else None,
                                _ptr(k_new), _ptr(v_new), _ptr(k_prefix), _ptr(v_prefix), _ptr(prefix_off),
@@ -347,7 +353,7 @@ def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out
 
 def kv_commit_paged(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out_logp, k_new, v_new,
                     k_pool, v_pool, page_table, page_off, prefix_off, prefix_off_host, free_stack, free_count,
-                    n_slots, table_capacity, keep_best=False, workspace=None, status=None, stream=None):
+                    n_slots, table_capacity, keep_best=False, workspace=None, status=None, stream=None, out=None):
     """dsbd_kv_commit_paged; the pools, free_stack and free_count are updated in place.  Returns a
     dict with new_req_beam_off, new_prefix_off, new_page_off, new_page_table, new_beam_slot and the
     status tensor (device tensors, nothing is synchronised)."""
@@ -365,12 +371,13 @@ def kv_commit_paged(forest, Hkv, d, out_off, out_width, out_parent, out_root_bea
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
-    res = dict(new_req_beam_off=torch.empty(forest.R + 1, dtype=torch.int32, device=dev),
-               new_prefix_off=torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev),
-               new_page_off=torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev),
-               new_page_table=torch.full((int(table_capacity),), -1, dtype=torch.int32, device=dev),
-               new_beam_slot=torch.empty(int(n_slots), dtype=torch.int32, device=dev),
-               status=status, workspace=workspace)
+    res = out if out is not None else dict(
+        new_req_beam_off=torch.empty(forest.R + 1, dtype=torch.int32, device=dev),
+        new_prefix_off=torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev),
+        new_page_off=torch.empty(int(n_slots) + 1, dtype=torch.int64, device=dev),
+        new_page_table=torch.full((int(table_capacity),), -1, dtype=torch.int32, device=dev),
+        new_beam_slot=torch.empty(int(n_slots), dtype=torch.int32, device=dev))
+    res["status"], res["workspace"] = status, workspace
     rc = load().dsbd_kv_commit_paged(
         C.addressof(f), C.addressof(desc), C.addressof(p), _ptr(out_off), _ptr(out_width), _ptr(out_parent),
         _ptr(out_root_beam), _ptr(out_logp) if out_logp is not None else None, _ptr(k_new), _ptr(v_new),

@@ -67,6 +67,8 @@ struct CommitArgs {
     int32_t *path;            // [n_slots][gamma+1] nodes root .. parent
     int32_t *path_len;        // [n_slots]
     int64_t *chunk_off;       // [n_slots+1] copy chunks before each beam; paged: fresh pages before it
+    int32_t *slot_req, *slot_depth, *req_best;   // [n_slots], [n_slots], [R]
+    double *slot_key;         // [n_slots]
     int32_t *status;
 };
 
@@ -104,64 +106,79 @@ k_commit_plan(CommitArgs a) {
     __shared__ int bad;
     if (threadIdx.x == 0) bad = 0;
     __syncthreads();
-    // kept slots per request
+    // every slot on its own thread: which request it belongs to, whether it is in use, the depth
+    // of its parent node (the walk to the root is a chain of dependent loads, so slots run in
+    // parallel), and its perplexity key
+    for (int s = threadIdx.x; s < a.n_slots; s += blockDim.x) {
+        int lo = 0, hi = a.R - 1;                       // last request whose range starts at or before s
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (a.out_off[mid] <= s) lo = mid; else hi = mid - 1;
+        }
+        const int r = lo;
+        int depth = -1;                                  // -1: slot not in use
+        double key = 0.0;
+        if (s >= a.out_off[r] && s < a.out_off[r] + a.out_width[r] && s < a.out_off[r + 1]) {
+            const int b = a.out_root_beam[s];
+            const int n = a.out_parent[s];
+            if (b < a.req_beam_off[r] || b >= a.req_beam_off[r + 1] || n < a.beam_node_off[b] ||
+                n >= a.beam_node_off[b + 1]) {
+                bad = DSBD_DEV_BAD_FOREST;
+            } else {
+                depth = 0;
+                for (int c = n; a.parent[c] >= 0 && depth <= a.gamma; c = a.parent[c]) ++depth;
+                if (depth > a.gamma) { bad = DSBD_DEV_BAD_FOREST; depth = -1; }
+                else if (a.keep_best)
+                    key = -(double)a.out_logp[s] / ((double)(a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 2);
+            }
+        }
+        a.slot_req[s] = r;
+        a.slot_depth[s] = depth;
+        a.slot_key[s] = key;
+    }
+    __syncthreads();
+    // kept slots per request; with keep_best the slot of lowest perplexity exp(-logp / length),
+    // i.e. of lowest -logp / length, the first one on a tie
     for (int r = threadIdx.x; r < a.R; r += blockDim.x) {
         const int w = a.out_width[r];
         a.req_count[r] = w <= 0 ? 0 : (a.keep_best ? 1 : w);
+        int best = -1;
+        if (a.keep_best && w > 0) {
+            const int s0 = a.out_off[r];
+            double best_key = 0.0;
+            for (int s = s0; s < s0 + w && s < a.n_slots; ++s)
+                if (a.slot_depth[s] >= 0 && (best < 0 || a.slot_key[s] < best_key)) { best = s; best_key = a.slot_key[s]; }
+        }
+        a.req_best[r] = best;
     }
     __syncthreads();
     const int n_beams = block_exclusive_scan<int32_t>(a.req_count, a.R, tot32);
     if (n_beams > a.n_slots) { if (threadIdx.x == 0) bad = DSBD_DEV_CAPACITY; }
     __syncthreads();
     const bool fits = !bad;
-    // per request: its kept slots -> source beam, path, new length
-    for (int r = threadIdx.x; r < a.R && fits; r += blockDim.x) {
-        const int first = a.req_count[r];
-        a.new_req_beam_off[r] = first;
-        const int s0 = a.out_off[r], w = a.out_width[r];
-        if (w <= 0) continue;
-        int s_lo = s0, s_hi = s0 + w;
-        const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
-        if (a.keep_best) {
-            // lowest perplexity exp(-logp / length) = lowest -logp / length; first slot on a tie
-            int best = -1;
-            double best_key = 0.0;
-            for (int s = s_lo; s < s_hi; ++s) {
-                const int b = a.out_root_beam[s];
-                int n = a.out_parent[s];
-                if (b < b_lo || b >= b_hi || n < a.beam_node_off[b] || n >= a.beam_node_off[b + 1]) { bad = DSBD_DEV_BAD_FOREST; break; }
-                int depth = 0;
-                while (a.parent[n] >= 0 && depth <= a.gamma) { n = a.parent[n]; ++depth; }
-                const double length = (double)(a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 2;
-                const double key = -(double)a.out_logp[s] / length;
-                if (best < 0 || key < best_key) { best = s; best_key = key; }
-            }
-            if (best < 0) continue;
-            s_lo = best; s_hi = best + 1;
-        }
-        for (int s = s_lo; s < s_hi; ++s) {
-            const int j = first + (s - s_lo);
-            const int b = a.out_root_beam[s];
-            int n = a.out_parent[s];
-            if (b < b_lo || b >= b_hi || n < a.beam_node_off[b] || n >= a.beam_node_off[b + 1]) { bad = DSBD_DEV_BAD_FOREST; break; }
-            int depth = 0;
-            for (int c = n; a.parent[c] >= 0 && depth <= a.gamma; c = a.parent[c]) ++depth;
-            if (depth > a.gamma) { bad = DSBD_DEV_BAD_FOREST; break; }
-            int32_t *pj = a.path + (int64_t)j * (a.gamma + 1);
-            for (int c = n, i = depth; i >= 0; --i, c = a.parent[c]) pj[i] = c;
-            a.path_len[j] = depth + 1;
-            a.src_beam[j] = b;
-            a.new_beam_slot[j] = s;
-            const int64_t len = (a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 1;
-            a.new_prefix_off[j] = len;
-            if (a.paged) {
-                const int64_t L_old = len - depth - 1;
-                const int64_t fresh = (L_old % kPage + depth + 1 + kPage - 1) / kPage;
-                a.chunk_off[j] = fresh;
-                a.new_page_off[j] = L_old / kPage + fresh;
-            } else {
-                a.chunk_off[j] = (len * a.row_bytes + kChunkBytes - 1) / kChunkBytes;
-            }
+    for (int r = threadIdx.x; r < a.R && fits; r += blockDim.x) a.new_req_beam_off[r] = a.req_count[r];
+    // every kept slot: its new beam number, source beam, path and new length
+    for (int s = threadIdx.x; s < a.n_slots && fits; s += blockDim.x) {
+        const int depth = a.slot_depth[s];
+        if (depth < 0) continue;
+        const int r = a.slot_req[s];
+        if (a.keep_best && a.req_best[r] != s) continue;
+        const int j = a.req_count[r] + (a.keep_best ? 0 : s - a.out_off[r]);
+        const int b = a.out_root_beam[s];
+        int32_t *pj = a.path + (int64_t)j * (a.gamma + 1);
+        for (int c = a.out_parent[s], i = depth; i >= 0; --i, c = a.parent[c]) pj[i] = c;
+        a.path_len[j] = depth + 1;
+        a.src_beam[j] = b;
+        a.new_beam_slot[j] = s;
+        const int64_t len = (a.prefix_off[b + 1] - a.prefix_off[b]) + depth + 1;
+        a.new_prefix_off[j] = len;
+        if (a.paged) {
+            const int64_t L_old = len - depth - 1;
+            const int64_t fresh = (L_old % kPage + depth + 1 + kPage - 1) / kPage;
+            a.chunk_off[j] = fresh;
+            a.new_page_off[j] = L_old / kPage + fresh;
+        } else {
+            a.chunk_off[j] = (len * a.row_bytes + kChunkBytes - 1) / kChunkBytes;
         }
     }
     __syncthreads();
@@ -307,13 +324,18 @@ k_commit_pages(CommitArgs a) {
     }
 }
 
-// The free stack after the update: every page that no new table names, ascending.
+// The free stack after the update: every page that no new table names, ascending.  One CTA;
+// the compaction walks the page flags in super-tiles of 16 flags per thread, loaded as four
+// independent 128-bit loads, with a block scan of the per-thread counts.
 __global__ void __launch_bounds__(kPlanThreads)
 k_commit_free(CommitArgs a) {
-    __shared__ int32_t tot32[32];
+    __shared__ int32_t warp_tot[32];
+    __shared__ int32_t carry;
     if (a.plan->error) return;
     const int n = (int)a.n_pages;
-    for (int i = threadIdx.x; i <= n; i += blockDim.x) a.used[i] = 1;            // 1 = free
+    const int n_pad = (n + 15) & ~15;                                             // the array holds n + 1 <= n_pad + 16
+    for (int i = threadIdx.x; i < n_pad; i += blockDim.x) a.used[i] = i < n ? 1 : 0;   // 1 = free
+    if (threadIdx.x == 0) carry = 0;
     __syncthreads();
     const int64_t entries = a.new_page_off[a.n_slots];
     for (int64_t i = threadIdx.x; i < entries; i += blockDim.x) {
@@ -321,16 +343,46 @@ k_commit_free(CommitArgs a) {
         if (pg >= 0 && pg < n) a.used[pg] = 0;
     }
     __syncthreads();
-    const int total = block_exclusive_scan<int32_t>(a.used, n, tot32);           // position of each free page
-    if (threadIdx.x == 0) a.used[n] = total;
-    __syncthreads();
-    for (int i = threadIdx.x; i < n; i += blockDim.x)
-        if (a.used[i + 1] != a.used[i]) a.free_stack[a.used[i]] = i;
-    if (threadIdx.x == 0) *a.free_count = total;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < n_pad; base += kPlanThreads * 16) {
+        const int i0 = base + threadIdx.x * 16;
+        int4 f[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            f[q] = i0 + 4 * q < n_pad ? *reinterpret_cast<const int4 *>(a.used + i0 + 4 * q) : make_int4(0, 0, 0, 0);
+        int cnt = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) cnt += f[q].x + f[q].y + f[q].z + f[q].w;
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int before = carry, tile_total = 0;
+        for (int w = 0; w < kPlanThreads / 32; ++w) {
+            if (w < warp) before += warp_tot[w];
+            tile_total += warp_tot[w];
+        }
+        int pos = before + incl - cnt;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int v[4] = {f[q].x, f[q].y, f[q].z, f[q].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (v[e]) a.free_stack[pos++] = i0 + 4 * q + e;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) carry += tile_total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *a.free_count = carry;
 }
 
 struct Layout {
-    size_t plan, req_count, src_beam, path, path_len, chunk_off, used, total;
+    size_t plan, req_count, src_beam, path, path_len, chunk_off, slot_req, slot_depth, req_best, slot_key, used, total;
 };
 
 Layout make_layout(const dsbd_forest_t *f, const dsbd_commit_params_t *p, int64_t n_pages = 0) {
@@ -342,7 +394,11 @@ Layout make_layout(const dsbd_forest_t *f, const dsbd_commit_params_t *p, int64_
     L.path = off;      off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots * ((size_t)f->max_depth + 1), 256);
     L.path_len = off;  off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots, 256);
     L.chunk_off = off; off = align_up(off + sizeof(int64_t) * ((size_t)p->n_slots + 1), 256);
-    L.used = off;      off = align_up(off + sizeof(int32_t) * ((size_t)n_pages + 1), 256);
+    L.slot_req = off;  off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots, 256);
+    L.slot_depth = off; off = align_up(off + sizeof(int32_t) * (size_t)p->n_slots, 256);
+    L.req_best = off;  off = align_up(off + sizeof(int32_t) * (size_t)f->R, 256);
+    L.slot_key = off;  off = align_up(off + sizeof(double) * (size_t)p->n_slots, 256);
+    L.used = off;      off = align_up(off + sizeof(int32_t) * ((size_t)n_pages + 32), 256);
     L.total = off;
     return L;
 }
@@ -404,6 +460,10 @@ extern "C" int dsbd_kv_commit(const dsbd_forest_t *f, const dsbd_attn_desc_t *de
     a.path = reinterpret_cast<int32_t *>(ws + L.path);
     a.path_len = reinterpret_cast<int32_t *>(ws + L.path_len);
     a.chunk_off = reinterpret_cast<int64_t *>(ws + L.chunk_off);
+    a.slot_req = reinterpret_cast<int32_t *>(ws + L.slot_req);
+    a.slot_depth = reinterpret_cast<int32_t *>(ws + L.slot_depth);
+    a.req_best = reinterpret_cast<int32_t *>(ws + L.req_best);
+    a.slot_key = reinterpret_cast<double *>(ws + L.slot_key);
     a.status = status;
 
     k_commit_plan<<<1, kPlanThreads, 0, stream>>>(a);
@@ -470,6 +530,10 @@ extern "C" int dsbd_kv_commit_paged(const dsbd_forest_t *f, const dsbd_attn_desc
     a.path = reinterpret_cast<int32_t *>(ws + L.path);
     a.path_len = reinterpret_cast<int32_t *>(ws + L.path_len);
     a.chunk_off = reinterpret_cast<int64_t *>(ws + L.chunk_off);
+    a.slot_req = reinterpret_cast<int32_t *>(ws + L.slot_req);
+    a.slot_depth = reinterpret_cast<int32_t *>(ws + L.slot_depth);
+    a.req_best = reinterpret_cast<int32_t *>(ws + L.req_best);
+    a.slot_key = reinterpret_cast<double *>(ws + L.slot_key);
     a.used = reinterpret_cast<int32_t *>(ws + L.used);
     a.status = status;
 
