@@ -219,6 +219,7 @@ struct Shared {
     double col_a[kMaxLive + 1], col_b[kMaxLive + 1];
     double tail[kMaxLive + 2];
     int bank, need_exact, res_j, run_j, chain_pos;
+    int n_out, n_fill;                      // output beams so far; p_beam fills left to the whole CTA
     int n_layers, n_tests, n_exact, n_respass;
     uint32_t wtot_p[kWarps], wtot_q[kWarps];
     double rho[kMaxLive], uu[kMaxLive];     // per live draft: p_beam/q_beam and its uniform
@@ -359,12 +360,10 @@ __device__ int locate_token(const VerifyArgs &a, int row, int t, float bp, float
     return last;
 }
 
-__device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, int node, int tok,
-                            int source, bool writer, int *err) {
-    const int cap = a.out.out_off[r + 1] - a.out.out_off[r];
-    if (*n_out >= cap) { *err = DSBD_DEV_CAPACITY; return; }
-    if (writer) {
-        const int s = a.out.out_off[r] + *n_out;
+// Writes output beam number `index` of request r (the caller has checked the slot range).
+__device__ void emit_at(const VerifyArgs &a, int r, int index, int parent, int node, int tok, int source) {
+    {
+        const int s = a.out.out_off[r] + index;
         // the tree of a node: walk to the root, then find which beam starts there
         int root = parent;
         while (a.parent[root] >= 0) root = a.parent[root];
@@ -381,6 +380,13 @@ __device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, 
         a.out.out_logp[s] = (float)(a.score[parent] + lp);
         a.out.out_logq[s] = (float)(a.score[a.N + parent] + lq);
     }
+}
+
+__device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, int node, int tok,
+                            int source, bool writer, int *err) {
+    const int cap = a.out.out_off[r + 1] - a.out.out_off[r];
+    if (*n_out >= cap) { *err = DSBD_DEV_CAPACITY; return; }
+    if (writer) emit_at(a, r, *n_out, parent, node, tok, source);
     (*n_out)++;
 }
 
@@ -949,7 +955,7 @@ k_verify(VerifyArgs a) {
     for (int i = cta_rank * kThreads + threadIdx.x; i < 2 * hist_len; i += n_cta * kThreads) ghist[i] = 0ull;
     if (warp == 0) {
         if (lane == 0) {
-            sh.err = 0; sh.done = 0;
+            sh.err = 0; sh.done = 0; sh.n_out = 0; sh.n_fill = 0;
             sh.n_layers = sh.n_tests = sh.n_exact = sh.n_respass = 0;
             if (a.select_mode) {
                 const int lo = a.live_off[r], hi = a.live_off[r + 1];
@@ -1290,7 +1296,10 @@ k_verify(VerifyArgs a) {
                 n_out = __shfl_sync(kFull, n_out, 0);
                 err = __shfl_sync(kFull, err, 0);
                 int fill = 0;
-                for (int kk = count; kk < W && !err; ++kk) {
+                // unwarped: warp 0 makes the residual draw, the p_beam fills (independent draws)
+                // are then spread over the warps of the CTA
+                const int kk_end = warped ? W : count + 1;
+                for (int kk = count; kk < kk_end && !err; ++kk) {
                     const bool residual = (kk == count);
                     const bool use_res = residual && j > 1;
                     const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l,
@@ -1319,6 +1328,8 @@ k_verify(VerifyArgs a) {
                 if (lane == 0) {
                     sh.done = 1;
                     if (writer) a.out.l_last[r] = l;
+                    sh.n_out = n_out;
+                    sh.n_fill = (!warped && !err) ? W - count - 1 : 0;
                 }
             } else {
                 // the accepted drafts, ascending node id, are the next layer's input beams
@@ -1340,6 +1351,27 @@ k_verify(VerifyArgs a) {
             if (lane == 0 && err) sh.err = err;
         }
         __syncthreads();
+        if (!a.select_mode && sh.done && sh.n_fill > 0 && !sh.err) {
+            // fill f is output beam n_out + f, drawn from p_beam with its own uniform
+            const int cap = a.out.out_off[r + 1] - a.out.out_off[r];
+            const int base = sh.n_out, want = sh.n_fill;
+            const int n_draw = min(want, max(cap - base, 0));
+            __syncthreads();
+            for (int f = warp; f < n_draw; f += kWarps) {
+                const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l, 2u, (uint32_t)f);
+                int ia = 0;
+                const int tok = draw_cell(a, sh, u, false, 0.f, 0.0, nullptr, lane, &ia);
+                if (tok < 0) { if (lane == 0) sh.err = DSBD_DEV_EXHAUSTED; }
+                else if (lane == 0 && writer) emit_at(a, r, base + f, sh.A[ia], -1, tok, DSBD_SRC_FILL);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                if (!sh.err) { sh.n_out = base + n_draw; if (want > n_draw) sh.err = DSBD_DEV_CAPACITY; }
+                sh.n_fill = 0;
+            }
+            __syncthreads();
+            n_out = sh.n_out;
+        }
     }
 
     TS(11);
@@ -1356,7 +1388,25 @@ k_verify(VerifyArgs a) {
             if (!extra_err && warp == 0) finish_supports(wsx, false, lane);
         }
     }
-    if (extra && warp == 0) {
+    if (extra && a.top_k == 0) {
+        // W_nom independent draws from p_beam, one warp each
+        const int cap = a.out.out_off[r + 1] - a.out.out_off[r];
+        const int n_draw = min(W_nom, max(cap - n_out, 0));
+        if (writer && threadIdx.x == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
+        for (int kk = warp; kk < n_draw; kk += kWarps) {
+            const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1) + a.extra_layer_bias, 3u,
+                                              (uint32_t)kk);
+            int ia = 0;
+            const int tok = draw_cell(a, sh, u, false, 0.f, 0.0, nullptr, lane, &ia);
+            if (tok < 0) { if (lane == 0) sh.err = DSBD_DEV_EXHAUSTED; }
+            else if (lane == 0 && writer) emit_at(a, r, n_out + kk, sh.A[ia], -1, tok, DSBD_SRC_EXTRA);
+        }
+        __syncthreads();
+        if (!sh.err) {
+            n_out += n_draw;
+            if (W_nom > n_draw && threadIdx.x == 0) sh.err = DSBD_DEV_CAPACITY;
+        }
+    } else if (extra && warp == 0) {
         int err = extra_err;
         if (writer && lane == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
         for (int kk = 0; kk < W_nom && !err; ++kk) {
