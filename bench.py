@@ -183,7 +183,7 @@ def _host_views(data, spec):
                 h(data["v_new"][n0:n1]), h(data["k_prefix"][s:e]), h(data["v_prefix"][s:e]),
                 np.array([0, poff[b + 1] - poff[b]], np.int64))
 
-    return dict(forest=forest, verify_sub=verify_sub, attn_sub=attn_sub, max_reqs=8, max_beams=8)
+    return dict(forest=forest, verify_sub=verify_sub, attn_sub=attn_sub, max_reqs=48, max_beams=256)
 
 
 def run_reference(args):
