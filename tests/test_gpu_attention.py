@@ -90,7 +90,7 @@ def test_ragged_prefixes_and_tree_shapes(dtype, Hq, Hkv, d):
     attention_close(to_host_f32(out), ref, bf16=dtype == torch.bfloat16)
 
 
-@pytest.mark.parametrize("Hq,Hkv,max_nodes", [(8, 2, 32), (16, 2, 16), (4, 4, 64), (32, 8, 9)])
+@pytest.mark.parametrize("Hq,Hkv,max_nodes", [(8, 2, 32), (16, 2, 16), (4, 4, 64), (32, 8, 9), (40, 40, 20)])
 def test_tensor_core_kernel_row_counts(Hq, Hkv, max_nodes):
     """bf16, d = 128: the tcgen05 kernel with 64-row and with 128-row query tiles (nodes x group
     up to 128), ragged prefixes around its 64-token tiles."""
