@@ -9,7 +9,9 @@ cache of the input beam it descends from, extended by the keys/values of the for
 its path.  Section "Reducing Memory Cost": optionally only the output beam of lowest
 perplexity is kept per request, so that a single cache survives.
 
-Conventions (the paper fixes none of them; they mirror the attention's layout):
+Conventions (the paper fixes none of them, so the numbering of the kept beams and the tie rule
+are "parity unpinned"; the content of each cache is pinned through the attention; they mirror
+the attention's layout):
   * the cache of a beam holds every token of the beam except its last one (the last token is
     the root of the beam's next draft tree and brings its own key/value);
   * an output beam (parent node n, new token x) therefore keeps: cache of its input beam, then

@@ -9,7 +9,8 @@ say how a cache is stored.  Here a cache is a list of pages of PAGE = 64 tokens 
 only the last, partly filled page is private.  What a paged cache *means* is its gathered
 content, and that is what pins this file: gathering must give the packed oracle's result.
 
-Conventions of the commit (nothing in the paper; the CUDA path has to match them):
+Conventions of the commit (nothing in the paper fixes them, so the page ids are "parity
+unpinned": only the gathered content is pinned; the CUDA path has to match them):
   * kept output beams are selected and numbered exactly as in oracle.kv_commit;
   * new beam j keeps the first L_old // PAGE pages of its input beam, then gets
     ceil((L_old % PAGE + path length) / PAGE) fresh pages that hold the input beam's partial
