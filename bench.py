@@ -341,6 +341,34 @@ def main():
     torch.cuda.synchronize()
     dense_ms = d0.elapsed_time(d1) / n_dense
 
+    # the same step replayed from a CUDA graph (launch overhead removed; the decode-step counter is
+    # a call argument and therefore frozen into the graph, so this is a latency figure only)
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            stream_saved, stream = stream, side
+            with torch.cuda.graph(g, stream=side):
+                one_step(args.warmup)
+            stream = stream_saved
+        torch.cuda.synchronize()
+        for _ in range(3):
+            g.replay()
+        r0 = torch.cuda.Event(enable_timing=True); r1 = torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(args.steps):
+            g.replay()
+        r1.record()
+        torch.cuda.synchronize()
+        graph_ms = r0.elapsed_time(r1) / args.steps
+        del g
+    except Exception as e:                                   # a figure beside the metric: never fatal
+        print("graph replay skipped: %r" % (e,), file=sys.stderr)
+        stream = torch.cuda.current_stream()
+    assert int(status.item()) == 0, "device status %d" % int(status.item())
+
     # the KV-cache update of the step's output beams (reported beside the step, not part of it)
     esz = data["k_new"].element_size()
     n_slots = int(out_off[-1])
@@ -536,7 +564,8 @@ def main():
                            (a_bytes + v_bytes) * 1e-9),
                        "parallelism": "replicas x%d" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "kernels": kernels, "verify_stats_last_step": verify_stats, "cpu_baseline": cpu}
+            "roofline": roofline, "kernels": kernels, "graph_replay_ms_per_step": graph_ms,
+            "verify_stats_last_step": verify_stats, "cpu_baseline": cpu}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
