@@ -300,6 +300,23 @@ int dsbd_draft_layer(int32_t R, int32_t n_beams, const int32_t *req_beam_off,
 
 size_t dsbd_draft_workspace(int32_t R, int32_t n_beams, const dsbd_draft_params_t *params);
 
+/* The draft forest from the draft stage's draws (Section "Overview": the small model's beam
+ * sampling of width W_S over gamma steps traces a forest of W_L trees, one per input beam, every
+ * later layer holding W_S nodes).  draw_parent / draw_token: [gamma][R * W_S], layer l (1-based)
+ * at offset (l-1)*R*W_S, request r's draws at r*W_S .. as dsbd_draft_layer wrote them with
+ * out_off[r] = r*W_S: for l = 1 the parent is a global input-beam index, for l > 1 the index
+ * r*W_S + k' of a draw of layer l-1.  Output (device arrays sized for N = B + gamma*R*W_S nodes):
+ * the forest in the layout dsbd_forest_t describes -- trees beam-major, a tree's nodes contiguous,
+ * the root first and then its draws in (layer, draw) order, so parent[n] < n -- with
+ * draft_rank[n] = the draw index k, beam_node_off [B+1], and node_of_draw [gamma][R * W_S]: the node
+ * each draw became (to place the models' rows).  Node numbering inside a tree is a convention of
+ * this library; any topological order would do.  gamma * W_S <= 1024, beams per request <=
+ * DSBD_MAX_LIVE.  *status: DSBD_DEV_BAD_FOREST when a draw names a beam of another request. */
+int dsbd_forest_build(int32_t R, int32_t gamma, int32_t W_S, const int32_t *req_beam_off,
+                      const int32_t *draw_parent, const int32_t *draw_token,
+                      int32_t *beam_node_off, int32_t *parent, int32_t *token, int32_t *draft_rank,
+                      int32_t *node_of_draw, int32_t *status, dsbd_stream_t stream);
+
 /* KV-cache update at the end of a decode step (Section "Forest-based Parallel Decoding": after
  * the iteration the key-value caches are updated according to the output beams, an output beam
  * keeping the cache of the input beam it descends from; Section "Reducing Memory Cost": keeping

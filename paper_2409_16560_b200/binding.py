@@ -23,6 +23,7 @@ EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_for
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
            "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_draft_layer", "dsbd_draft_workspace",
            "dsbd_forest_attention_paged", "dsbd_kv_commit_paged", "dsbd_kv_commit_paged_workspace",
+           "dsbd_forest_build",
            "dsbd_status_string"]
 
 _vp = C.c_void_p
@@ -103,6 +104,8 @@ def load():
     lib.dsbd_kv_commit_paged_workspace.argtypes = [_vp, _vp, C.c_int64]
     lib.dsbd_kv_commit_paged.restype = C.c_int
     lib.dsbd_kv_commit_paged.argtypes = [_vp] * 22 + [C.c_size_t, _vp, _vp]
+    lib.dsbd_forest_build.restype = C.c_int
+    lib.dsbd_forest_build.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [_vp] * 10
     lib.dsbd_draft_workspace.restype = C.c_size_t
     lib.dsbd_draft_workspace.argtypes = [C.c_int32, C.c_int32, _vp]
     lib.dsbd_draft_layer.restype = C.c_int
@@ -143,6 +146,18 @@ def _require_cuda(*tensors):
 
 class Forest:
     """Device copy of a draft forest plus the host-side facts the launches are sized by."""
+
+    @classmethod
+    def from_device(cls, R, B, N, max_depth, dev_arrays, max_tree_nodes, max_req_beams, max_layer_nodes):
+        """A forest whose arrays are already on the device; the launch facts are given as bounds."""
+        self = cls.__new__(cls)
+        self.R, self.B, self.N, self.max_depth = int(R), int(B), int(N), int(max_depth)
+        self.host = None
+        self.dev = dict(dev_arrays)
+        self.dev.setdefault("draft_rank", None)
+        self.max_tree_nodes, self.max_req_beams = int(max_tree_nodes), int(max_req_beams)
+        self.max_layer_nodes = int(max_layer_nodes)
+        return self
 
     def __init__(self, arrays, device):
         a = {k: np.ascontiguousarray(arrays[k], dtype=np.int32)
@@ -227,6 +242,31 @@ def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_pre
     if rc != OK:
         raise DsbdError("dsbd_forest_attention", rc)
     return out, status
+
+
+def forest_build(req_beam_off, req_beam_off_host, gamma, W_S, draw_parent, draw_token, status=None, stream=None):
+    """dsbd_forest_build.  draw_parent / draw_token: int32 device tensors [gamma, R*W_S].  Returns a
+    Forest whose arrays live on the device (host-side launch facts are the static bounds
+    1 + gamma*W_S nodes per tree and W_S nodes per layer), node_of_draw and the status tensor."""
+    _require_cuda(req_beam_off, draw_parent, draw_token)
+    dev = draw_parent.device
+    rbo = np.asarray(req_beam_off_host)
+    R, B = len(rbo) - 1, int(rbo[-1])
+    N = B + gamma * R * W_S
+    i32 = lambda n: torch.empty(n, dtype=torch.int32, device=dev)
+    arrays = dict(req_beam_off=req_beam_off, beam_node_off=i32(B + 1), parent=i32(N), token=i32(N),
+                  draft_rank=i32(N))
+    node_of_draw = torch.empty(gamma, R * W_S, dtype=torch.int32, device=dev)
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rc = load().dsbd_forest_build(R, gamma, W_S, _ptr(req_beam_off), _ptr(draw_parent), _ptr(draw_token),
+                                  _ptr(arrays["beam_node_off"]), _ptr(arrays["parent"]), _ptr(arrays["token"]),
+                                  _ptr(arrays["draft_rank"]), _ptr(node_of_draw), _ptr(status), _stream(stream))
+    if rc != OK:
+        raise DsbdError("dsbd_forest_build", rc)
+    f = Forest.from_device(R, B, N, gamma, arrays, max_tree_nodes=1 + gamma * W_S,
+                           max_req_beams=int(np.diff(rbo).max()), max_layer_nodes=W_S)
+    return f, node_of_draw, status
 
 
 class KvPagesT(C.Structure):

@@ -7,7 +7,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 BUILD_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(BUILD_DIR, "libdsbd.so")
-SOURCES = ["dsbd_api.cu", "dsbd_verify.cu", "dsbd_attention.cu", "dsbd_attention_tc.cu", "dsbd_kv_commit.cu"]
+SOURCES = ["dsbd_api.cu", "dsbd_verify.cu", "dsbd_attention.cu", "dsbd_attention_tc.cu", "dsbd_kv_commit.cu", "dsbd_forest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xptxas=-v", "-Xcompiler", "-fPIC",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("DSBD_NVCC_EXTRA", "").split()
