@@ -833,7 +833,9 @@ k_verify(VerifyArgs a) {
     unsigned long long *ghist = a.hist + (int64_t)r * 2 * (kBins + 1);     // [2 banks][kBins+1]
     const int hist_len = kBins + 1;
     int n_out = 0;
-    int ts_n = 0; (void)ts_n;
+#ifdef DSBD_PHASE_TIMING
+    int ts_n = 0;
+#endif
 
     TS(1);
     if (!a.select_mode) {
