@@ -100,6 +100,12 @@ def test_many_draws_follow_the_stream():
         _case(rng, [4, 2, 7], 3000, 64, 1, step=step)
 
 
+def test_the_largest_live_set():
+    rng = np.random.default_rng(8)
+    _case(rng, [64, 1, 64], 4096, 64, 5)
+    _case(rng, [64, 64], 1500, 64, 2, top_k=64, top_p=0.9)
+
+
 def test_capacity_error_is_per_request():
     rng = np.random.default_rng(6)
     rbo, z, s = _problem(rng, [2, 3], 1000)
