@@ -345,6 +345,14 @@ typedef struct {
     int32_t n_slots;
     int32_t keep_best;
     int64_t dst_capacity;
+    /* dsbd_kv_commit_paged only: the caches of all transformer layers in one call.  Every layer
+     * has its own pools and its own k_new / v_new, at the same address offsets from layer to
+     * layer, and all layers share the page tables (a page id means the same slot in every
+     * layer's pool), so the plan, the tables and the allocator update are made once.
+     * n_layers 0 or 1: a single layer. */
+    int32_t n_layers;
+    int64_t pool_layer_stride;     /* elements between consecutive layers' pools            */
+    int64_t new_layer_stride;      /* elements between consecutive layers' k_new / v_new    */
 } dsbd_commit_params_t;
 
 int dsbd_kv_commit(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,

@@ -349,7 +349,8 @@ def draft_layer(req_beam_off, req_beam_off_host, params, layer, W_S, logits_q, b
 
 
 class CommitParamsT(C.Structure):
-    _fields_ = [("n_slots", C.c_int32), ("keep_best", C.c_int32), ("dst_capacity", C.c_int64)]
+    _fields_ = [("n_slots", C.c_int32), ("keep_best", C.c_int32), ("dst_capacity", C.c_int64),
+                ("n_layers", C.c_int32), ("pool_layer_stride", C.c_int64), ("new_layer_stride", C.c_int64)]
 
 
 def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out_logp, k_new, v_new,
@@ -394,7 +395,9 @@ def kv_commit(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out
 def kv_commit_paged(forest, Hkv, d, out_off, out_width, out_parent, out_root_beam, out_logp, k_new, v_new,
                     k_pool, v_pool, page_table, page_off, prefix_off, prefix_off_host, free_stack, free_count,
                     n_slots, table_capacity, keep_best=False, workspace=None, status=None, stream=None, out=None):
-    """dsbd_kv_commit_paged; the pools, free_stack and free_count are updated in place.  Returns a
+    """dsbd_kv_commit_paged; the pools, free_stack and free_count are updated in place.  Pools of
+    shape [n_layers, n_pages, Hkv, 64, d] with k_new / v_new [n_layers, N, Hkv, d] update all
+    layers in one call (the layers share the page tables).  Returns a
     dict with new_req_beam_off, new_prefix_off, new_page_off, new_page_table, new_beam_slot and the
     status tensor (device tensors, nothing is synchronised)."""
     _require_cuda(out_off, out_width, out_parent, out_root_beam, k_new, v_new, k_pool, v_pool, page_table,
@@ -405,7 +408,13 @@ def kv_commit_paged(forest, Hkv, d, out_off, out_width, out_parent, out_root_bea
     p = CommitParamsT()
     p.n_slots, p.keep_best, p.dst_capacity = int(n_slots), int(bool(keep_best)), int(table_capacity)
     pages = KvPagesT()
-    pages.page_table, pages.page_off, pages.n_pages = _ptr(page_table), _ptr(page_off), int(k_pool.shape[0])
+    if k_pool.dim() == 5:
+        p.n_layers = int(k_pool.shape[0])
+        p.pool_layer_stride = int(k_pool.stride(0))
+        p.new_layer_stride = int(k_new.stride(0))
+        assert k_new.dim() == 4 and k_new.shape[0] == p.n_layers
+    pages.page_table, pages.page_off = _ptr(page_table), _ptr(page_off)
+    pages.n_pages = int(k_pool.shape[-4])
     need = int(load().dsbd_kv_commit_paged_workspace(C.addressof(f), C.addressof(p), pages.n_pages))
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)

@@ -60,6 +60,7 @@ struct CommitArgs {
     int64_t *new_page_off;
     int32_t *free_stack, *free_count;
     int32_t *used;            // [n_pages + 1] workspace
+    int64_t pool_layer_bytes, new_layer_bytes;   // several layers: blockIdx.y is the layer
     // workspace
     Plan *plan;
     int32_t *req_count;       // [R]     kept beams of the request, then its first new beam
@@ -303,14 +304,15 @@ k_commit_pages(CommitArgs a) {
     const int32_t *old_pages = a.page_table + a.page_off[b];
     const int32_t *fresh = a.free_stack + (*a.free_count - 1 - a.chunk_off[j]);     // fresh page i = fresh[-i]
     int32_t *table = a.new_page_table + a.new_page_off[j];
-    if (g == 0 && kv == 0) {
+    if (g == 0 && kv == 0 && blockIdx.y == 0) {
         for (int i = threadIdx.x; i < full; i += blockDim.x) table[i] = old_pages[i];
         for (int i = threadIdx.x; i < n_fresh; i += blockDim.x) table[full + i] = fresh[-i];
     }
     const int rb = a.row_bytes, upr = rb / 16;                   // 16-byte units per row
-    const unsigned char *pool_in = kv ? a.v_prefix : a.k_prefix;
-    unsigned char *pool_out = kv ? a.v_dst : a.k_dst;
-    const unsigned char *src_new = kv ? a.v_new : a.k_new;
+    const int64_t pool_shift = (int64_t)blockIdx.y * a.pool_layer_bytes;
+    const unsigned char *pool_in = (kv ? a.v_prefix : a.k_prefix) + pool_shift;
+    unsigned char *pool_out = (kv ? a.v_dst : a.k_dst) + pool_shift;
+    const unsigned char *src_new = (kv ? a.v_new : a.k_new) + (int64_t)blockIdx.y * a.new_layer_bytes;
     const int32_t *path = a.path + (int64_t)j * (a.gamma + 1);
     const int64_t part_row0 = rem ? ((int64_t)old_pages[full] * a.Hkv + g) * kPage : 0;
     const int units = n_fresh * kPage * upr;
@@ -499,6 +501,11 @@ extern "C" int dsbd_kv_commit_paged(const dsbd_forest_t *f, const dsbd_attn_desc
     if (desc->Hkv <= 0 || desc->d <= 0) return DSBD_ERR_INVALID_ARG;
     if (desc->dtype != DSBD_DTYPE_BF16 && desc->dtype != DSBD_DTYPE_F32) return DSBD_ERR_UNSUPPORTED;
     if (pages->n_pages >= (int64_t)1 << 31) return DSBD_ERR_UNSUPPORTED;
+    if (p->n_layers > 1 && (p->pool_layer_stride <= 0 || p->new_layer_stride <= 0 ||
+                            (p->pool_layer_stride * (desc->dtype == DSBD_DTYPE_BF16 ? 2 : 4)) % 16 ||
+                            (p->new_layer_stride * (desc->dtype == DSBD_DTYPE_BF16 ? 2 : 4)) % 16 ||
+                            p->n_layers > 65535))
+        return DSBD_ERR_INVALID_ARG;
     const int row_bytes = desc->d * (desc->dtype == DSBD_DTYPE_BF16 ? 2 : 4);
     if (row_bytes % 16) return DSBD_ERR_UNSUPPORTED;
     const uintptr_t ptrs = reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
@@ -538,7 +545,11 @@ extern "C" int dsbd_kv_commit_paged(const dsbd_forest_t *f, const dsbd_attn_desc
     a.status = status;
 
     k_commit_plan<<<1, kPlanThreads, 0, stream>>>(a);
-    k_commit_pages<<<(unsigned)(p->n_slots * desc->Hkv * 2), kCopyThreads, 0, stream>>>(a);
+    const int n_layers = p->n_layers > 1 ? p->n_layers : 1;
+    const int esz = desc->dtype == DSBD_DTYPE_BF16 ? 2 : 4;
+    a.pool_layer_bytes = p->pool_layer_stride * esz;
+    a.new_layer_bytes = p->new_layer_stride * esz;
+    k_commit_pages<<<dim3((unsigned)(p->n_slots * desc->Hkv * 2), (unsigned)n_layers), kCopyThreads, 0, stream>>>(a);
     k_commit_free<<<1, kPlanThreads, 0, stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }

@@ -195,3 +195,51 @@ def test_paged_commit_without_free_pages_changes_nothing():
     assert int(res["status"].item()) == 3
     assert torch.equal(dk, before) and int(d_nfree.item()) == nfree
     assert np.array_equal(d_free.cpu().numpy(), free)
+
+
+def test_paged_commit_of_several_layers_shares_the_tables():
+    """Three transformer layers: one call, one plan, one set of page tables; every layer's pools
+    must gather to what the oracle gives for that layer alone."""
+    rng = np.random.default_rng(21)
+    Hkv, d, n_layers, n_pages = 2, 128, 3, 40
+    rbo = np.array([0, 2, 5], np.int32)
+    L = [70, 70, 200, 200, 200]
+    poff = np.concatenate([[0], np.cumsum(L)]).astype(np.int64)
+    g = torch.Generator(device="cuda"); g.manual_seed(2)
+    mk = lambda *s: torch.randn(*s, generator=g, device="cuda").to(torch.bfloat16)
+    forest = _forest_on(rng, rbo, 5)
+    outs = _outputs(rng, forest, 3)
+    hosts, dks, dvs, kns, vns = [], [], [], [], []
+    ids = rng.permutation(n_pages)
+    for layer in range(n_layers):
+        kp, vp = mk(int(poff[-1]) * Hkv * d), mk(int(poff[-1]) * Hkv * d)
+        # the same page ids in every layer: seed the shuffle identically
+        hk, hv, table, page_off, free, nfree = kvp.pack_into_pages(_bits(kp), _bits(vp), poff, Hkv, d, n_pages,
+                                                                   np.random.default_rng(77))
+        hosts.append((hk, hv))
+        dks.append(_from_bits(hk, torch.bfloat16)); dvs.append(_from_bits(hv, torch.bfloat16))
+        kns.append(mk(forest["N"], Hkv, d)); vns.append(mk(forest["N"], Hkv, d))
+    dk, dv = torch.stack(dks).cuda(), torch.stack(dvs).cuda()
+    kn, vn = torch.stack(kns), torch.stack(vns)
+    i32 = lambda a: torch.as_tensor(np.asarray(a, np.int32)).cuda()
+    d_free, d_nfree = torch.as_tensor(free).cuda(), torch.tensor([nfree], dtype=torch.int32, device="cuda")
+    refs = [kvp.kv_commit_paged(forest, *outs, _bits(kns[l]), _bits(vns[l]), hosts[l][0], hosts[l][1], table,
+                                page_off, poff, free, nfree) for l in range(n_layers)]
+    assert all(r["error"] == 0 for r in refs)
+    res = dsbd.kv_commit_paged(dsbd.Forest(forest, "cuda"), Hkv, d, i32(outs[0]), i32(outs[1]), i32(outs[2]),
+                               i32(outs[3]), None, kn, vn, dk, dv, torch.as_tensor(table).cuda(),
+                               torch.as_tensor(page_off).cuda(), torch.as_tensor(poff).cuda(), poff, d_free, d_nfree,
+                               n_slots=int(outs[0][-1]), table_capacity=len(refs[0]["new_page_table"]))
+    torch.cuda.synchronize()
+    assert int(res["status"].item()) == 0
+    nt = len(refs[0]["new_page_table"])
+    for l in range(n_layers):
+        ref = refs[l]
+        assert np.array_equal(ref["new_page_table"], refs[0]["new_page_table"])
+        assert np.array_equal(res["new_page_table"].cpu().numpy()[:nt], ref["new_page_table"])
+        gk, gv = kvp.gather(_bits(dk[l]).reshape(hosts[l][0].shape), _bits(dv[l]).reshape(hosts[l][1].shape),
+                            ref["new_page_table"], ref["new_page_off"], ref["new_prefix_off"])
+        wk, wv = kvp.gather(ref["k_pool"], ref["v_pool"], ref["new_page_table"], ref["new_page_off"],
+                            ref["new_prefix_off"])
+        assert np.array_equal(gk, wk) and np.array_equal(gv, wv), l
+    assert int(d_nfree.item()) == refs[0]["free_count"]
