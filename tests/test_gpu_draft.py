@@ -61,6 +61,12 @@ def _compare(ref, gpu, W_r, out_off):
             x, y = ref["out_logq"][s], gpu["out_logq"][s]
             assert abs(x - y) <= 1e-4 + 1e-5 * abs(x), (r, k, x, y)
     assert exempt <= math.ceil(1e-4 * draws), (exempt, draws)
+    # slots past a request's W_S draws keep their initial -1
+    used = np.zeros(len(gpu["out_token"]), bool)
+    for r in range(len(W_r)):
+        # (a request that reported an error leaves its own slot range unspecified)
+        used[out_off[r]:(out_off[r + 1] if ref["error"][r] else out_off[r] + W_r[r])] = True
+    assert (gpu["out_token"][~used] == -1).all() and (gpu["out_parent"][~used] == -1).all()
     return draws
 
 

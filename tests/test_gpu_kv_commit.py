@@ -49,11 +49,12 @@ def _run_both(data, outs, keep_best, capacity=None):
     cap = total + 7 if capacity is None else capacity
     f = dsbd.Forest(forest, "cuda")
     dv = lambda a, dt: torch.as_tensor(np.asarray(a), dtype=dt).cuda()
+    canary = lambda: torch.full((cap * Hkv * d,), 7.0, dtype=data["k_new"].dtype, device="cuda")
     res = dsbd.kv_commit(f, Hkv, d, dv(out_off, torch.int32), dv(out_width, torch.int32),
                          dv(out_parent, torch.int32), dv(out_root, torch.int32), dv(out_logp, torch.float32),
                          data["k_new"], data["v_new"], data["k_prefix"], data["v_prefix"],
                          torch.as_tensor(poff).cuda(), poff, n_slots=int(out_off[-1]), dst_capacity=cap,
-                         keep_best=keep_best)
+                         keep_best=keep_best, k_dst=canary(), v_dst=canary())
     torch.cuda.synchronize()
     return ref, res, total
 
@@ -70,6 +71,8 @@ def _compare(ref, res, total, spec):
     n = total * spec["Hkv"] * spec["d"]
     assert np.array_equal(_bits(res["k_dst"])[:n], ref["k_cache"])
     assert np.array_equal(_bits(res["v_dst"])[:n], ref["v_cache"])
+    # nothing is written past the kept caches
+    assert bool((res["k_dst"][n:] == 7.0).all()) and bool((res["v_dst"][n:] == 7.0).all())
 
 
 @pytest.mark.parametrize("name,kw", [("C1", {}), ("C2", {}), ("C3", {}), ("C4", {}), ("C5", dict(R=6))])
