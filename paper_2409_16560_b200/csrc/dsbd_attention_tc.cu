@@ -52,11 +52,14 @@ constexpr long long kWaitCycles = 2000000000ll;   // about a second
 // One work item: the query rows of unit (b, g) against the prefix tokens [t0, t1) of its beam,
 // plus the tree tile when `last`.  A unit split into several items leaves partial results
 // (reference maximum, row sum, unnormalised O) that a second kernel merges.
-struct AttnItem { int b, g, t0, t1, last, nparts, slot, pad; };
+// Trees with more than 128 query rows (nodes x query heads per KV head) are cut into row blocks
+// of 128 rows; every row block is an item of its own that streams the same keys and values.
+struct AttnItem { int b, g, t0, t1, last, nparts, slot, rb; };
 
 struct TcArgs {
     int B, N, Hq, Hkv, group, n_units;
     int max_rows;                     // max over trees of nodes * group
+    int row_blocks;                   // ceil(max_rows / 128)
     const AttnItem *items;            // nullptr: one item per unit, in unit order
     const int *n_items;               // device count of items (with items)
     float *partial;                   // [slot][max_rows][130]: m_ref, l, O[128]
@@ -176,13 +179,25 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
            ((uint32_t)(M >> 4) << 24);
 }
 
-__device__ __forceinline__ int item_count(const TcArgs &a) { return a.items ? *a.n_items : a.n_units; }
+__device__ __forceinline__ int item_count(const TcArgs &a) {
+    return a.items ? *a.n_items : a.n_units * a.row_blocks;
+}
+// The item, with b = -1 when there is nothing to do: a padding entry of the plan, or a row block
+// beyond the rows of this tree.  All three roles of the CTA skip such items alike.
 __device__ __forceinline__ AttnItem get_item(const TcArgs &a, int it) {
-    if (a.items) return a.items[it];
     AttnItem x;
-    x.b = it / a.Hkv; x.g = it - x.b * a.Hkv;
-    x.t0 = 0; x.t1 = (int)(a.prefix_off[x.b + 1] - a.prefix_off[x.b]);
-    x.last = 1; x.nparts = 1; x.slot = 0; x.pad = 0;
+    if (a.items) {
+        x = a.items[it];
+    } else {
+        const int u = it / a.row_blocks;
+        x.rb = it - u * a.row_blocks;
+        x.b = u / a.Hkv; x.g = u - x.b * a.Hkv;
+        x.t0 = 0; x.t1 = (int)(a.prefix_off[x.b + 1] - a.prefix_off[x.b]);
+        x.last = 1; x.nparts = 1; x.slot = 0;
+    }
+    if (x.b >= 0 && x.rb > 0 &&
+        x.rb * kRows >= (a.beam_node_off[x.b + 1] - a.beam_node_off[x.b]) * a.group)
+        x.b = -1;
     return x;
 }
 
@@ -346,18 +361,19 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const int n_lo = a.beam_node_off[b];
             const int n_tree = a.beam_node_off[b + 1] - n_lo;
             const int M = n_tree * a.group;
-            const bool warp_active = warp * 32 < M;
-            const bool active = row < M;
-            const int node = active ? row / a.group : 0;
-            const int hq = g * a.group + (active ? row - node * a.group : 0);
+            const int r0 = item.rb * kRows;                     // first row of this row block
+            const bool warp_active = r0 + warp * 32 < M;
+            const bool active = r0 + row < M;
+            const int node = active ? (r0 + row) / a.group : 0;
+            const int hq = g * a.group + (active ? r0 + row - node * a.group : 0);
             // ---- stage Q (rows >= M zero) and the ancestor masks; the previous unit's MMAs are done
             {
                 const int t128 = threadIdx.x;                        // 0..127
                 for (int i = t128; i < QROWS * 16; i += 128) {
                     const int r = i >> 4, c = i & 15;                // row, 16-byte chunk of the 256-byte row
                     uint4 v = make_uint4(0, 0, 0, 0);
-                    if (r < M) {
-                        const int nd = r / a.group, hh = g * a.group + (r - nd * a.group);
+                    if (r0 + r < M) {
+                        const int nd = (r0 + r) / a.group, hh = g * a.group + (r0 + r - nd * a.group);
                         v = *reinterpret_cast<const uint4 *>(a.q + ((int64_t)(n_lo + nd) * a.Hq + hh) * kD + c * 8);
                     }
                     const int half = c >> 3, cc = c & 7;
@@ -472,7 +488,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     }
                 } else {
                     // partial result of this part of the unit: reference maximum, row sum, raw O
-                    float *dst = a.partial + ((int64_t)item.slot * a.max_rows + row) * 130;
+                    float *dst = a.partial + ((int64_t)item.slot * a.max_rows + r0 + row) * 130;
                     if (active) { dst[0] = m_ref; dst[1] = l_run; }
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
@@ -516,7 +532,7 @@ __device__ __forceinline__ void unit_parts(int64_t L, int chunk, int *np, int *p
 }
 
 __global__ void __launch_bounds__(1024)
-k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, int grid,
+k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, int grid, int row_blocks,
             AttnItem *__restrict__ items, int *__restrict__ n_items, UnitParts *__restrict__ units) {
     __shared__ int bucket[1024];
     __shared__ int scan[1024];
@@ -550,7 +566,7 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, i
                 const int64_t t0 = (int64_t)p * plen;
                 const int64_t t1 = t0 + plen < L ? t0 + plen : L;
                 int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
-                atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
+                atomicAdd(&bucket[nt < 1023 ? nt : 1023], row_blocks);
             }
         }
         __syncthreads();
@@ -572,7 +588,7 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, i
     // The list is read in rounds of `grid` items, CTA k taking entry k of every round.  Odd rounds
     // are stored back to front, so that the CTA with the longest item of one round gets the
     // shortest of the next; the last round is padded with empty entries (b = -1).
-    const int total_items = carry;
+    const int total_items = carry * row_blocks;
     const int padded = (total_items + grid - 1) / grid * grid;
     for (int i = total_items - total_items % grid + tid; i < padded; i += 1024) items[i].b = -1;
     if (tid == 0) *n_items = padded;
@@ -586,13 +602,15 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, i
             const int64_t t0 = (int64_t)p * plen;
             const int64_t t1 = t0 + plen < L ? t0 + plen : L;
             const int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
-            int pos = atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
-            const int round = pos / grid;
-            if (round & 1) pos = round * grid + (grid - 1 - (pos - round * grid));
-            AttnItem it;
-            it.b = b; it.g = g; it.t0 = (int)t0; it.t1 = (int)t1; it.last = (p == np - 1);
-            it.nparts = np; it.slot = units[u].first_slot + p; it.pad = 0;
-            items[pos] = it;
+            for (int rb = 0; rb < row_blocks; ++rb) {
+                int pos = atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
+                const int round = pos / grid;
+                if (round & 1) pos = round * grid + (grid - 1 - (pos - round * grid));
+                AttnItem it;
+                it.b = b; it.g = g; it.t0 = (int)t0; it.t1 = (int)t1; it.last = (p == np - 1);
+                it.nparts = np; it.slot = units[u].first_slot + p; it.rb = rb;
+                items[pos] = it;
+            }
         }
     }
 }
@@ -675,7 +693,8 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     const int group = d->Hq / d->Hkv;
     const bool small_q = f->max_tree_nodes * group <= 64;
     p.grid = small_q ? 2 * sms : sms;
-    const int64_t n_units = (int64_t)f->B * d->Hkv;
+    const int row_blocks = (f->max_tree_nodes * group + kRows - 1) / kRows;
+    const int64_t n_units = (int64_t)f->B * d->Hkv * row_blocks;     // counted with their row blocks
     // Splitting a unit costs a pipeline drain, a Q reload and a partial result per part, so it
     // pays only when there are fewer units than CTAs: then the prefix is cut so that about two
     // items per CTA exist, in parts of at least 512 tokens.  Ragged batches with enough units
@@ -694,12 +713,12 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     }
     if (!p.split) c = (int64_t)1 << 30;                  // one part per unit
     p.chunk = (int)c;
-    p.items_max = (p.split ? (int64_t)d->Hkv * (d->total_prefix / c + f->B) : n_units) + p.grid;
+    p.items_max = (p.split ? (int64_t)d->Hkv * row_blocks * (d->total_prefix / c + f->B) : n_units) + p.grid;
     if (p.grid > p.items_max - p.grid) p.grid = (int)(p.items_max - p.grid);
     if (p.grid < 1) p.grid = 1;
     size_t off = 256;
     p.off_items = off;   off = align_up(off + sizeof(AttnItem) * (size_t)p.items_max, 256);
-    p.off_units = off;   off = align_up(off + sizeof(UnitParts) * (size_t)n_units, 256);
+    p.off_units = off;   off = align_up(off + sizeof(UnitParts) * (size_t)f->B * d->Hkv, 256);
     p.off_partial = off;
     if (p.split)
         off = align_up(off + sizeof(float) * 130 * (size_t)p.items_max * (size_t)(f->max_tree_nodes * group), 256);
@@ -713,7 +732,7 @@ namespace dsbd {
 
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages) {
     if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
-    if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows) return false;
+    if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows * 8) return false;      // up to 8 row blocks
     if (f->max_tree_nodes > kBN) return false;
     if (d->total_prefix <= 0) return false;
     // row coordinates of the K/V maps are 32-bit
@@ -746,6 +765,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;
     a.n_units = f->B * d->Hkv;
     a.max_rows = f->max_tree_nodes * a.group;
+    a.row_blocks = (a.max_rows + kRows - 1) / kRows;
     a.scale_log2 = d->scale * 1.4426950408889634f;
     a.beam_node_off = f->beam_node_off; a.parent = f->parent; a.prefix_off = prefix_off;
     if (pages) { a.page_table = pages->page_table; a.page_off = pages->page_off; }
@@ -758,7 +778,8 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
         AttnItem *items = reinterpret_cast<AttnItem *>(ws + plan.off_items);
         units = reinterpret_cast<UnitParts *>(ws + plan.off_units);
         int *n_items = reinterpret_cast<int *>(ws);
-        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, plan.chunk, plan.grid, items, n_items, units);
+        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, plan.chunk, plan.grid, a.row_blocks, items,
+                                            n_items, units);
         a.items = items;
         a.n_items = n_items;
         a.partial = reinterpret_cast<float *>(ws + plan.off_partial);

@@ -116,6 +116,25 @@ def test_few_units_long_prefix_is_split_and_merged(L):
     attention_close(to_host_f32(out), ref, bf16=True)
 
 
+@pytest.mark.parametrize("Hq,Hkv,sizes,L", [
+    (32, 2, [40, 1, 9, 64], [300, 64, 1000, 77]),        # 16 query heads per KV head: up to 1024 rows, 8 row blocks
+    (16, 4, [64, 33, 5], [129, 700, 63]),                # 256 and 132 rows next to a small tree
+    (8, 2, [50, 60], [6000, 4000]),                      # few units: row blocks of split units are merged
+    (24, 8, [45, 2, 45, 7, 30, 64, 12, 1], [900, 100, 2500, 64, 1, 333, 1500, 4000]),   # ragged: planned order
+])
+def test_trees_with_more_than_128_query_rows(Hq, Hkv, sizes, L):
+    """nodes x (query heads per KV head) > 128: the tensor-core kernel cuts the tree's query rows
+    into blocks of 128, each block an item of its own over the same keys and values."""
+    rng = np.random.default_rng(Hq + len(L))
+    rand_tree = lambda n: [-1] + [int(rng.integers(0, i)) for i in range(1, n)]
+    trees = [rand_tree(n) for n in sizes]
+    forest, spec, t, poff = _custom(rng, trees, L, Hq, Hkv, 128, torch.bfloat16)
+    assert dsbd.forest_attention_launches(dsbd.Forest(forest, "cuda"), Hq, Hkv, 128, torch.bfloat16, 0.1, poff) >= 1
+    out = _gpu(forest, spec, t, poff)
+    nodes, ref = _oracle_beams(forest, spec, t, poff, list(range(len(trees))))
+    attention_close(to_host_f32(out), ref, bf16=True)
+
+
 def test_host_side_errors():
     rng = np.random.default_rng(0)
     forest, spec, t, poff = _custom(rng, [[-1, 0]], [8], 4, 4, 64, torch.bfloat16)
