@@ -48,6 +48,8 @@ enum {
 
 /* limits of this build */
 #define DSBD_MAX_TREE_NODES 64   /* nodes per draft tree (forest attention)                  */
+#define DSBD_MAX_TREE_NODES_TC 128 /* the same on the tensor-core path (bf16, d = 128, up to
+                                      1024 query rows per tree and KV head)                  */
 #define DSBD_MAX_LIVE 64         /* beams of a request / live drafts of a layer (verify)     */
 
 /* The draft forest of one decode step (Section "Draft and Verification Scheme", Overview):
@@ -68,8 +70,8 @@ typedef struct {
                                       values, so a forest whose node numbering is not the draw
                                       order has to pass it.  NULL = ascending node id.       */
     /* host-side facts about the arrays above; they size launches and are trusted */
-    int32_t max_tree_nodes;        /* max_b nodes of tree b, <= DSBD_MAX_TREE_NODES for
-                                      dsbd_forest_attention                                  */
+    int32_t max_tree_nodes;        /* max_b nodes of tree b (an upper bound will do), <=
+                                      DSBD_MAX_TREE_NODES(_TC) for dsbd_forest_attention     */
     int32_t max_req_beams;         /* max_r trees of request r, <= DSBD_MAX_LIVE             */
     int32_t max_layer_nodes;       /* max over (request, depth >= 1) of the nodes at that
                                       depth, <= DSBD_MAX_LIVE                                */

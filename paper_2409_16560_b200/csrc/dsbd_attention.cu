@@ -215,7 +215,7 @@ int check(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     if (d->d != 64 && d->d != 128) return DSBD_ERR_UNSUPPORTED;
     if (d->dtype != DSBD_DTYPE_BF16 && d->dtype != DSBD_DTYPE_F32) return DSBD_ERR_UNSUPPORTED;
     if (f->max_tree_nodes <= 0) return DSBD_ERR_INVALID_ARG;
-    if (f->max_tree_nodes > DSBD_MAX_TREE_NODES) return DSBD_ERR_UNSUPPORTED;
+    if (f->max_tree_nodes > DSBD_MAX_TREE_NODES_TC) return DSBD_ERR_UNSUPPORTED;
     return DSBD_OK;
 }
 
@@ -253,6 +253,7 @@ extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_des
         return launch_attention_tc(f, d, q, k_new, v_new, k_prefix, v_prefix, prefix_off, out, workspace,
                                    workspace_bytes, status, stream);
 
+    if (f->max_tree_nodes > DSBD_MAX_TREE_NODES) return DSBD_ERR_UNSUPPORTED;      // CUDA-core kernel: 64-bit masks
     AttnArgs a = {};
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;
     a.scale_log2 = d->scale * 1.4426950408889634f;

@@ -201,6 +201,11 @@ __device__ __forceinline__ AttnItem get_item(const TcArgs &a, int it) {
     return x;
 }
 
+// Tiles of 64 tokens that hold the tree's own keys and values (trees of up to 128 nodes).
+__device__ __forceinline__ int tree_tiles(const TcArgs &a, int b) {
+    return (a.beam_node_off[b + 1] - a.beam_node_off[b] + kBN - 1) / kBN;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t *>(&v);
@@ -258,7 +263,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 int page_next = (pages && item.t1 > item.t0) ? pages[0] : 0;
                 const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
                 const int n_lo = a.beam_node_off[b];
-                const int nt = nt_p + item.last;
+                const int nt = nt_p + (item.last ? tree_tiles(a, b) : 0);
                 for (int j = 0; j < nt && ok; ++j, ++tile) {
                     const int s = tile % kStages;
                     const uint32_t par = (tile / kStages) & 1;
@@ -277,11 +282,11 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                         tma_load_2d(vs, &map_vp, 0, y, &sb.kv_full[s]);
                         tma_load_2d(vs + kTileBytes / 2, &map_vp, 64, y, &sb.kv_full[s]);
                     } else {
-                        const int x = g * kD;
-                        tma_load_2d(ks, &map_kn, x, n_lo, &sb.kv_full[s]);
-                        tma_load_2d(ks + kTileBytes / 2, &map_kn, x + 64, n_lo, &sb.kv_full[s]);
-                        tma_load_2d(vs, &map_vn, x, n_lo, &sb.kv_full[s]);
-                        tma_load_2d(vs + kTileBytes / 2, &map_vn, x + 64, n_lo, &sb.kv_full[s]);
+                        const int x = g * kD, y = n_lo + (j - nt_p) * kBN;      // tree tile j - nt_p
+                        tma_load_2d(ks, &map_kn, x, y, &sb.kv_full[s]);
+                        tma_load_2d(ks + kTileBytes / 2, &map_kn, x + 64, y, &sb.kv_full[s]);
+                        tma_load_2d(vs, &map_vn, x, y, &sb.kv_full[s]);
+                        tma_load_2d(vs + kTileBytes / 2, &map_vn, x + 64, y, &sb.kv_full[s]);
                     }
                 }
             }
@@ -307,7 +312,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
                 const AttnItem item = get_item(a, u);
                 if (item.b < 0) continue;
-                const int nt = (item.t1 - item.t0 + kBN - 1) / kBN + item.last;
+                const int nt = (item.t1 - item.t0 + kBN - 1) / kBN + (item.last ? tree_tiles(a, item.b) : 0);
                 ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
                 // S(t) = Q K(t)^T into S buffer t & 1; issued one tile ahead of the P V product so
                 // that it runs while the softmax warps work on the previous tile
@@ -357,9 +362,9 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const int b = item.b, g = item.g;
             const int64_t L = item.t1;                         // tokens beyond t1 belong to other items
             const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
-            const int nt = nt_p + item.last;
             const int n_lo = a.beam_node_off[b];
             const int n_tree = a.beam_node_off[b + 1] - n_lo;
+            const int nt = nt_p + (item.last ? (n_tree + kBN - 1) / kBN : 0);
             const int M = n_tree * a.group;
             const int r0 = item.rb * kRows;                     // first row of this row block
             const bool warp_active = r0 + warp * 32 < M;
@@ -383,11 +388,11 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 mbar_arrive(&sb.q_full);
             }
             // ancestor-or-self mask of this row's node: walk up the tree
-            unsigned long long my_anc = 0;
+            unsigned long long anc_lo = 0ull, anc_hi = 0ull;       // nodes 0..63, 64..127
             {
                 int n = node;
-                for (int hop = 0; hop < DSBD_MAX_TREE_NODES && n >= 0 && n < n_tree; ++hop) {
-                    my_anc |= 1ull << n;
+                for (int hop = 0; hop < 2 * kBN && n >= 0 && n < n_tree; ++hop) {
+                    if (n < 64) anc_lo |= 1ull << n; else anc_hi |= 1ull << (n - 64);
                     const int par = a.parent[n_lo + n];
                     if (par >= n_lo + n) { report(a.status, DSBD_DEV_BAD_FOREST); break; }
                     n = par < 0 ? -1 : par - n_lo;
@@ -405,10 +410,13 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     tmem_ld32(tmem + lane_base + s_col + 32, sv[1]);
                     tmem_wait_ld();
                     float mx = -INFINITY;
-                    const bool tree = (j == nt_p);
+                    const bool tree = (j >= nt_p);
                     // visibility of the tile's 64 tokens for this row, as a bit mask
                     unsigned long long vis;
-                    if (tree) vis = my_anc & (n_tree >= 64 ? ~0ull : ((1ull << n_tree) - 1));
+                    if (tree) {
+                        const int jt = j - nt_p, left = n_tree - jt * kBN;
+                        vis = (jt ? anc_hi : anc_lo) & (left >= 64 ? ~0ull : ((1ull << left) - 1));
+                    }
                     else {
                         const int64_t left = L - item.t0 - (int64_t)j * kBN;
                         vis = left >= 64 ? ~0ull : ((1ull << left) - 1);
@@ -733,7 +741,7 @@ namespace dsbd {
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages) {
     if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
     if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows * 8) return false;      // up to 8 row blocks
-    if (f->max_tree_nodes > kBN) return false;
+    if (f->max_tree_nodes > 2 * kBN) return false;                           // two tree tiles
     if (d->total_prefix <= 0) return false;
     // row coordinates of the K/V maps are 32-bit
     const int64_t rows = n_pages > 0 ? n_pages * d->Hkv * kBN : (int64_t)d->total_prefix * d->Hkv;

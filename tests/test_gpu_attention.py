@@ -121,6 +121,8 @@ def test_few_units_long_prefix_is_split_and_merged(L):
     (16, 4, [64, 33, 5], [129, 700, 63]),                # 256 and 132 rows next to a small tree
     (8, 2, [50, 60], [6000, 4000]),                      # few units: row blocks of split units are merged
     (24, 8, [45, 2, 45, 7, 30, 64, 12, 1], [900, 100, 2500, 64, 1, 333, 1500, 4000]),   # ragged: planned order
+    (8, 2, [128, 65, 100, 3], [500, 64, 1, 2000]),       # more than 64 nodes: two tiles of the tree's own K/V
+    (4, 4, [127, 66], [7000, 9000]),                     # the same with split units
 ])
 def test_trees_with_more_than_128_query_rows(Hq, Hkv, sizes, L):
     """nodes x (query heads per KV head) > 128: the tensor-core kernel cuts the tree's query rows

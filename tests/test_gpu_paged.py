@@ -73,8 +73,8 @@ def test_partial_pages_and_split_units(L):
 def test_paged_attention_with_row_blocks():
     rng = np.random.default_rng(12)
     rand_tree = lambda n: [-1] + [int(rng.integers(0, i)) for i in range(1, n)]
-    trees = [rand_tree(64), rand_tree(3), rand_tree(40)]
-    L = [200, 4000, 65]
+    trees = [rand_tree(64), rand_tree(3), rand_tree(40), rand_tree(101)]
+    L = [200, 4000, 65, 130]
     forest, spec, t, poff = _custom(rng, trees, L, 16, 2, 128, torch.bfloat16)        # up to 512 query rows
     pg = _paged(t, poff, 2, 128, 4, rng)
     out = _gpu_paged(forest, spec, t, poff, pg)
