@@ -290,10 +290,11 @@ def test_host_side_errors():
     assert e.value.code == -1
 
 
-def test_select_width_matches_oracle():
+@pytest.mark.parametrize("top_k,top_p", [(0, 1.0), (10, 0.8), (40, 1.0)])
+def test_select_width_matches_oracle(top_k, top_p):
     rng = np.random.default_rng(8)
     forest, prm, zp, zq, rp, rq, stride = _random_problem(rng, R=4, V=3000, gamma=2, max_w=5)
-    prm = dict(prm, W_min_r=None)
+    prm = dict(prm, W_min_r=None, top_k=top_k, top_p=top_p)
     rbo, bno = forest["req_beam_off"], forest["beam_node_off"]
     live = [bno[rbo[r]:rbo[r + 1]] for r in range(forest["R"])]      # the roots
     live_off = np.concatenate([[0], np.cumsum([len(x) for x in live])]).astype(np.int32)
