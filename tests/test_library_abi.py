@@ -44,3 +44,18 @@ def test_no_cpu_fallback():
     out = dsbd.alloc_verify_out(f, np.array([0, 1]), "cpu")
     with pytest.raises(RuntimeError):
         dsbd.verify_step(f, dict(V=8), z, z, torch.zeros(1), torch.zeros(1), out)
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/dsbd.h is a C header: a C99 compiler accepts it with warnings as errors."""
+    import shutil
+    import subprocess
+    import pytest
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "dsbd.h"\n'
+                   "int main(void) { dsbd_forest_t f; dsbd_verify_params_t p; dsbd_commit_params_t c;\n"
+                   "  (void)f; (void)p; (void)c; return dsbd_status_string(0) == 0; }\n")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                    "-I", os.path.join(ROOT, "include"), str(src)], check=True)
