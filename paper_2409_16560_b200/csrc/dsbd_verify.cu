@@ -578,7 +578,13 @@ struct WarpScratch {
     int sel[256];                 // tiles whose bound reaches the threshold
     int n_sel, n_cand, err;
     float theta;
+    int rhist[256];               // radix select of the k-th largest tile bound
+    unsigned rprefix;
+    int rk, n_finite;
 };
+constexpr int kBoundCache = 2560;  // tile bounds kept in shared memory behind the WarpScratch
+static_assert(sizeof(WarpScratch) + 16 + kBoundCache * sizeof(float) <= (kBins + 2) * sizeof(uint32_t),
+              "the support scratch and the bound cache overlay one histogram array");
 
 // Support of the warped joint of one model; called by ALL threads of the CTA.
 // Returns 0 or a DSBD_DEV_* code (the same on every thread).
@@ -599,28 +605,78 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
         const int ia = i / T;
         return fmaf(stats[(int64_t)sh.A[ia] * T + (i - ia * T)].mx, inv_tau_f, ws.off[ia]);
     };
-    if (warp == 0) {
-        // k-th largest distinct tile bound; with fewer than k distinct bounds every tile counts
-        float thr = INFINITY, top_bound = -INFINITY;
-        bool enough = true;
-        for (int kk = 0; kk < k; ++kk) {
-            float best = -INFINITY;
-            for (int i = lane; i < nt; i += 32) {
-                const float v = bound(i);
-                if (v < thr && v > best) best = v;
+    // The k-th largest tile bound (with multiplicity: k tiles each hold a cell at least that
+    // large); with fewer than k finite bounds every tile counts.
+    float *bcache = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(&ws) +
+                                              ((sizeof(WarpScratch) + 15) & ~size_t(15)));
+    const bool cached = nt <= kBoundCache;
+    if (cached) {
+        // all warps: bounds into shared memory, then a radix select over their order-preserving
+        // integer images, one byte per pass from the top
+        auto image = [](float v) -> unsigned {
+            const unsigned b = __float_as_uint(v);
+            return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+        };
+        if (threadIdx.x == 0) { ws.rprefix = 0u; ws.rk = k; ws.n_finite = 0; }
+        __syncthreads();
+        int finite = 0;
+        for (int i = threadIdx.x; i < nt; i += blockDim.x) {
+            const float v = bound(i);
+            bcache[i] = v;
+            finite += v > -INFINITY;
+        }
+        if (finite) atomicAdd(&ws.n_finite, finite);
+        for (int pass = 3; pass >= 0; --pass) {
+            for (int i = threadIdx.x; i < 256; i += blockDim.x) ws.rhist[i] = 0;
+            __syncthreads();
+            const unsigned prefix = ws.rprefix;
+            for (int i = threadIdx.x; i < nt; i += blockDim.x) {
+                const unsigned u = image(bcache[i]);
+                if (pass == 3 || (u >> (8 * (pass + 1))) == prefix) atomicAdd(&ws.rhist[(u >> (8 * pass)) & 255u], 1);
             }
-            best = warp_max(best);
-            if (!(best > -INFINITY)) { enough = false; break; }
-            if (kk == 0) top_bound = best;
-            thr = best;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int need = ws.rk, d = 255;
+                for (; d > 0; --d) {
+                    if (ws.rhist[d] >= need) break;
+                    need -= ws.rhist[d];
+                }
+                ws.rk = need;
+                ws.rprefix = (prefix << 8) | (unsigned)d;
+            }
+            __syncthreads();
+        }
+    }
+    if (warp == 0) {
+        float thr = INFINITY;
+        bool enough = true, any = false;
+        if (cached) {
+            const unsigned u = ws.rprefix;
+            thr = __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+            enough = ws.n_finite >= k && thr > -INFINITY;
+            any = ws.n_finite > 0;
+        } else {
+            // too many live rows x tiles for the cache: k rounds of arg-max over distinct bounds
+            for (int kk = 0; kk < k; ++kk) {
+                float best = -INFINITY;
+                for (int i = lane; i < nt; i += 32) {
+                    const float v = bound(i);
+                    if (v < thr && v > best) best = v;
+                }
+                best = warp_max(best);
+                if (!(best > -INFINITY)) { enough = false; break; }
+                any = true;
+                thr = best;
+            }
         }
         // the float keys carry an error of about 1e-5; the slack keeps the selection conservative
         const float theta = enough ? thr - 5e-5f - 4e-6f * fabsf(thr) : -INFINITY;
         int n_sel = 0;
-        if (top_bound > -INFINITY)
+        if (any)
             for (int base = 0; base < nt; base += 32) {
                 const int i = base + lane;
-                const bool hit = i < nt && bound(i) >= theta && bound(i) > -INFINITY;
+                const float bv = i < nt ? (cached ? bcache[i] : bound(i)) : -INFINITY;
+                const bool hit = i < nt && bv >= theta && bv > -INFINITY;
                 const unsigned mask = __ballot_sync(kFull, hit);
                 if (hit) {
                     const int pos = n_sel + __popc(mask & ((1u << lane) - 1));
@@ -711,32 +767,26 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
         if (!found) return DSBD_DEV_CAPACITY;              // a huge tie at the cut
         n_cand = sweep(theta, true);
     }
-    // exact top k of the candidates (warp 0): k rounds of arg-max (key descending, cell ascending)
-    if (warp == 0) {
-        int n_sup = 0;
-        for (int kk = 0; kk < k; ++kk) {
-            double bk = -INFINITY;
-            int bc = 0x7fffffff, bi = -1;
-            for (int j = lane; j < n_cand; j += 32) {
-                const double key = cand_key[j];
-                const int cell = cand_cell[j];
-                if (key > bk || (key == bk && key > -INFINITY && cell < bc)) { bk = key; bc = cell; bi = j; }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const double ok = __shfl_xor_sync(kFull, bk, o);
-                const int oc = __shfl_xor_sync(kFull, bc, o), oi = __shfl_xor_sync(kFull, bi, o);
-                if (ok > bk || (ok == bk && ok > -INFINITY && oc < bc)) { bk = ok; bc = oc; bi = oi; }
-            }
-            if (bi < 0 || !(bk > -INFINITY)) break;
-            if (lane == 0) {
-                ws.prob[model][n_sup] = exp(bk);
-                ws.cell[model][n_sup] = bc;
-                cand_key[bi] = -INFINITY;
-            }
-            ++n_sup;
-            __syncwarp();
+    // exact top k of the candidates: every candidate counts those that beat it (key descending,
+    // cell ascending -- a total order, cells are unique) and, if fewer than k do, that count is its
+    // place in the support
+    if (n_cand > kMaxCand) n_cand = kMaxCand;
+    for (int jc = threadIdx.x; jc < n_cand; jc += blockDim.x) {
+        const double key = cand_key[jc];
+        const int cell = cand_cell[jc];
+        int rank = 0;
+        for (int i = 0; i < n_cand; ++i) {
+            const double ki = cand_key[i];
+            rank += (ki > key) || (ki == key && cand_cell[i] < cell);
         }
+        if (rank < k) {
+            ws.prob[model][rank] = exp(key);
+            ws.cell[model][rank] = cell;
+        }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int n_sup = n_cand < k ? n_cand : k;
         // renormalise over the top k, then the top-p cut and its renormalisation (sorted order)
         if (lane == 0) {
             double zsum = 0.0;
