@@ -635,14 +635,32 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
                 if (pass == 3 || (u >> (8 * (pass + 1))) == prefix) atomicAdd(&ws.rhist[(u >> (8 * pass)) & 255u], 1);
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                int need = ws.rk, d = 255;
-                for (; d > 0; --d) {
-                    if (ws.rhist[d] >= need) break;
-                    need -= ws.rhist[d];
+            if (warp == 0) {
+                // the digit whose bin holds the rk-th largest: lane l owns bins 8l .. 8l+7; a suffix
+                // sum over the lanes finds the owning lane, which then walks its own bins
+                int mine = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) mine += ws.rhist[lane * 8 + q];
+                int above = mine;                              // bins of this lane and of the lanes above
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_down_sync(kFull, above, o);
+                    if (lane + o < 32) above += t;
                 }
-                ws.rk = need;
-                ws.rprefix = (prefix << 8) | (unsigned)d;
+                const int need0 = ws.rk;
+                const bool owner = above >= need0 && above - mine < need0;
+                const unsigned who = __ballot_sync(kFull, owner);
+                if (who == 0u) {
+                    if (lane == 0) { ws.rprefix = prefix << 8; ws.rk = need0 - above; }   // fewer than rk values
+                } else if (owner) {
+                    int need = need0 - (above - mine), d = lane * 8 + 7;
+                    for (; d > lane * 8; --d) {
+                        if (ws.rhist[d] >= need) break;
+                        need -= ws.rhist[d];
+                    }
+                    ws.rk = need;
+                    ws.rprefix = (prefix << 8) | (unsigned)d;
+                }
             }
             __syncthreads();
         }
@@ -700,6 +718,13 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
     auto sweep = [&](float th, bool collect) {
         if (threadIdx.x == 0) ws.n_cand = 0;
         __syncthreads();
+        // this warp's tiles into L2 first (a tile is 32 lines of 128 bytes: one per lane), so that
+        // the dependent tile loads below do not each pay a trip to HBM
+        for (int sidx = warp; sidx < n_sel; sidx += kWarps) {
+            const int ti = ws.sel[sidx], ia = ti / T, t = ti - ia * T;
+            const int e = t * kTile + lane * 32;
+            if (e < a.V) asm volatile("prefetch.global.L2 [%0];" ::"l"(z + (int64_t)sh.A[ia] * a.stride + e));
+        }
         for (int sidx = warp; sidx < n_sel; sidx += kWarps) {
             const int ti = ws.sel[sidx], ia = ti / T, t = ti - ia * T, row = sh.A[ia];
             const float *rowp = z + (int64_t)row * a.stride;
@@ -842,13 +867,13 @@ __device__ int draw_support(const WarpScratch &ws, double u, double s) {
 // After build_support(p) [and q]: q~ at the p cells and the canonical order of the p support.
 __device__ void finish_supports(WarpScratch &ws, bool have_q, int lane) {
     for (int i = lane; i < ws.n[0]; i += 32) ws.qat[i] = have_q ? support_lookup(ws, 1, ws.cell[0][i]) : 0.0;
-    if (lane == 0) {
-        const int n = ws.n[0];
-        for (int i = 0; i < n; ++i) {
-            int j = i - 1;
-            while (j >= 0 && ws.cell[0][ws.order[j]] > ws.cell[0][i]) { ws.order[j + 1] = ws.order[j]; --j; }
-            ws.order[j + 1] = i;
-        }
+    // canonical order: the place of a cell is the number of support cells below it (cells are unique)
+    const int n = ws.n[0];
+    for (int i = lane; i < n; i += 32) {
+        const int c = ws.cell[0][i];
+        int place = 0;
+        for (int j = 0; j < n; ++j) place += ws.cell[0][j] < c;
+        ws.order[place] = i;
     }
     __syncwarp();
 }
