@@ -414,7 +414,8 @@ __device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, 
 
 // Acceptance-count recursion by one warp (lanes over n): tail[K] = P(at least K accepts),
 // returns W~ = max{K : tail[K] >= thresh}.
-__device__ int width_rule(Shared &sh, int m, double thresh, int lane) {
+// k_stop >= 0: stop once W = min(W_max = k_stop, max(W_min, W~)) is decided; -1: the whole tail
+__device__ int width_rule(Shared &sh, int m, double thresh, int lane, int k_stop) {
     if (lane == 0) {
         double none = 1.0;
         for (int i = 1; i <= m; ++i) {
@@ -433,6 +434,11 @@ __device__ int width_rule(Shared &sh, int m, double thresh, int lane) {
         below += prev[m];
         if (lane == 0) sh.tail[k + 1] = 1.0 - below;
         if (k == m) break;
+        // tails only fall: past the first one below the threshold, or past the cap, nothing changes W
+        if (k_stop >= 0 && (1.0 - below < thresh || k + 1 >= k_stop)) {
+            for (int K = k + 2 + lane; K <= m + 1; K += 32) sh.tail[K] = 0.0;
+            break;
+        }
         for (int n = lane; n <= m; n += 32) {
             double acc = 0.0;
             if (n >= k + 1)
@@ -581,6 +587,7 @@ struct WarpScratch {
     int rhist[256];               // radix select of the k-th largest tile bound
     unsigned rprefix;
     int rk, n_finite;
+    double zsum;
 };
 constexpr int kBoundCache = 2560;  // tile bounds kept in shared memory behind the WarpScratch
 static_assert(sizeof(WarpScratch) + 16 + kBoundCache * sizeof(float) <= (kBins + 2) * sizeof(uint32_t),
@@ -828,9 +835,12 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
                 zsum = 0.0;
                 for (int q = 0; q < keep; ++q) zsum += ws.prob[model][q];
             }
-            for (int j = 0; j < keep; ++j) ws.prob[model][j] = zsum > 0.0 ? ws.prob[model][j] / zsum : 0.0;
             ws.n[model] = keep;
+            ws.zsum = zsum;
         }
+        __syncwarp();
+        const double inv = ws.zsum > 0.0 ? 1.0 / ws.zsum : 0.0;
+        for (int j = lane; j < ws.n[model]; j += 32) ws.prob[model][j] *= inv;
     }
     __syncthreads();
     return 0;
@@ -1282,21 +1292,18 @@ k_verify(VerifyArgs a) {
         TS(8);
         // ---- width and accept loop (warp 0) ----
         if (warp == 0 && !sh.err) {
-            if (lane == 0) {
-                // alpha_j = 1 - c_{j+1}/c_j; once a residual has no mass every later alpha is 1
-                for (int j = 1; j <= m; ++j) {
-                    if (j <= sh.chain_len && sh.c_arr[j] > 0.0) {
-                        double al = 1.0 - sh.c_arr[j + 1] / sh.c_arr[j];
-                        if (!(sh.c_arr[j + 1] > 0.0)) al = 1.0;
-                        sh.alpha[j] = fmin(fmax(al, 0.0), 1.0);
-                    } else {
-                        sh.alpha[j] = 1.0;
-                    }
-                }
-                sh.res_j = 0;
+            // alpha_j = 1 - c_{j+1}/c_j; once a residual has no mass every later alpha is 1
+            for (int j = 1 + lane; j <= m; j += 32) {
+                double al = 1.0;
+                if (j <= sh.chain_len && sh.c_arr[j] > 0.0 && sh.c_arr[j + 1] > 0.0)
+                    al = fmin(fmax(1.0 - sh.c_arr[j + 1] / sh.c_arr[j], 0.0), 1.0);
+                sh.alpha[j] = al;
             }
+            if (lane == 0) sh.res_j = 0;
             __syncwarp();
-            const int wt = width_rule(sh, m, a.thresh, lane);
+            // (the verification only needs W~ up to W_max and can stop at the first tail below the
+            // threshold; dsbd_select_width returns the whole tail)
+            const int wt = width_rule(sh, m, a.thresh, lane, a.select_mode ? -1 : W_max);
             int W = wt > W_min ? wt : W_min;
             if (W > W_max) W = W_max;
             if (a.select_mode) {
@@ -1312,7 +1319,7 @@ k_verify(VerifyArgs a) {
                 if (lane == 0) sh.done = 1;
             } else if (lane == 0) {
                 if (writer) a.out.layer_width[(int64_t)r * (a.gamma + 1) + (l - 1)] = W;
-                int count = 0, j = 1, err = 0;
+                int count = 0, j = 1, err = 0, tests = 0;
                 for (int i = 0; i < m && count < W; ++i) {
                     const int n = sh.S[i];
                     const double rho = sh.rho[i];
@@ -1321,7 +1328,7 @@ k_verify(VerifyArgs a) {
                     else ratio = fmax(rho - sh.s_arr[j - 1], 0.0) / sh.c_arr[j];
                     if (ratio > 1.0) ratio = 1.0;
                     const double u = sh.uu[i];
-                    ++sh.n_tests;
+                    ++tests;
                     if (u <= ratio) {
                         st[n - n_lo] = DSBD_NODE_ACCEPTED;
                         if (writer) a.out.node_status[n] = DSBD_NODE_ACCEPTED;
@@ -1342,6 +1349,7 @@ k_verify(VerifyArgs a) {
                     }
                 sh.W = W;
                 sh.count = count;
+                sh.n_tests += tests;
                 ++sh.n_layers;
                 sh.res_j = (count < W && j > 1) ? j : 0;   // residual draw at run position j needs tile sums
                 sh.run_j = j;
