@@ -908,6 +908,9 @@ k_verify(VerifyArgs a) {
     __shared__ int8_t st[kMaxLive * kMaxLive];     // status of the request's nodes, local index
     __shared__ __align__(16) uint32_t hp[kBins + 2], hq[kBins + 2];   // p and q mass per ratio bin, fixed point
 
+    // launched with programmatic stream serialization: everything before this line overlaps the
+    // tail of the kernel ahead in the stream, nothing after it may run before that kernel is done
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
     const int n_lo = a.beam_node_off[b_lo], n_hi = a.beam_node_off[b_hi];
     const int W_min = a.W_min_r ? a.W_min_r[r] : a.W_min;
@@ -1599,13 +1602,17 @@ int launch_verify(const VerifyArgs &args, int R, int tiles, cudaStream_t stream)
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)cs;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // the clusters may be set up while the dense pass before them drains; the kernel waits for
+    // that grid's results (griddepcontrol.wait) before it reads anything
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, k_verify, args) == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 
