@@ -572,50 +572,68 @@ __device__ int draw_cell(const VerifyArgs &a, const Shared &sh, double u, bool u
 // Only those (about k) tiles are read.
 // ---------------------------------------------------------------------------------------
 constexpr int kMaxTopK = 64;
-constexpr int kMaxCand = 1024;
+constexpr int kMaxCand = 680;      // candidate cells per model (two lists overlay one histogram array)
+constexpr int kHalf = 128;         // threads that build one model's support (the two models run side by side)
+// scratch of one build_support instance
+struct SupportTmp {
+    float off[kMaxLive];          // log(beam weight) - lse of each live row
+    int sel[256];                 // tiles whose bound reaches the threshold
+    int rhist[256];               // radix select of the k-th largest tile bound
+    int n_sel, n_cand, err, n_finite, rk;
+    unsigned rprefix;
+    float theta;
+    double zsum;
+};
 struct WarpScratch {
     double prob[2][kMaxTopK];     // warped probabilities, most probable first (0: p, 1: q)
     double qat[kMaxTopK];         // q~ at the cells of the p support
     int cell[2][kMaxTopK];        // live parent index * V + token
     int order[kMaxTopK];          // the p support in canonical (cell-ascending) order
     int n[2];
-    // scratch of build_support
-    float off[kMaxLive];          // log(beam weight) - lse of each live row
-    int sel[256];                 // tiles whose bound reaches the threshold
-    int n_sel, n_cand, err;
-    float theta;
-    int rhist[256];               // radix select of the k-th largest tile bound
-    unsigned rprefix;
-    int rk, n_finite;
-    double zsum;
+    SupportTmp tmp[2];
 };
-constexpr int kBoundCache = 2560;  // tile bounds kept in shared memory behind the WarpScratch
-static_assert(sizeof(WarpScratch) + 16 + kBoundCache * sizeof(float) <= (kBins + 2) * sizeof(uint32_t),
-              "the support scratch and the bound cache overlay one histogram array");
+constexpr int kBoundCache = 1152;  // tile bounds per model kept in shared memory behind the WarpScratch
+static_assert(((sizeof(WarpScratch) + 15) & ~size_t(15)) + 2 * kBoundCache * sizeof(float) <=
+                  (kBins + 2) * sizeof(uint32_t),
+              "the support scratch and the two bound caches overlay one histogram array");
+static_assert(2 * kMaxCand * (sizeof(double) + sizeof(int)) <= (kBins + 2) * sizeof(uint32_t),
+              "the two candidate lists overlay the other histogram array");
 
-// Support of the warped joint of one model; called by ALL threads of the CTA.
-// Returns 0 or a DSBD_DEV_* code (the same on every thread).
-__device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, double *cand_key, int *cand_cell,
-                             WarpScratch &ws) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+// barrier of the 128 threads that work on one model (ids 1 and 2; 0 is __syncthreads)
+__device__ __forceinline__ void half_sync(int half) {
+    asm volatile("bar.sync %0, %1;" ::"r"(half + 1), "r"(kHalf) : "memory");
+}
+
+// Support of the warped joint of one model; called by the 128 threads of half `model` of the CTA
+// (warps 0-3: p, warps 4-7: q), the two halves side by side on their own scratch.  hist_p / hist_q:
+// the two idle histogram arrays.  Returns 0 or a DSBD_DEV_* code (the same on every thread of the
+// half).
+__device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, uint32_t *hist_p, uint32_t *hist_q) {
+    WarpScratch &ws = *reinterpret_cast<WarpScratch *>(hist_q);
+    SupportTmp &tp = ws.tmp[model];
+    double *cand_key = reinterpret_cast<double *>(hist_p) + model * kMaxCand;
+    int *cand_cell = reinterpret_cast<int *>(reinterpret_cast<double *>(hist_p) + 2 * kMaxCand) + model * kMaxCand;
+    const int tl = threadIdx.x & (kHalf - 1);                 // thread and warp inside the half
+    const int lane = threadIdx.x & 31, warp = tl >> 5;
+    constexpr int kHalfWarps = kHalf / 32;
     const int T = a.T, nt = sh.nA * T, k = a.top_k;
     const TileStat *stats = a.stats + (int64_t)model * a.N * T;
     const double *lw = model ? sh.lwq : sh.lwp;
     const double *lse = a.lse + (int64_t)model * a.N;
     const float *z = model ? a.zq : a.zp;
     const float inv_tau_f = (float)a.inv_tau;
-    for (int i = threadIdx.x; i < sh.nA; i += blockDim.x) ws.off[i] = (float)(lw[i] - lse[sh.A[i]]);
-    if (threadIdx.x == 0) { ws.n_sel = 0; ws.n_cand = 0; ws.err = 0; ws.n[model] = 0; }
-    __syncthreads();
+    for (int i = tl; i < sh.nA; i += kHalf) tp.off[i] = (float)(lw[i] - lse[sh.A[i]]);
+    if (tl == 0) { tp.n_sel = 0; tp.n_cand = 0; tp.err = 0; ws.n[model] = 0; }
+    half_sync(model);
     // float upper bound of log(joint probability) over tile i
     auto bound = [&](int i) -> float {
         const int ia = i / T;
-        return fmaf(stats[(int64_t)sh.A[ia] * T + (i - ia * T)].mx, inv_tau_f, ws.off[ia]);
+        return fmaf(stats[(int64_t)sh.A[ia] * T + (i - ia * T)].mx, inv_tau_f, tp.off[ia]);
     };
     // The k-th largest tile bound (with multiplicity: k tiles each hold a cell at least that
     // large); with fewer than k finite bounds every tile counts.
     float *bcache = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(&ws) +
-                                              ((sizeof(WarpScratch) + 15) & ~size_t(15)));
+                                              ((sizeof(WarpScratch) + 15) & ~size_t(15))) + model * kBoundCache;
     const bool cached = nt <= kBoundCache;
     if (cached) {
         // all warps: bounds into shared memory, then a radix select over their order-preserving
@@ -624,62 +642,62 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
             const unsigned b = __float_as_uint(v);
             return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
         };
-        if (threadIdx.x == 0) { ws.rprefix = 0u; ws.rk = k; ws.n_finite = 0; }
-        __syncthreads();
+        if (tl == 0) { tp.rprefix = 0u; tp.rk = k; tp.n_finite = 0; }
+        half_sync(model);
         int finite = 0;
-        for (int i = threadIdx.x; i < nt; i += blockDim.x) {
+        for (int i = tl; i < nt; i += kHalf) {
             const float v = bound(i);
             bcache[i] = v;
             finite += v > -INFINITY;
         }
-        if (finite) atomicAdd(&ws.n_finite, finite);
+        if (finite) atomicAdd(&tp.n_finite, finite);
         for (int pass = 3; pass >= 0; --pass) {
-            for (int i = threadIdx.x; i < 256; i += blockDim.x) ws.rhist[i] = 0;
-            __syncthreads();
-            const unsigned prefix = ws.rprefix;
-            for (int i = threadIdx.x; i < nt; i += blockDim.x) {
+            for (int i = tl; i < 256; i += kHalf) tp.rhist[i] = 0;
+            half_sync(model);
+            const unsigned prefix = tp.rprefix;
+            for (int i = tl; i < nt; i += kHalf) {
                 const unsigned u = image(bcache[i]);
-                if (pass == 3 || (u >> (8 * (pass + 1))) == prefix) atomicAdd(&ws.rhist[(u >> (8 * pass)) & 255u], 1);
+                if (pass == 3 || (u >> (8 * (pass + 1))) == prefix) atomicAdd(&tp.rhist[(u >> (8 * pass)) & 255u], 1);
             }
-            __syncthreads();
+            half_sync(model);
             if (warp == 0) {
                 // the digit whose bin holds the rk-th largest: lane l owns bins 8l .. 8l+7; a suffix
                 // sum over the lanes finds the owning lane, which then walks its own bins
                 int mine = 0;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) mine += ws.rhist[lane * 8 + q];
+                for (int q = 0; q < 8; ++q) mine += tp.rhist[lane * 8 + q];
                 int above = mine;                              // bins of this lane and of the lanes above
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const int t = __shfl_down_sync(kFull, above, o);
                     if (lane + o < 32) above += t;
                 }
-                const int need0 = ws.rk;
+                const int need0 = tp.rk;
                 const bool owner = above >= need0 && above - mine < need0;
                 const unsigned who = __ballot_sync(kFull, owner);
                 if (who == 0u) {
-                    if (lane == 0) { ws.rprefix = prefix << 8; ws.rk = need0 - above; }   // fewer than rk values
+                    if (lane == 0) { tp.rprefix = prefix << 8; tp.rk = need0 - above; }   // fewer than rk values
                 } else if (owner) {
                     int need = need0 - (above - mine), d = lane * 8 + 7;
                     for (; d > lane * 8; --d) {
-                        if (ws.rhist[d] >= need) break;
-                        need -= ws.rhist[d];
+                        if (tp.rhist[d] >= need) break;
+                        need -= tp.rhist[d];
                     }
-                    ws.rk = need;
-                    ws.rprefix = (prefix << 8) | (unsigned)d;
+                    tp.rk = need;
+                    tp.rprefix = (prefix << 8) | (unsigned)d;
                 }
             }
-            __syncthreads();
+            half_sync(model);
         }
     }
     if (warp == 0) {
         float thr = INFINITY;
         bool enough = true, any = false;
         if (cached) {
-            const unsigned u = ws.rprefix;
+            const unsigned u = tp.rprefix;
             thr = __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
-            enough = ws.n_finite >= k && thr > -INFINITY;
-            any = ws.n_finite > 0;
+            enough = tp.n_finite >= k && thr > -INFINITY;
+            any = tp.n_finite > 0;
         } else {
             // too many live rows x tiles for the cache: k rounds of arg-max over distinct bounds
             for (int kk = 0; kk < k; ++kk) {
@@ -705,40 +723,40 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
                 const unsigned mask = __ballot_sync(kFull, hit);
                 if (hit) {
                     const int pos = n_sel + __popc(mask & ((1u << lane) - 1));
-                    if (pos < 256) ws.sel[pos] = i;
+                    if (pos < 256) tp.sel[pos] = i;
                 }
                 n_sel += __popc(mask);
             }
         if (lane == 0) {
-            ws.theta = theta;
-            ws.n_sel = n_sel;
-            if (n_sel > 256) ws.err = DSBD_DEV_CAPACITY;       // hundreds of tiles tie at the cut
+            tp.theta = theta;
+            tp.n_sel = n_sel;
+            if (n_sel > 256) tp.err = DSBD_DEV_CAPACITY;       // hundreds of tiles tie at the cut
         }
     }
-    __syncthreads();
-    if (ws.err) return ws.err;
-    float theta = ws.theta;
-    const int n_sel = ws.n_sel;
+    half_sync(model);
+    if (tp.err) return tp.err;
+    float theta = tp.theta;
+    const int n_sel = tp.n_sel;
     // One sweep over the selected tiles by all warps: counts the cells whose key reaches th and,
     // when asked, appends them to the candidate list (order is irrelevant: the final choice is
     // by (key, cell)).
     auto sweep = [&](float th, bool collect) {
-        if (threadIdx.x == 0) ws.n_cand = 0;
-        __syncthreads();
+        if (tl == 0) tp.n_cand = 0;
+        half_sync(model);
         // this warp's tiles into L2 first (a tile is 32 lines of 128 bytes: one per lane), so that
         // the dependent tile loads below do not each pay a trip to HBM
-        for (int sidx = warp; sidx < n_sel; sidx += kWarps) {
-            const int ti = ws.sel[sidx], ia = ti / T, t = ti - ia * T;
+        for (int sidx = warp; sidx < n_sel; sidx += kHalfWarps) {
+            const int ti = tp.sel[sidx], ia = ti / T, t = ti - ia * T;
             const int e = t * kTile + lane * 32;
             if (e < a.V) asm volatile("prefetch.global.L2 [%0];" ::"l"(z + (int64_t)sh.A[ia] * a.stride + e));
         }
-        for (int sidx = warp; sidx < n_sel; sidx += kWarps) {
-            const int ti = ws.sel[sidx], ia = ti / T, t = ti - ia * T, row = sh.A[ia];
+        for (int sidx = warp; sidx < n_sel; sidx += kHalfWarps) {
+            const int ti = tp.sel[sidx], ia = ti / T, t = ti - ia * T, row = sh.A[ia];
             const float *rowp = z + (int64_t)row * a.stride;
             const bool al = (reinterpret_cast<uintptr_t>(rowp) & 15) == 0;
             float4 v[8];
             load_tile(rowp, t * kTile, a.V, al, lane, v);
-            const float off_f = ws.off[ia];
+            const float off_f = tp.off[ia];
             const double off_d = lw[ia] - lse[row];
             unsigned hits = 0;                               // bit (it*4+c) of this lane's 32 cells
 #pragma unroll
@@ -759,7 +777,7 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
             }
             const int total = __shfl_sync(kFull, incl, 31);
             int base_pos = 0;
-            if (lane == 0 && total) base_pos = atomicAdd(&ws.n_cand, total);
+            if (lane == 0 && total) base_pos = atomicAdd(&tp.n_cand, total);
             base_pos = __shfl_sync(kFull, base_pos, 0);
             if (collect && mine) {
                 int pos = base_pos + incl - mine;
@@ -778,15 +796,15 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
                 }
             }
         }
-        __syncthreads();
-        return ws.n_cand;
+        half_sync(model);
+        return tp.n_cand;
     };
     int n_cand = sweep(theta, true);
     if (n_cand > kMaxCand) {
         // too many cells reach the conservative threshold (few tiles, large k, or near ties):
         // bisect for a threshold with between k and kMaxCand cells above it
         float lo_t = theta, hi_t = -INFINITY;
-        for (int sidx = 0; sidx < n_sel; ++sidx) hi_t = fmaxf(hi_t, bound(ws.sel[sidx]));
+        for (int sidx = 0; sidx < n_sel; ++sidx) hi_t = fmaxf(hi_t, bound(tp.sel[sidx]));
         if (!(lo_t > -INFINITY)) lo_t = hi_t - 400.f;
         bool found = false;
         for (int itn = 0; itn < 60 && hi_t > lo_t; ++itn) {
@@ -803,7 +821,7 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
     // cell ascending -- a total order, cells are unique) and, if fewer than k do, that count is its
     // place in the support
     if (n_cand > kMaxCand) n_cand = kMaxCand;
-    for (int jc = threadIdx.x; jc < n_cand; jc += blockDim.x) {
+    for (int jc = tl; jc < n_cand; jc += kHalf) {
         const double key = cand_key[jc];
         const int cell = cand_cell[jc];
         int rank = 0;
@@ -816,7 +834,7 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
             ws.cell[model][rank] = cell;
         }
     }
-    __syncthreads();
+    half_sync(model);
     if (warp == 0) {
         const int n_sup = n_cand < k ? n_cand : k;
         // renormalise over the top k, then the top-p cut and its renormalisation (sorted order)
@@ -836,13 +854,13 @@ __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, d
                 for (int q = 0; q < keep; ++q) zsum += ws.prob[model][q];
             }
             ws.n[model] = keep;
-            ws.zsum = zsum;
+            tp.zsum = zsum;
         }
         __syncwarp();
-        const double inv = ws.zsum > 0.0 ? 1.0 / ws.zsum : 0.0;
+        const double inv = tp.zsum > 0.0 ? 1.0 / tp.zsum : 0.0;
         for (int j = lane; j < ws.n[model]; j += 32) ws.prob[model][j] *= inv;
     }
-    __syncthreads();
+    half_sync(model);
     return 0;
 }
 
@@ -1164,10 +1182,12 @@ k_verify(VerifyArgs a) {
         if (warped) {
             // ---- supports of T o p_beam and T o q_beam, then the whole chain on <= 64 cells ----
             if (!sh.err) {
-                double *cand_key = reinterpret_cast<double *>(hp);
-                int *cand_cell = reinterpret_cast<int *>(hp + 2 * kMaxCand);
-                int e = build_support(a, sh, 0, cand_key, cand_cell, wsup);
-                if (!e) e = build_support(a, sh, 1, cand_key, cand_cell, wsup);
+                // warps 0-3 build the support of p, warps 4-7 that of q, side by side
+                const int half = warp >> 2;
+                const int e_half = build_support(a, sh, half, hp, hq);
+                if (e_half && (threadIdx.x & (kHalf - 1)) == 0) wsup.tmp[half].err = e_half;
+                __syncthreads();
+                const int e = wsup.tmp[0].err ? wsup.tmp[0].err : wsup.tmp[1].err;
                 if (e) { if (threadIdx.x == 0) sh.err = e; }
                 else if (warp == 0) {
                     finish_supports(wsup, true, lane);
@@ -1471,8 +1491,12 @@ k_verify(VerifyArgs a) {
         if (warp == 0) live_weights(a, sh, sp_live, sq_live, lane);
         __syncthreads();
         if (a.top_k > 0) {
-            extra_err = build_support(a, sh, 0, reinterpret_cast<double *>(hp),
-                                      reinterpret_cast<int *>(hp + 2 * kMaxCand), wsx);
+            if (warp < kHalf / 32) {                            // one model only: the first half builds it
+                const int e_half = build_support(a, sh, 0, hp, hq);
+                if (e_half && threadIdx.x == 0) wsx.tmp[0].err = e_half;
+            }
+            __syncthreads();
+            extra_err = wsx.tmp[0].err;
             if (!extra_err && warp == 0) finish_supports(wsx, false, lane);
         }
     }
