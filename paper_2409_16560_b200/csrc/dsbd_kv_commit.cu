@@ -326,15 +326,63 @@ k_commit_pages(CommitArgs a) {
     }
 }
 
-// The free stack after the update: every page that no new table names, ascending.  One CTA;
-// the compaction walks the page flags in super-tiles of 16 flags per thread, loaded as four
-// independent 128-bit loads, with a block scan of the per-thread counts.
+// The free stack after the update: every page that no new table names, ascending.  One CTA; a
+// bitmap in shared memory for pools of up to 256 K pages, else flags in the workspace that the
+// compaction walks in super-tiles of 16 per thread (four independent 128-bit loads), with a
+// block scan of the per-thread counts either way.
 __global__ void __launch_bounds__(kPlanThreads)
 k_commit_free(CommitArgs a) {
     __shared__ int32_t warp_tot[32];
     __shared__ int32_t carry;
     if (a.plan->error) return;
     const int n = (int)a.n_pages;
+    // Pools of up to 256 K pages: one bit per page in shared memory (1 = free), so that marking
+    // and compaction never leave the SM; larger pools use the flag array in the workspace.
+    constexpr int kBitWords = 8192;
+    __shared__ uint32_t bits[kBitWords];
+    if (n <= kBitWords * 32) {
+        const int words = (n + 31) >> 5;
+        for (int w = threadIdx.x; w < words; w += blockDim.x)
+            bits[w] = (w + 1) * 32 <= n ? 0xffffffffu : ((1u << (n & 31)) - 1u);
+        if (threadIdx.x == 0) carry = 0;
+        __syncthreads();
+        const int64_t entries = a.new_page_off[a.n_slots];
+        for (int64_t i = threadIdx.x; i < entries; i += blockDim.x) {
+            const int pg = a.new_page_table[i];
+            if (pg >= 0 && pg < n) atomicAnd(&bits[pg >> 5], ~(1u << (pg & 31)));
+        }
+        __syncthreads();
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        for (int base = 0; base < words; base += kPlanThreads) {
+            const int w = base + threadIdx.x;
+            uint32_t m = w < words ? bits[w] : 0u;
+            const int cnt = __popc(m);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) warp_tot[warp] = incl;
+            __syncthreads();
+            int before = carry, tile_total = 0;
+            for (int x = 0; x < kPlanThreads / 32; ++x) {
+                if (x < warp) before += warp_tot[x];
+                tile_total += warp_tot[x];
+            }
+            int pos = before + incl - cnt;
+            while (m) {
+                const int b = __ffs(m) - 1;
+                a.free_stack[pos++] = w * 32 + b;
+                m &= m - 1;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) carry += tile_total;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) *a.free_count = carry;
+        return;
+    }
     const int n_pad = (n + 15) & ~15;                                             // the array holds n + 1 <= n_pad + 16
     for (int i = threadIdx.x; i < n_pad; i += blockDim.x) a.used[i] = i < n ? 1 : 0;   // 1 = free
     if (threadIdx.x == 0) carry = 0;
