@@ -14,8 +14,9 @@
  *     distribution without mass, a bounded wait that ran out) are written to `*status`
  *     (device int32, must be zero before the call, first error wins) and, per request, to
  *     `req_error`; kernels never trap.
- *   - There is no CPU fallback and no global state; the same inputs and (seed, step) give the
- *     same outputs whatever the launch shape.
+ *   - There is no CPU fallback and no global state (dsbd_node_stats_static, which says so, is
+ *     the one exception); the same inputs and (seed, step) give the same outputs whatever the
+ *     launch shape.
  */
 #ifndef DSBD_H
 #define DSBD_H
@@ -41,8 +42,10 @@ enum {
 enum {
     DSBD_DEV_BAD_TOKEN = 1,      /* draft token outside [0, V)                               */
     DSBD_DEV_EXHAUSTED = 2,      /* a draw from a distribution without mass                  */
-    DSBD_DEV_CAPACITY = 3,       /* more output beams than the request's out_off range holds */
-    DSBD_DEV_BAD_FOREST = 4,     /* parent index outside its tree, too many live beams/drafts */
+    DSBD_DEV_CAPACITY = 3,       /* a range the caller sized is too small: output slots of a
+                                    request, cache tokens, page-table entries, free pages    */
+    DSBD_DEV_BAD_FOREST = 4,     /* an index that contradicts the forest: parent outside its
+                                    tree, beam outside its request, too many live beams      */
     DSBD_DEV_TIMEOUT = 5         /* a bounded wait gave up                                   */
 };
 
