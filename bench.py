@@ -221,7 +221,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="dsbd", choices=["dsbd", "reference"])
     ap.add_argument("--workload", default="C5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -301,6 +301,10 @@ def main():
         sampler.start()
         time.sleep(0.3)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4 * args.steps + 1)]
+    # workloads whose inputs would sit in the 126 MB L2 get it flushed between steps (a 256 MB
+    # write outside the per-step events; the step time is then the sum of the per-step times)
+    step_bytes = inputs.attention_bytes(spec, forest, poff) + inputs.verify_bytes(spec, forest)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < 4 * (126 << 20) else None
     t_wall0 = time.time()
     barrier()
     ev[0].record(stream)
@@ -308,6 +312,8 @@ def main():
     for s in range(args.steps):
         a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
         a2 = torch.cuda.Event(enable_timing=True)
+        if flush is not None:
+            flush.zero_()
         a0.record(stream)
         attention()
         a1.record(stream)
@@ -318,9 +324,11 @@ def main():
     barrier()
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    total_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), world, dev)
-    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in e_attn]))
-    ver_ms = float(np.mean([a.elapsed_time(b) for a, b in e_ver]))
+    t_attn = [a.elapsed_time(b) for a, b in e_attn]
+    t_ver = [a.elapsed_time(b) for a, b in e_ver]
+    total_local = ev[0].elapsed_time(ev[1]) if flush is None else float(np.sum(t_attn) + np.sum(t_ver))
+    total_ms = max_over_ranks(total_local, world, dev)
+    attn_ms, ver_ms = float(np.median(t_attn)), float(np.median(t_ver))
     assert int(status.item()) == 0, "device status %d" % int(status.item())
     st = vout["req_stats"].cpu().numpy().reshape(-1, 4).astype(float)
     verify_stats = {"layers_per_request": float(st[:, 0].mean()), "accept_tests_per_request": float(st[:, 1].mean()),
@@ -560,8 +568,9 @@ def main():
             "config": {"workload": args.workload, "requests": f.R, "beams": f.B, "nodes": f.N,
                        "heads": "%dq/%dkv x %d" % (spec["Hq"], spec["Hkv"], spec["d"]), "vocab": spec["V"],
                        "prefix": list(spec["prefix"]), "temperature": spec["temperature"],
-                       "thresh": prm["thresh"], "top_k": args.top_k, "top_p": args.top_p, "l2": "inputs (%.1f GB) far exceed the 126 MB L2; no flush" % (
-                           (a_bytes + v_bytes) * 1e-9),
+                       "thresh": prm["thresh"], "top_k": args.top_k, "top_p": args.top_p, "l2": ("inputs (%.1f GB) far exceed the 126 MB L2; no flush" % ((a_bytes + v_bytes) * 1e-9)) if flush is None
+                       else "inputs (%.0f MB) would fit the 126 MB L2: flushed by a 256 MB write between steps" % (
+                           (a_bytes + v_bytes) * 1e-6),
                        "parallelism": "replicas x%d" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "kernels": kernels, "graph_replay_ms_per_step": graph_ms,
