@@ -1199,15 +1199,23 @@ k_verify(VerifyArgs a) {
                             sh.rho[i] = qw > 0.0 ? pw / qw : (pw > 0.0 ? INFINITY : 0.0);
                         }
                     // c_{j+1} = F(s_j) over the p support, lanes over cells
+                    // (every lane keeps its at most two cells and the running s, c in registers)
+                    const int ns = wsup.n[0];
+                    const double p0 = lane < ns ? wsup.prob[0][lane] : 0.0, q0 = lane < ns ? wsup.qat[lane] : 0.0;
+                    const double p1 = lane + 32 < ns ? wsup.prob[0][lane + 32] : 0.0;
+                    const double q1 = lane + 32 < ns ? wsup.qat[lane + 32] : 0.0;
+                    double s_prev = 0.0, c_cur = 1.0;
                     for (int j = 1; j <= m; ++j) {
-                        const double s_j = sh.s_arr[j - 1] + sh.c_arr[j];
-                        double acc = 0.0;
-                        for (int i = lane; i < wsup.n[0]; i += 32) acc += fmax(wsup.prob[0][i] - s_j * wsup.qat[i], 0.0);
+                        const double s_j = s_prev + c_cur;
+                        double acc = fmax(p0 - s_j * q0, 0.0);
+                        if (lane + 32 < ns) acc += fmax(p1 - s_j * q1, 0.0);
                         acc = warp_sum(acc);
                         if (lane == 0) { sh.s_arr[j] = s_j; sh.c_arr[j + 1] = acc; sh.chain_len = j; }
-                        __syncwarp();
+                        s_prev = s_j;
+                        c_cur = acc;
                         if (!(acc > 0.0)) break;
                     }
+                    __syncwarp();
                 }
             }
             __syncthreads();
