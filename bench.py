@@ -225,6 +225,9 @@ def main():
     ap.add_argument("--impl", default="dsbd", choices=["dsbd", "reference"])
     ap.add_argument("--workload", default="C5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pipeline-steps", type=int, default=0,
+                    help="also time whole decode steps (draft stage, forest assembly, paged attention, "
+                         "verification, paged cache update) and report them under 'pipeline'")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--top-k", type=int, default=0, help="warp the joint distributions: top-k (0 = off)")
     ap.add_argument("--top-p", type=float, default=1.0, help="and top-p (needs --top-k); the paper uses 10 / 0.8")
@@ -459,6 +462,84 @@ def main():
         assert int(status.item()) == 0, "device status %d" % int(status.item())
         del pg, attn_out_pg
 
+    # ---- whole decode steps: draft stage -> forest -> paged attention -> verification -> cache update
+    pipeline = None
+    if args.pipeline_steps > 0 and data["k_new"].dtype == torch.bfloat16 and spec["d"] == 128:
+        gamma, B = int(forest["max_depth"]), f.B
+        W_S = max(1, (f.N - B) // max(gamma * f.R, 1))                # the configuration's nodes per layer
+        rbo_h = np.asarray(forest["req_beam_off"], dtype=np.int32)
+        rbo_d = torch.as_tensor(rbo_h).to(dev)
+        lay_off_h = (W_S * np.arange(f.R + 1)).astype(np.int32)
+        lay_off_d = torch.as_tensor(lay_off_h).to(dev)
+        ppg = inputs.paginate(data["k_prefix"], data["v_prefix"], poff, spec["Hkv"], spec["d"],
+                              extra_pages=2 * n_slots + 64, seed=int(spec["seed"]))
+        free0, count0 = ppg["free_stack"].clone(), ppg["free_count"].clone()
+        need_rows = B + (gamma - 1) * f.R * W_S
+        assert need_rows <= f.N, "not enough logits rows to stand for the draft stage"
+        pout = dsbd.alloc_verify_out(f, out_off, dev)
+        # attention workspace for whatever forest the draft stage samples: sized by the bound
+        bound = dsbd.Forest.from_device(f.R, B, f.N, gamma, f.dev, max_tree_nodes=min(1 + gamma * W_S, 128),
+                                        max_req_beams=f.max_req_beams, max_layer_nodes=W_S)
+        ws_pipe = torch.empty(max(dsbd.forest_attention_workspace(bound, spec["Hq"], spec["Hkv"], spec["d"],
+                                                                  data["q"].dtype, scale, poff), 256),
+                              dtype=torch.uint8, device=dev)
+        st = {"draft": [None] * gamma, "commit": None}
+        names = ["draft", "forest", "attention", "verify", "commit"]
+
+        def pipeline_step(step, ev):
+            ev[0].record(stream)
+            cur_off_h, cur_off_d, cur_s, row0 = rbo_h, rbo_d, data["root_logq"], 0
+            dp, dt = [], []
+            for l in range(gamma):
+                n_cur = int(cur_off_h[-1])
+                d = dsbd.draft_layer(cur_off_d, cur_off_h, dict(prm, step=step), l + 1, W_S,
+                                     data["logits_q"][row0:row0 + n_cur], cur_s, lay_off_d, f.R * W_S,
+                                     workspace=st["draft"][l]["workspace"] if st["draft"][l] else None,
+                                     status=status, stream=stream, out=st["draft"][l])
+                st["draft"][l] = d
+                dp.append(d["out_parent"]); dt.append(d["out_token"])
+                row0 += n_cur
+                cur_off_h, cur_off_d, cur_s = lay_off_h, lay_off_d, d["out_logq"]
+            ev[1].record(stream)
+            bf, _, _ = dsbd.forest_build(rbo_d, rbo_h, gamma, W_S, torch.stack(dp), torch.stack(dt), status=status,
+                                         stream=stream, exact=True)
+            ev[2].record(stream)
+            dsbd.forest_attention_paged(bf, spec["Hq"], spec["Hkv"], spec["d"], scale, data["q"], data["k_new"],
+                                        data["v_new"], ppg["k_pool"], ppg["v_pool"], ppg["page_table"],
+                                        ppg["page_off"], poff_dev, poff, out=attn_out, workspace=ws_pipe,
+                                        status=status, stream=stream)
+            ev[3].record(stream)
+            dsbd.verify_step(bf, dict(prm_dev, step=step), data["logits_p"], data["logits_q"], data["root_logp"],
+                             data["root_logq"], pout, workspace=ws_v, status=status, stream=stream)
+            ev[4].record(stream)
+            ppg["free_stack"].copy_(free0); ppg["free_count"].copy_(count0)
+            st["commit"] = dsbd.kv_commit_paged(
+                bf, spec["Hkv"], spec["d"], out_off_dev, pout["out_width"], pout["out_parent"], pout["out_root_beam"],
+                pout["out_logp"], data["k_new"], data["v_new"], ppg["k_pool"], ppg["v_pool"], ppg["page_table"],
+                ppg["page_off"], poff_dev, poff, ppg["free_stack"], ppg["free_count"], n_slots=n_slots,
+                table_capacity=int(ppg["page_table"].numel()) + 2 * n_slots,
+                workspace=st["commit"]["workspace"] if st["commit"] else None, status=status, stream=stream,
+                out=st["commit"])
+            ev[5].record(stream)
+            return bf
+
+        mk = lambda: [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        for s_ in range(3):
+            bf_last = pipeline_step(s_, mk())
+        torch.cuda.synchronize()
+        evs = []
+        for s_ in range(args.pipeline_steps):
+            e = mk(); pipeline_step(3 + s_, e); evs.append(e)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, "device status %d" % int(status.item())
+        parts = {n: float(np.median([e[i].elapsed_time(e[i + 1]) for e in evs])) for i, n in enumerate(names)}
+        total = float(np.median([e[0].elapsed_time(e[5]) for e in evs]))
+        pipeline = {"ms_per_step": total, "nodes_per_s": f.N / total * 1e3, "parts_ms": parts, "gamma": gamma,
+                    "W_S": W_S, "largest_tree": bf_last.max_tree_nodes, "steps": args.pipeline_steps,
+                    "note": "every step starts from the same beams and caches; the forest is the one the draft "
+                            "stage samples (ragged trees), the models' rows are the synthetic tensors"}
+        del ppg
+
     # one draft-stage sampling step of the same shape (W_S = beams of the request), reported
     # beside the step: the small model's logits of the first B rows stand for a draft layer
     rbo_host = np.asarray(forest["req_beam_off"], dtype=np.int32)
@@ -573,7 +654,7 @@ def main():
                            (a_bytes + v_bytes) * 1e-6),
                        "parallelism": "replicas x%d" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "kernels": kernels, "graph_replay_ms_per_step": graph_ms,
+            "roofline": roofline, "kernels": kernels, "graph_replay_ms_per_step": graph_ms, "pipeline": pipeline,
             "verify_stats_last_step": verify_stats, "cpu_baseline": cpu}
     print(json.dumps(line))
     if world > 1:

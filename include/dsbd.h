@@ -316,11 +316,15 @@ size_t dsbd_draft_workspace(int32_t R, int32_t n_beams, const dsbd_draft_params_
  * draft_rank[n] = the draw index k, beam_node_off [B+1], and node_of_draw [gamma][R * W_S]: the node
  * each draw became (to place the models' rows).  Node numbering inside a tree is a convention of
  * this library; any topological order would do.  gamma * W_S <= 1024, beams per request <=
- * DSBD_MAX_LIVE.  *status: DSBD_DEV_BAD_FOREST when a draw names a beam of another request. */
+ * DSBD_MAX_LIVE.  max_tree_nodes (optional device int32, set it to 0 before the call) is raised
+ * to the size of the largest tree: dsbd_forest_t.max_tree_nodes may be the bound 1 + gamma*W_S,
+ * but the attention picks a faster kernel shape when it is given the true, usually much smaller
+ * value.  *status: DSBD_DEV_BAD_FOREST when a draw names a beam of another request. */
 int dsbd_forest_build(int32_t R, int32_t gamma, int32_t W_S, const int32_t *req_beam_off,
                       const int32_t *draw_parent, const int32_t *draw_token,
                       int32_t *beam_node_off, int32_t *parent, int32_t *token, int32_t *draft_rank,
-                      int32_t *node_of_draw, int32_t *status, dsbd_stream_t stream);
+                      int32_t *node_of_draw, int32_t *max_tree_nodes, int32_t *status,
+                      dsbd_stream_t stream);
 
 /* KV-cache update at the end of a decode step (Section "Forest-based Parallel Decoding": after
  * the iteration the key-value caches are updated according to the output beams, an output beam

@@ -105,7 +105,7 @@ def load():
     lib.dsbd_kv_commit_paged.restype = C.c_int
     lib.dsbd_kv_commit_paged.argtypes = [_vp] * 22 + [C.c_size_t, _vp, _vp]
     lib.dsbd_forest_build.restype = C.c_int
-    lib.dsbd_forest_build.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [_vp] * 10
+    lib.dsbd_forest_build.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [_vp] * 11
     lib.dsbd_draft_workspace.restype = C.c_size_t
     lib.dsbd_draft_workspace.argtypes = [C.c_int32, C.c_int32, _vp]
     lib.dsbd_draft_layer.restype = C.c_int
@@ -244,10 +244,13 @@ def forest_attention(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_prefix, v_pre
     return out, status
 
 
-def forest_build(req_beam_off, req_beam_off_host, gamma, W_S, draw_parent, draw_token, status=None, stream=None):
+def forest_build(req_beam_off, req_beam_off_host, gamma, W_S, draw_parent, draw_token, status=None, stream=None,
+                 exact=False):
     """dsbd_forest_build.  draw_parent / draw_token: int32 device tensors [gamma, R*W_S].  Returns a
-    Forest whose arrays live on the device (host-side launch facts are the static bounds
-    1 + gamma*W_S nodes per tree and W_S nodes per layer), node_of_draw and the status tensor."""
+    Forest whose arrays live on the device, node_of_draw and the status tensor.  The host-side
+    launch facts are the static bounds 1 + gamma*W_S nodes per tree and W_S nodes per layer; with
+    exact=True the size of the largest tree is read back (4 bytes, one synchronisation of the
+    stream), which lets the attention use its shape for small trees."""
     _require_cuda(req_beam_off, draw_parent, draw_token)
     dev = draw_parent.device
     rbo = np.asarray(req_beam_off_host)
@@ -259,12 +262,15 @@ def forest_build(req_beam_off, req_beam_off_host, gamma, W_S, draw_parent, draw_
     node_of_draw = torch.empty(gamma, R * W_S, dtype=torch.int32, device=dev)
     if status is None:
         status = torch.zeros(1, dtype=torch.int32, device=dev)
+    largest = torch.zeros(1, dtype=torch.int32, device=dev) if exact else None
     rc = load().dsbd_forest_build(R, gamma, W_S, _ptr(req_beam_off), _ptr(draw_parent), _ptr(draw_token),
                                   _ptr(arrays["beam_node_off"]), _ptr(arrays["parent"]), _ptr(arrays["token"]),
-                                  _ptr(arrays["draft_rank"]), _ptr(node_of_draw), _ptr(status), _stream(stream))
+                                  _ptr(arrays["draft_rank"]), _ptr(node_of_draw),
+                                  _ptr(largest) if exact else None, _ptr(status), _stream(stream))
     if rc != OK:
         raise DsbdError("dsbd_forest_build", rc)
-    f = Forest.from_device(R, B, N, gamma, arrays, max_tree_nodes=1 + gamma * W_S,
+    f = Forest.from_device(R, B, N, gamma, arrays,
+                           max_tree_nodes=int(largest.item()) if exact else 1 + gamma * W_S,
                            max_req_beams=int(np.diff(rbo).max()), max_layer_nodes=W_S)
     return f, node_of_draw, status
 

@@ -59,7 +59,8 @@ struct AttnItem { int b, g, t0, t1, last, nparts, slot, rb; };
 struct TcArgs {
     int B, N, Hq, Hkv, group, n_units;
     int max_rows;                     // max over trees of nodes * group
-    int row_blocks;                   // ceil(max_rows / 128)
+    int block_rows;                   // query rows per row block: 64 or 128 (the kernel's Q tile)
+    int row_blocks;                   // ceil(max_rows / block_rows)
     const AttnItem *items;            // nullptr: one item per unit, in unit order
     const int *n_items;               // device count of items (with items)
     float *partial;                   // [slot][max_rows][130]: m_ref, l, O[128]
@@ -196,7 +197,7 @@ __device__ __forceinline__ AttnItem get_item(const TcArgs &a, int it) {
         x.last = 1; x.nparts = 1; x.slot = 0;
     }
     if (x.b >= 0 && x.rb > 0 &&
-        x.rb * kRows >= (a.beam_node_off[x.b + 1] - a.beam_node_off[x.b]) * a.group)
+        x.rb * a.block_rows >= (a.beam_node_off[x.b + 1] - a.beam_node_off[x.b]) * a.group)
         x.b = -1;
     return x;
 }
@@ -366,9 +367,10 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const int n_tree = a.beam_node_off[b + 1] - n_lo;
             const int nt = nt_p + (item.last ? (n_tree + kBN - 1) / kBN : 0);
             const int M = n_tree * a.group;
-            const int r0 = item.rb * kRows;                     // first row of this row block
-            const bool warp_active = r0 + warp * 32 < M;
-            const bool active = r0 + row < M;
+            const int r0 = item.rb * QROWS;                     // first row of this row block
+            // (with the 64-row tile the MMA's rows 64..127 hold no query: never active)
+            const bool warp_active = warp * 32 < QROWS && r0 + warp * 32 < M;
+            const bool active = row < QROWS && r0 + row < M;
             const int node = active ? (r0 + row) / a.group : 0;
             const int hq = g * a.group + (active ? r0 + row - node * a.group : 0);
             // ---- stage Q (rows >= M zero) and the ancestor masks; the previous unit's MMAs are done
@@ -540,12 +542,18 @@ __device__ __forceinline__ void unit_parts(int64_t L, int chunk, int *np, int *p
 }
 
 __global__ void __launch_bounds__(1024)
-k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, int grid, int row_blocks,
-            AttnItem *__restrict__ items, int *__restrict__ n_items, UnitParts *__restrict__ units) {
+k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, const int32_t *__restrict__ beam_node_off,
+            int group, int block_rows, int chunk, int grid, AttnItem *__restrict__ items,
+            int *__restrict__ n_items, UnitParts *__restrict__ units) {
     __shared__ int bucket[1024];
     __shared__ int scan[1024];
     __shared__ int carry;
     const int tid = threadIdx.x, n_units = B * Hkv;
+    // row blocks a tree really has: only those become items
+    auto blocks_of = [&](int b) {
+        const int rows = (beam_node_off[b + 1] - beam_node_off[b]) * group;
+        return rows > block_rows ? (rows + block_rows - 1) / block_rows : 1;
+    };
     bucket[tid] = 0;
     if (tid == 0) carry = 0;
     __syncthreads();
@@ -574,7 +582,7 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, i
                 const int64_t t0 = (int64_t)p * plen;
                 const int64_t t1 = t0 + plen < L ? t0 + plen : L;
                 int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
-                atomicAdd(&bucket[nt < 1023 ? nt : 1023], row_blocks);
+                atomicAdd(&bucket[nt < 1023 ? nt : 1023], blocks_of(b));
             }
         }
         __syncthreads();
@@ -591,12 +599,12 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, i
         __syncthreads();
     }
     const int start = scan[tid] - bucket[1023 - tid];
+    const int total_items = scan[1023];          // all buckets together
     __syncthreads();
     bucket[1023 - tid] = start;                 // bucket[k] becomes the cursor of tile count k
     // The list is read in rounds of `grid` items, CTA k taking entry k of every round.  Odd rounds
     // are stored back to front, so that the CTA with the longest item of one round gets the
     // shortest of the next; the last round is padded with empty entries (b = -1).
-    const int total_items = carry * row_blocks;
     const int padded = (total_items + grid - 1) / grid * grid;
     for (int i = total_items - total_items % grid + tid; i < padded; i += 1024) items[i].b = -1;
     if (tid == 0) *n_items = padded;
@@ -610,7 +618,8 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, int chunk, i
             const int64_t t0 = (int64_t)p * plen;
             const int64_t t1 = t0 + plen < L ? t0 + plen : L;
             const int nt = (int)((t1 - t0 + kBN - 1) / kBN) + (p == np - 1);
-            for (int rb = 0; rb < row_blocks; ++rb) {
+            const int nrb = blocks_of(b);
+            for (int rb = 0; rb < nrb; ++rb) {
                 int pos = atomicAdd(&bucket[nt < 1023 ? nt : 1023], 1);
                 const int round = pos / grid;
                 if (round & 1) pos = round * grid + (grid - 1 - (pos - round * grid));
@@ -694,14 +703,25 @@ struct TcPlan {
     size_t off_items, off_units, off_partial, total;
 };
 
+// Query rows per row block.  Trees of up to 64 rows take the 64-row tile (two CTAs per SM).  So do
+// forests whose AVERAGE tree has at most 64 rows even when the largest is bigger (a sampled
+// forest puts most drafts under a few roots and leaves the other trees tiny): the big trees then
+// run as several 64-row blocks, the many small ones at the faster shape.
+int block_rows_for(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+    const int group = d->Hq / d->Hkv;
+    if (f->max_tree_nodes * group <= 64) return 64;
+    return (int64_t)f->N * group <= (int64_t)64 * f->B ? 64 : kRows;
+}
+
 TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     TcPlan p = {};
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int group = d->Hq / d->Hkv;
-    const bool small_q = f->max_tree_nodes * group <= 64;
+    const int block_rows = block_rows_for(f, d);
+    const bool small_q = block_rows == 64;
     p.grid = small_q ? 2 * sms : sms;
-    const int row_blocks = (f->max_tree_nodes * group + kRows - 1) / kRows;
+    const int row_blocks = (f->max_tree_nodes * group + block_rows - 1) / block_rows;
     const int64_t n_units = (int64_t)f->B * d->Hkv * row_blocks;     // counted with their row blocks
     // Splitting a unit costs a pipeline drain, a Q reload and a partial result per part, so it
     // pays only when there are fewer units than CTAs: then the prefix is cut so that about two
@@ -712,7 +732,10 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     c = (c + kBN - 1) / kBN * kBN;
     p.split = n_units < p.grid && c < d->max_prefix;
     const bool ragged = (int64_t)d->max_prefix * f->B * 100 > (int64_t)d->total_prefix * 115;
-    if (!p.split && !(ragged && n_units > p.grid)) {
+    // trees with several row blocks always go through the plan, which lists only the blocks that
+    // exist (in unit order most (unit, block) pairs of a ragged forest would be empty, and the
+    // CTAs whose stride hits the first blocks would do all the work)
+    if (!p.split && !(ragged && n_units > p.grid) && row_blocks == 1) {
         p.chunk = 0;
         p.items_max = n_units;
         if (p.grid > n_units) p.grid = (int)n_units;
@@ -773,7 +796,8 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;
     a.n_units = f->B * d->Hkv;
     a.max_rows = f->max_tree_nodes * a.group;
-    a.row_blocks = (a.max_rows + kRows - 1) / kRows;
+    a.block_rows = block_rows_for(f, d);
+    a.row_blocks = (a.max_rows + a.block_rows - 1) / a.block_rows;
     a.scale_log2 = d->scale * 1.4426950408889634f;
     a.beam_node_off = f->beam_node_off; a.parent = f->parent; a.prefix_off = prefix_off;
     if (pages) { a.page_table = pages->page_table; a.page_off = pages->page_off; }
@@ -786,15 +810,15 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
         AttnItem *items = reinterpret_cast<AttnItem *>(ws + plan.off_items);
         units = reinterpret_cast<UnitParts *>(ws + plan.off_units);
         int *n_items = reinterpret_cast<int *>(ws);
-        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, plan.chunk, plan.grid, a.row_blocks, items,
-                                            n_items, units);
+        k_attn_plan<<<1, 1024, 0, stream>>>(f->B, d->Hkv, prefix_off, f->beam_node_off, a.group, a.block_rows,
+                                            plan.chunk, plan.grid, items, n_items, units);
         a.items = items;
         a.n_items = n_items;
         a.partial = reinterpret_cast<float *>(ws + plan.off_partial);
     }
     const int grid = plan.grid;
     // up to 64 query rows: 16 KB of Q, three stages, two CTAs per SM; more rows: one CTA per SM
-    const bool small_q = a.max_rows <= 64;
+    const bool small_q = a.block_rows == 64;
 #define DSBD_LAUNCH_TC(QR, ST)                                                                              \
     do {                                                                                                   \
         constexpr uint32_t bytes = smem_bytes(QR, ST);                                                     \

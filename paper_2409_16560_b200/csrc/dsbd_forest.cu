@@ -22,6 +22,7 @@ struct BuildArgs {
     const int32_t *req_beam_off;
     const int32_t *draw_parent, *draw_token;      // [gamma][R * W_S]
     int32_t *beam_node_off, *parent, *token, *draft_rank, *node_of_draw;
+    int32_t *max_tree_nodes;                      // optional: raised to the largest tree (atomicMax)
     int32_t *status;
 };
 
@@ -75,6 +76,7 @@ k_forest_build(BuildArgs a) {
     }
     __syncthreads();
     for (int t = threadIdx.x; t < nb; t += blockDim.x) {
+        if (a.max_tree_nodes) atomicMax(a.max_tree_nodes, tree_size[t + 1] - tree_size[t]);
         const int root = node0 + tree_size[t];
         a.beam_node_off[b0 + t] = root;
         a.parent[root] = -1;
@@ -105,7 +107,7 @@ k_forest_build(BuildArgs a) {
 extern "C" int dsbd_forest_build(int32_t R, int32_t gamma, int32_t W_S, const int32_t *req_beam_off,
                                  const int32_t *draw_parent, const int32_t *draw_token, int32_t *beam_node_off,
                                  int32_t *parent, int32_t *token, int32_t *draft_rank, int32_t *node_of_draw,
-                                 int32_t *status, dsbd_stream_t stream_) {
+                                 int32_t *max_tree_nodes, int32_t *status, dsbd_stream_t stream_) {
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
     if (R <= 0 || gamma <= 0 || W_S <= 0 || !req_beam_off || !draw_parent || !draw_token || !beam_node_off ||
         !parent || !token || !draft_rank || !node_of_draw || !status)
@@ -115,7 +117,7 @@ extern "C" int dsbd_forest_build(int32_t R, int32_t gamma, int32_t W_S, const in
     a.R = R; a.gamma = gamma; a.W_S = W_S;
     a.req_beam_off = req_beam_off; a.draw_parent = draw_parent; a.draw_token = draw_token;
     a.beam_node_off = beam_node_off; a.parent = parent; a.token = token; a.draft_rank = draft_rank;
-    a.node_of_draw = node_of_draw; a.status = status;
+    a.node_of_draw = node_of_draw; a.max_tree_nodes = max_tree_nodes; a.status = status;
     k_forest_build<<<R, kThreads, 0, stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }

@@ -39,6 +39,11 @@ def test_against_the_oracle(R, max_beams, gamma, W_S):
     for k in ("beam_node_off", "parent", "token", "draft_rank"):
         assert np.array_equal(f.dev[k].cpu().numpy(), ref[k]), k
     assert np.array_equal(nod.cpu().numpy(), ref["node_of_draw"])
+    # the size of the largest tree, read back on request
+    i32 = lambda a: torch.as_tensor(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+    f2, _, _ = dsbd.forest_build(i32(rbo), rbo, gamma, W_S, i32(dp), i32(dt), exact=True)
+    assert f2.max_tree_nodes == int(np.diff(ref["beam_node_off"]).max())
+    assert f.max_tree_nodes == 1 + gamma * W_S
 
 
 def test_errors():
