@@ -46,7 +46,9 @@ enum {
                                     request, cache tokens, page-table entries, free pages    */
     DSBD_DEV_BAD_FOREST = 4,     /* an index that contradicts the forest: parent outside its
                                     tree, beam outside its request, too many live beams      */
-    DSBD_DEV_TIMEOUT = 5         /* a bounded wait gave up                                   */
+    DSBD_DEV_TIMEOUT = 5,        /* a bounded wait gave up                                   */
+    DSBD_DEV_BAD_PARAM = 6       /* a per-request width (W_min_r, W_max_r, W_nom_r) below 1, or
+                                    W_max_r below W_min_r                                    */
 };
 
 /* limits of this build */

@@ -16,7 +16,8 @@ OK = 0
 DTYPE_BF16, DTYPE_F32 = 0, 1
 NODE_UNREACHED, NODE_ACCEPTED, NODE_REJECTED, NODE_CUT, NODE_PRUNED = 0, 1, 2, 3, 4
 SRC_DRAFT, SRC_RESIDUAL, SRC_FILL, SRC_EXTRA = 0, 1, 2, 3
-MAX_TREE_NODES = 64
+MAX_TREE_NODES = 64          # DSBD_MAX_TREE_NODES: the CUDA-core attention kernel
+MAX_TREE_NODES_TC = 128      # DSBD_MAX_TREE_NODES_TC: the tensor-core kernel (bf16, d = 128)
 MAX_LIVE = 64
 
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
@@ -144,6 +145,23 @@ def _require_cuda(*tensors):
             raise RuntimeError("dsbd: device tensors required; there is no CPU path")
 
 
+def _node_depths(parent):
+    """Depth of every node (roots 0) by pointer doubling: O(N log depth) array work, no Python
+    loop over the nodes.  A malformed array (a cycle) ends after 32 rounds with wrong depths;
+    the kernels check the forest themselves."""
+    parent = np.asarray(parent, dtype=np.int64)
+    jump = parent.copy()                      # ancestor 2^k levels up, -1 past the root
+    depth = (parent >= 0).astype(np.int64)    # levels climbed so far
+    for _ in range(32):
+        live = jump >= 0
+        if not live.any():
+            break
+        j = jump[live]
+        depth[live] += depth[j]
+        jump[live] = jump[j]
+    return depth
+
+
 class Forest:
     """Device copy of a draft forest plus the host-side facts the launches are sized by."""
 
@@ -173,9 +191,7 @@ class Forest:
         self.max_tree_nodes = int(tree_sizes.max())
         self.max_req_beams = int(np.diff(a["req_beam_off"]).max())
         # nodes per (request, depth)
-        depth = np.zeros(self.N, np.int64)
-        for n, p in enumerate(a["parent"]):
-            depth[n] = 0 if p < 0 else depth[p] + 1
+        depth = _node_depths(a["parent"])
         tree_of = np.repeat(np.arange(self.B), tree_sizes)
         req_of = np.searchsorted(a["req_beam_off"], tree_of, side="right") - 1
         nz = depth > 0

@@ -13,6 +13,7 @@ extern "C" const char *dsbd_status_string(int code) {
         case DSBD_DEV_CAPACITY: return "device: output range too small";
         case DSBD_DEV_BAD_FOREST: return "device: malformed forest";
         case DSBD_DEV_TIMEOUT: return "device: bounded wait gave up";
+        case DSBD_DEV_BAD_PARAM: return "device: per-request width out of range";
         default: return "unknown status";
     }
 }

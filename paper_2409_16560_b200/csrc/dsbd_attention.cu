@@ -11,8 +11,6 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
-#include <stdlib.h>
-#include <string.h>
 
 #include "dsbd_attention.cuh"
 
@@ -247,9 +245,7 @@ extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_des
                            reinterpret_cast<uintptr_t>(v_prefix) | reinterpret_cast<uintptr_t>(out);
     if (bits & 15) return DSBD_ERR_UNSUPPORTED;
 
-    // DSBD_ATTN_IMPL=simt forces the CUDA-core kernel (debugging aid)
-    const char *impl = getenv("DSBD_ATTN_IMPL");
-    if (!(impl && strcmp(impl, "simt") == 0) && attention_tc_supported(f, d))
+    if (attention_tc_supported(f, d))
         return launch_attention_tc(f, d, q, k_new, v_new, k_prefix, v_prefix, prefix_off, out, workspace,
                                    workspace_bytes, status, stream);
 

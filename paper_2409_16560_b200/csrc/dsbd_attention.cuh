@@ -5,9 +5,9 @@
 
 namespace dsbd {
 
-// True when the tcgen05 kernel covers this problem (bf16, d = 128, at most 128 query rows and
-// 64 nodes per tree, a non-empty KV prefix).  n_pages > 0: the caches are paged (k_prefix /
-// v_prefix are then the page pools).
+// True when the tcgen05 kernel covers this problem (bf16, d = 128, at most DSBD_MAX_TREE_NODES_TC
+// nodes and 1024 query rows per tree and KV head, a non-empty KV prefix).  n_pages > 0: the caches
+// are paged (k_prefix / v_prefix are then the page pools).
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages = 0);
 
 // Workspace bytes of the tensor-core path (work plan and partial results of split units).

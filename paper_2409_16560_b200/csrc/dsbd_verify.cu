@@ -83,7 +83,8 @@ __device__ __forceinline__ void load_half_tile(const float *__restrict__ row, in
 // ---------------------------------------------------------------------------------------
 // Dense pass: tile statistics of every (model, row).  Item = (model, row, tile), tile fastest,
 // one warp per item.  rows == nullptr: all n_rows rows; else the listed rows (n_rows read
-// from *n_rows_dev when it is given).
+// from *n_rows_dev when it is given, never more than the n_rows the launch was sized for; a
+// listed row outside [0, N) is skipped -- the kernel that consumes the list reports it).
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
 k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t stride, int V,
@@ -94,7 +95,7 @@ k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    if (n_rows_dev) n_rows = *n_rows_dev;
+    if (n_rows_dev) n_rows = min(max(*n_rows_dev, 0), n_rows);
     const int64_t total = (int64_t)(one_model ? 1 : 2) * n_rows * T;
     for (int64_t item = warp; item < total; item += nwarps) {
         const int t = (int)(item % T);
@@ -102,6 +103,7 @@ k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t
         const int model = (int)(rm / n_rows);
         const int ri = (int)(rm % n_rows);
         const int row = rows ? rows[ri] : ri;
+        if (row < 0 || row >= N) continue;
         const float *z = (model ? zq : zp) + (int64_t)row * stride;
         const bool aligned = (reinterpret_cast<uintptr_t>(z) & 15) == 0;
         float4 v[8];
@@ -136,11 +138,12 @@ __global__ void k_row_finish(const TileStat *__restrict__ stats, int T, int N, i
                              float *__restrict__ lse_p_out, float *__restrict__ lse_q_out) {
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (n_rows_dev) n_rows = *n_rows_dev;
+    if (n_rows_dev) n_rows = min(max(*n_rows_dev, 0), n_rows);
     if (warp >= (int64_t)2 * n_rows) return;
     const int model = (int)(warp / n_rows);
     const int ri = (int)(warp % n_rows);
     const int row = rows ? rows[ri] : ri;
+    if (row < 0 || row >= N) return;
     const TileStat *s = stats + ((int64_t)model * N + row) * T;
     double mx = -INFINITY;
     for (int t = lane; t < T; t += 32) mx = fmax(mx, (double)s[t].mx);
@@ -190,6 +193,7 @@ struct VerifyArgs {
     int32_t *depth_w;
     const float *root_logp, *root_logq;
     int max_m, max_live;
+    int check_widths;            // verification / width selection: per-request widths are validated
     uint32_t extra_layer_bias;   // added to the layer number in the Philox counter of the extra layer
     // outputs
     dsbd_verify_out_t out;
@@ -198,6 +202,7 @@ struct VerifyArgs {
     int select_mode;
     const float *sel_logp, *sel_logq;
     const int32_t *live_off, *live_nodes, *m_in;
+    int sel_rows;             // list entries the dense pass was sized for
     int32_t *width_out;
     float *alpha_out, *tail_out;
     int out_stride;
@@ -931,9 +936,13 @@ k_verify(VerifyArgs a) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b_lo = a.req_beam_off[r], b_hi = a.req_beam_off[r + 1];
     const int n_lo = a.beam_node_off[b_lo], n_hi = a.beam_node_off[b_hi];
-    const int W_min = a.W_min_r ? a.W_min_r[r] : a.W_min;
-    const int W_max = a.W_max_r ? a.W_max_r[r] : a.W_max;
-    const int W_nom = a.W_nom_r ? a.W_nom_r[r] : a.W_nom;
+    int W_min = a.W_min_r ? a.W_min_r[r] : a.W_min;
+    int W_max = a.W_max_r ? a.W_max_r[r] : a.W_max;
+    int W_nom = a.W_nom_r ? a.W_nom_r[r] : a.W_nom;
+    // per-request widths come from device memory: a width below 1 or a cap below the minimum is
+    // reported (after the set-up below) and the request is not verified
+    const bool bad_widths = a.check_widths && (W_min < 1 || W_max < W_min || W_nom < 1);
+    if (bad_widths) { W_min = W_max = W_nom = 1; }
     double *sums_base = a.tile_sums + (int64_t)r * 2 * a.max_m * ((int64_t)a.max_live * a.T);
     const int64_t slot_stride = (int64_t)a.max_live * a.T;
     unsigned long long *ghist = a.hist + (int64_t)r * 2 * (kBins + 1);     // [2 banks][kBins+1]
@@ -1068,7 +1077,14 @@ k_verify(VerifyArgs a) {
             if (a.select_mode) {
                 const int lo = a.live_off[r], hi = a.live_off[r + 1];
                 sh.nA = hi - lo;
-                if (sh.nA > kMaxLive || sh.nA < 0) { sh.err = DSBD_DEV_BAD_FOREST; sh.nA = 0; }
+                // the dense pass before this kernel covered the first sel_rows list entries only
+                if (sh.nA > kMaxLive || sh.nA < 0 || lo < 0 || hi > a.sel_rows) {
+                    sh.err = DSBD_DEV_BAD_FOREST;
+                    sh.nA = 0;
+                }
+                for (int i = 0; i < sh.nA; ++i)
+                    if (a.live_nodes[lo + i] < 0 || a.live_nodes[lo + i] >= a.N) sh.err = DSBD_DEV_BAD_FOREST;
+                if (sh.err) sh.nA = 0;
                 for (int i = 0; i < sh.nA; ++i) {
                     sh.A[i] = a.live_nodes[lo + i];
                     sp_live[i] = (double)a.sel_logp[sh.A[i]];
@@ -1105,6 +1121,7 @@ k_verify(VerifyArgs a) {
     __threadfence();
     cluster.sync();                                   // the histogram banks are zero from here on
     if (!a.select_mode && !st_ok && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_FOREST;
+    if (bad_widths && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_PARAM;
     __syncthreads();
 
     for (int l = 1; l <= n_layers && !sh.done && !sh.err; ++l) {
@@ -1602,6 +1619,17 @@ int check_forest(const dsbd_forest_t *f) {
     return DSBD_OK;
 }
 
+// The widths of the width rule W_L^(l) = min(W_max, max(W_min, W~)): without per-request
+// overrides a zero width or a cap below the minimum is a caller's mistake (a zero-initialised
+// struct), not a setting.
+int check_widths(const dsbd_verify_params_t *p) {
+    if (!p->W_min_r && p->W_min < 1) return DSBD_ERR_INVALID_ARG;
+    if (!p->W_max_r && p->W_max < 1) return DSBD_ERR_INVALID_ARG;
+    if (!p->W_nom_r && p->W_nom < 1) return DSBD_ERR_INVALID_ARG;
+    if (!p->W_min_r && !p->W_max_r && p->W_max < p->W_min) return DSBD_ERR_INVALID_ARG;
+    return DSBD_OK;
+}
+
 int check_params(const dsbd_verify_params_t *p) {
     if (!p || p->V <= 0 || !(p->temperature > 0.f)) return DSBD_ERR_INVALID_ARG;
     if (p->W_min < 1 && !p->W_min_r) return DSBD_ERR_INVALID_ARG;
@@ -1674,6 +1702,8 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
     if (rc) return rc;
     rc = check_params(p);
     if (rc) return rc;
+    rc = check_widths(p);
+    if (rc) return rc;
     if (!logits_p || !logits_q || !root_logp || !root_logq || !out || !workspace || !status)
         return DSBD_ERR_INVALID_ARG;
     if (row_stride < p->V) return DSBD_ERR_INVALID_ARG;
@@ -1714,7 +1744,7 @@ extern "C" int dsbd_verify_step(const dsbd_forest_t *f, const dsbd_verify_params
 #ifdef DSBD_PHASE_TIMING
     a.dbg = reinterpret_cast<unsigned long long *>(ws + L.total) - (size_t)f->R * 256;
 #endif
-    a.out = *out; a.status = status; a.select_mode = 0;
+    a.out = *out; a.status = status; a.select_mode = 0; a.check_widths = 1;
     a.lse_w = lse; a.score_w = score; a.depth_w = depth;
     a.root_logp = root_logp; a.root_logq = root_logq;
     return launch_verify(a, f->R, L.max_live * L.T, stream);
@@ -1944,6 +1974,8 @@ extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_param
     if (rc) return rc;
     rc = check_params(p);
     if (rc) return rc;
+    rc = check_widths(p);
+    if (rc) return rc;
     if (!logits_p || !logits_q || !node_logp || !node_logq || !live_off || !live_nodes || !m ||
         !width || !workspace || !status)
         return DSBD_ERR_INVALID_ARG;
@@ -1961,11 +1993,11 @@ extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_param
     const int max_rows = f->R * L.max_live < f->N ? f->R * L.max_live : f->N;
     const int64_t items = (int64_t)2 * max_rows * L.T;
     k_tile_stats<<<stats_grid(items), kThreads, 0, stream>>>(logits_p, logits_q, row_stride, p->V, L.T,
-                                                            f->N, 0, live_nodes, live_off + f->R, k2, stats);
+                                                            f->N, max_rows, live_nodes, live_off + f->R, k2, stats);
     {
         const int64_t warps = (int64_t)2 * max_rows;
         k_row_finish<<<(unsigned)((warps + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
-            stats, L.T, f->N, 0, live_nodes, live_off + f->R, inv_tau, lse, nullptr, nullptr);
+            stats, L.T, f->N, max_rows, live_nodes, live_off + f->R, inv_tau, lse, nullptr, nullptr);
     }
     if (cudaGetLastError() != cudaSuccess) return DSBD_ERR_CUDA;
 
@@ -1986,9 +2018,9 @@ extern "C" int dsbd_select_width(const dsbd_forest_t *f, const dsbd_verify_param
 #ifdef DSBD_PHASE_TIMING
     a.dbg = reinterpret_cast<unsigned long long *>(ws + L.total) - (size_t)f->R * 256;
 #endif
-    a.status = status; a.select_mode = 1;
+    a.status = status; a.select_mode = 1; a.check_widths = 1;
     a.sel_logp = node_logp; a.sel_logq = node_logq;
-    a.live_off = live_off; a.live_nodes = live_nodes; a.m_in = m;
+    a.live_off = live_off; a.live_nodes = live_nodes; a.m_in = m; a.sel_rows = max_rows;
     a.width_out = width; a.alpha_out = alpha; a.tail_out = tail; a.out_stride = out_stride;
     return launch_verify(a, f->R, L.max_live * L.T, stream);
 }

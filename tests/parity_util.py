@@ -6,10 +6,20 @@ Bars
               accumulation); 1e-4 + 1e-4 * |oracle| for fp32 inputs.
   verify    : widths, node statuses, l_last, output parents / nodes / tokens / sources
               bit-exact.  The only exception: a request whose first differing layer holds a
-              decision the oracle flags as a near tie (|u - ratio| < 1e-5, a CDF boundary
-              within 1e-5 of u, or the width threshold within 1e-5 of the tail probability);
-              such requests are counted, compared up to that layer only, and their number
-              must stay <= ceil(1e-4 * decisions).  Scores: 1e-4 + 1e-5 * |oracle|.
+              decision of the kind that differs which the oracle flags as a near tie.  Such a
+              request is compared up to that layer only and counted in one of two classes:
+                "decision" -- an accept test with |u - ratio| < 1e-5, a layer width whose
+                    threshold lies within 1e-5 of the tail probability, or a top-k / top-p cut
+                    within 1e-5 (relative) of a tie.  At most 1e-4 of the decisions, rounded
+                    DOWN: none at all in a test with fewer than 10 000 decisions.
+                "draw" -- the statuses and widths agree and only a sampled token differs, the
+                    uniform lying within 1e-6 of a boundary of the oracle's cell in the
+                    cumulative distribution.  The CUDA path evaluates cell masses in fp32, the
+                    oracle in fp64, and a large vocabulary has thousands of cells narrower than
+                    the difference, so this class cannot be emptied; it is counted on its own
+                    and must stay below 1e-3 of the decisions (rounded up per test).
+              The session's totals are printed at its end and checked against the same bars.
+              Scores: 1e-4 + 1e-5 * |oracle|.
 """
 import math
 
@@ -72,7 +82,7 @@ def compare_verify(ref, gpu, forest, req_ids=None):
     for n, p in enumerate(parent):
         depth[n] = 0 if p < 0 else depth[p] + 1
     gamma = int(forest["max_depth"])
-    exempt = 0
+    exempt = Exempt()
     tr_start = np.searchsorted(ref["trace_req"], np.arange(R + 1))
     for r in range(R):
         n0, n1 = bno[rbo[r]], bno[rbo[r + 1]]
@@ -117,18 +127,59 @@ def compare_verify(ref, gpu, forest, req_ids=None):
                 assert np.all(np.abs(x - y) <= 1e-4 + 1e-5 * np.abs(x)), (r, k)
             continue
         recs = np.arange(tr_start[r], tr_start[r + 1])
-        near = recs[(ref["trace_layer"][recs] == first_bad) & (ref["trace_near"][recs] != 0)]
-        assert len(near) > 0, (
-            "request %d diverges at layer %d with no near-tie decision there: "
+        recs = recs[ref["trace_layer"][recs] == first_bad]
+        kind, near = ref["trace_kind"][recs], ref["trace_near"][recs] != 0
+        l = first_bad
+        ids = np.arange(n0, n1)[depth[n0:n1] == l]
+        warp_tie = bool(np.any(near & (kind == oracle.TR_WARP)))
+        if l <= gamma and ref["layer_width"][r, l - 1] != gpu["layer_width"][r, l - 1]:
+            ok, cls = warp_tie or bool(np.any(near & (kind == oracle.TR_WIDTH))), "decision"
+        elif l <= gamma and not np.array_equal(ref["node_status"][ids], gpu["node_status"][ids]):
+            ok, cls = warp_tie or bool(np.any(near & (kind == oracle.TR_ACCEPT))), "decision"
+        else:
+            # same statuses and width: a sampled token differs
+            draws = recs[np.isin(kind, (oracle.TR_RESIDUAL, oracle.TR_FILL, oracle.TR_EXTRA))]
+            u, lo, hi = ref["trace_u"][draws], ref["trace_a"][draws], ref["trace_b"][draws]
+            tight = bool(np.any(np.minimum(np.abs(u - lo), np.abs(u - hi)) < DRAW_BAND))
+            ok, cls = tight or warp_tie, ("draw" if tight else "decision")
+        assert ok, (
+            "request %d diverges at layer %d with no near tie of that kind there: "
             "oracle width %s gpu width %s, l_last %d/%d" % (
                 r if req_ids is None else req_ids[r], first_bad, ref["layer_width"][r],
                 gpu["layer_width"][r], ref["l_last"][r], gpu["l_last"][r]))
-        exempt += 1
+        exempt[cls] += 1
     return exempt, len(ref["trace_req"])
 
 
+DRAW_BAND = 1e-6       # distance of a draw's uniform from a cell boundary inside which tokens may differ
+DRAW_RATE = 1e-3       # allowed "draw" class divergences per decision
+
+# exempt requests and decisions of every check_exempt call of this session
+TOTALS = {"decision": 0, "draw": 0, "decisions": 0, "checks": 0}
+
+
+class Exempt(dict):
+    """Counts of exempt requests by class; adds like a vector."""
+
+    def __init__(self, decision=0, draw=0):
+        super().__init__(decision=decision, draw=draw)
+
+    def __add__(self, other):
+        return Exempt(self["decision"] + other["decision"], self["draw"] + other["draw"])
+
+    __radd__ = lambda self, other: self if other == 0 else self.__add__(other)
+
+
 def check_exempt(exempt, decisions):
-    assert exempt <= math.ceil(1e-4 * decisions), (exempt, decisions)
+    """The near-tie allowance of one test (see the module docstring); feeds the session totals."""
+    TOTALS["decision"] += exempt["decision"]
+    TOTALS["draw"] += exempt["draw"]
+    TOTALS["decisions"] += int(decisions)
+    TOTALS["checks"] += 1
+    assert exempt["decision"] <= math.floor(1e-4 * decisions), \
+        "%d exempt decisions in %d decisions" % (exempt["decision"], decisions)
+    assert exempt["draw"] <= math.ceil(DRAW_RATE * decisions), \
+        "%d draws differ inside a tie in %d decisions" % (exempt["draw"], decisions)
 
 
 def attention_close(gpu, ref, bf16):

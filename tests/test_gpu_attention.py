@@ -46,17 +46,24 @@ def _oracle_beams(forest, spec, t, prefix_off, beams, threads=8):
     return nodes, ref
 
 
-@pytest.mark.parametrize("name,n_beams", [("C1", None), ("C2", None), ("C3", 3), ("C4", 4), ("C5", 2)])
+def _spread(B, n):
+    """n tree ids spread evenly over 0..B-1 (all of them when n is None or >= B): the work units
+    of consecutive trees go to consecutive CTAs, so an even spread meets every CTA's every round."""
+    if n is None or n >= B:
+        return list(range(B))
+    return sorted(set(int(round(i * (B - 1) / (n - 1))) for i in range(n)))
+
+
+@pytest.mark.parametrize("name,n_beams", [("C1", None), ("C2", None), ("C3", None), ("C4", 24), ("C5", 74)])
 def test_configs_full_size(name, n_beams):
-    """The GPU runs the full configuration; the oracle checks all trees (C1, C2) or a seeded
-    sample of trees (C3-C5: all nodes and heads of those trees)."""
+    """The GPU runs the full configuration; the oracle checks all trees (C1-C3) or an even
+    spread of trees (C4: 24 of about 72, C5: 74 of 512; all nodes and heads of those trees)."""
     spec = inputs.config(name)
     t = inputs.generate(spec, "cuda", parts=("attention",))
     forest, poff = t["forest"], t["prefix_off"]
     out = _gpu(forest, spec, t, poff)
-    beams = list(range(forest["B"])) if n_beams is None else \
-        sorted(np.random.default_rng(2).choice(forest["B"], size=n_beams, replace=False).tolist())
-    nodes, ref = _oracle_beams(forest, spec, t, poff, beams)
+    beams = _spread(forest["B"], n_beams)
+    nodes, ref = _oracle_beams(forest, spec, t, poff, beams, threads=16)
     attention_close(to_host_f32(out[torch.as_tensor(nodes).cuda()]), ref, bf16=spec["dtype"] == "bf16")
     assert torch.isfinite(out.float()).all()
 

@@ -1,7 +1,7 @@
 """GPU parity of dsbd_draft_layer against the oracle: the beam each draw extends and its token
-are compared bit for bit (a draw whose uniform lies within 1e-5 of a boundary of its cell's CDF
-interval may differ and is counted; at most ceil(1e-4 * draws) such draws), the new cumulative
-score within 1e-4 + 1e-5 |oracle|."""
+are compared bit for bit (a draw whose uniform lies within 1e-6 of a boundary of its cell's CDF
+interval may differ and is counted in the "draw" class of the parity helper), the new
+cumulative score within 1e-4 + 1e-5 |oracle|."""
 import math
 
 import numpy as np
@@ -10,6 +10,7 @@ import torch
 
 import oracle
 import paper_2409_16560_b200 as dsbd
+import parity_util
 
 pytestmark = pytest.mark.gpu
 
@@ -54,13 +55,15 @@ def _compare(ref, gpu, W_r, out_off):
             same = ref["out_parent"][s] == gpu["out_parent"][s] and ref["out_token"][s] == gpu["out_token"][s]
             if not same:
                 u = oracle.uniform(ref_prm["seed"], ref_prm["step"], r, (1 << 29) + ref_layer, 3, k)
-                near = min(abs(u - ref["cdf_lo"][s]), abs(ref["cdf_hi"][s] - u)) < 1e-5
+                near = min(abs(u - ref["cdf_lo"][s]), abs(ref["cdf_hi"][s] - u)) < parity_util.DRAW_BAND
                 assert near, (r, k, ref["out_parent"][s], gpu["out_parent"][s], ref["out_token"][s], gpu["out_token"][s])
                 exempt += 1
                 continue
             x, y = ref["out_logq"][s], gpu["out_logq"][s]
             assert abs(x - y) <= 1e-4 + 1e-5 * abs(x), (r, k, x, y)
-    assert exempt <= math.ceil(1e-4 * draws), (exempt, draws)
+    # a sampled token may differ only inside a tie of the cumulative distribution (fp32 cell masses
+    # on the device, fp64 in the oracle); counted with the verification's draws
+    parity_util.check_exempt(parity_util.Exempt(draw=exempt), draws)
     # slots past a request's W_S draws keep their initial -1
     used = np.zeros(len(gpu["out_token"]), bool)
     for r in range(len(W_r)):

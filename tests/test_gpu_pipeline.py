@@ -103,7 +103,7 @@ def test_three_decode_steps():
         ov = oracle.verify_step(of, vprm, h(zp_nodes), h(zq_nodes), o_sp, o_sq)
         e, dcs = compare_verify(ov, gpu, of)
         exempt += e; decisions += dcs
-        assert e == 0                                        # the chains must stay in lockstep
+        assert not any(e.values())                           # the chains must stay in lockstep
         # ---- cache update, paged
         n_slots = int(oo[-1])
         oc = kvp.kv_commit_paged(of, ov["out_off"], ov["out_width"], ov["out_parent"], ov["out_root_beam"],

@@ -59,3 +59,18 @@ def test_header_is_plain_c(tmp_path):
                    "  (void)f; (void)p; (void)c; return dsbd_status_string(0) == 0; }\n")
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
                     "-I", os.path.join(ROOT, "include"), str(src)], check=True)
+
+
+def test_forest_depths_match_a_plain_walk():
+    """The binding computes node depths (they size the verification's launches) with array
+    operations; a plain walk over the parent array must agree on random trees."""
+    import numpy as np
+    from paper_2409_16560_b200.binding import _node_depths
+    rng = np.random.default_rng(0)
+    for _ in range(100):
+        n = int(rng.integers(1, 400))
+        parent = np.array([-1] + [int(rng.integers(-1, i)) for i in range(1, n)])
+        ref = np.zeros(n, np.int64)
+        for i, p in enumerate(parent):
+            ref[i] = 0 if p < 0 else ref[p] + 1
+        assert np.array_equal(_node_depths(parent), ref)
