@@ -126,13 +126,27 @@ int dsbd_forest_attention_launches(const dsbd_forest_t *forest, const dsbd_attn_
  * DSBD_PAGE_TOKENS) of them, L_b = prefix_off[b+1] - prefix_off[b] (prefix_off only carries the
  * lengths here; desc->total_prefix / max_prefix as before).  Rows of a last page past L_b are
  * never used but must hold finite values.  Supported: bf16, d = 128 (the tensor-core kernel);
- * otherwise UNSUPPORTED.  Workspace: dsbd_forest_attention_workspace. */
+ * otherwise UNSUPPORTED.  Workspace: dsbd_forest_attention_paged_workspace. */
 enum { DSBD_PAGE_TOKENS = 64 };
 
 typedef struct {
     const int32_t *page_table;     /* device                                                 */
     const int64_t *page_off;       /* device [B+1]                                           */
     int64_t n_pages;               /* host: pages in the pool                                */
+    /* dsbd_forest_attention_paged only: the attention of several transformer layers in one call
+     * (Section "Forest-based Parallel Decoding": the large model's forward runs the whole forest
+     * through every layer, each layer attending over its own key-value cache).  All layers share
+     * the forest, the page tables and the work plan; layer l reads its pools at k_pool / v_pool +
+     * l * pool_layer_stride, its new keys/values at k_new / v_new + l * new_layer_stride and its
+     * queries at q + l * q_layer_stride, and writes out + l * q_layer_stride (strides in
+     * elements).  pool_layer_stride must be a multiple of DSBD_PAGE_TOKENS * d and at least one
+     * pool, new_layer_stride a multiple of Hkv * d and at least N * Hkv * d, q_layer_stride a
+     * multiple of 8 and at least N * Hq * d; otherwise INVALID_ARG.  n_layers 0 or 1: one layer,
+     * strides ignored.  (In a model the layers run one after the other, each on the previous
+     * layer's output; a caller that has the queries of several layers at hand -- a benchmark, a
+     * pipeline stage replaying a step -- gets them in one launch with one plan.) */
+    int32_t n_layers;
+    int64_t pool_layer_stride, new_layer_stride, q_layer_stride;
 } dsbd_kv_pages_t;
 
 int dsbd_forest_attention_paged(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
@@ -140,6 +154,11 @@ int dsbd_forest_attention_paged(const dsbd_forest_t *forest, const dsbd_attn_des
                                 const void *k_pool, const void *v_pool, const dsbd_kv_pages_t *pages,
                                 const int64_t *prefix_off, void *out, void *workspace,
                                 size_t workspace_bytes, int32_t *status, dsbd_stream_t stream);
+
+/* Workspace of dsbd_forest_attention_paged for these page tables and layer count (for one layer
+ * the same as dsbd_forest_attention_workspace); 0 for arguments the call would refuse. */
+size_t dsbd_forest_attention_paged_workspace(const dsbd_forest_t *forest, const dsbd_attn_desc_t *desc,
+                                             const dsbd_kv_pages_t *pages);
 
 /* Parameters of the verification (Section "Details", Algorithm 1, and Section
  * "Dynamic-Width Speculative Beam Decoding"). */

@@ -23,7 +23,7 @@ MAX_LIVE = 64
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
            "dsbd_kv_commit", "dsbd_kv_commit_workspace", "dsbd_draft_layer", "dsbd_draft_workspace",
-           "dsbd_forest_attention_paged", "dsbd_kv_commit_paged", "dsbd_kv_commit_paged_workspace",
+           "dsbd_forest_attention_paged", "dsbd_forest_attention_paged_workspace", "dsbd_kv_commit_paged", "dsbd_kv_commit_paged_workspace",
            "dsbd_forest_build",
            "dsbd_status_string"]
 
@@ -99,6 +99,8 @@ def load():
     lib.dsbd_kv_commit_workspace.argtypes = [_vp, _vp]
     lib.dsbd_kv_commit.restype = C.c_int
     lib.dsbd_kv_commit.argtypes = [_vp] * 19 + [C.c_size_t, _vp, _vp]
+    lib.dsbd_forest_attention_paged_workspace.restype = C.c_size_t
+    lib.dsbd_forest_attention_paged_workspace.argtypes = [_vp, _vp, _vp]
     lib.dsbd_forest_attention_paged.restype = C.c_int
     lib.dsbd_forest_attention_paged.argtypes = [_vp] * 11 + [C.c_size_t, _vp, _vp]
     lib.dsbd_kv_commit_paged_workspace.restype = C.c_size_t
@@ -292,21 +294,31 @@ def forest_build(req_beam_off, req_beam_off_host, gamma, W_S, draw_parent, draw_
 
 
 class KvPagesT(C.Structure):
-    _fields_ = [("page_table", _vp), ("page_off", _vp), ("n_pages", C.c_int64)]
+    _fields_ = [("page_table", _vp), ("page_off", _vp), ("n_pages", C.c_int64), ("n_layers", C.c_int32),
+                ("pool_layer_stride", C.c_int64), ("new_layer_stride", C.c_int64), ("q_layer_stride", C.c_int64)]
 
 
 def forest_attention_paged(forest, Hq, Hkv, d, scale, q, k_new, v_new, k_pool, v_pool, page_table, page_off,
                            prefix_off, prefix_off_host, out=None, workspace=None, status=None, stream=None):
-    """dsbd_forest_attention_paged; k_pool / v_pool: [n_pages, Hkv, 64, d]; returns (out, status)."""
+    """dsbd_forest_attention_paged; k_pool / v_pool: [n_pages, Hkv, 64, d]; returns (out, status).
+    Several transformer layers in one call: pools [n_layers, n_pages, Hkv, 64, d], q [n_layers, N,
+    Hq, d], k_new / v_new [n_layers, N, Hkv, d]; the leading strides are passed on as they are."""
     _require_cuda(q, k_new, v_new, k_pool, v_pool, page_table, page_off, prefix_off)
     assert page_table.dtype == torch.int32 and page_off.dtype == torch.int64
     f = forest.struct()
     desc = _attn_desc(Hq, Hkv, d, q.dtype, scale, prefix_off_host)
     pages = KvPagesT()
-    pages.page_table, pages.page_off, pages.n_pages = _ptr(page_table), _ptr(page_off), int(k_pool.shape[0])
+    pages.page_table, pages.page_off, pages.n_pages = _ptr(page_table), _ptr(page_off), int(k_pool.shape[-4])
     if out is None:
         out = torch.empty_like(q)
-    need = int(load().dsbd_forest_attention_workspace(C.addressof(f), C.addressof(desc)))
+    if k_pool.dim() == 5:
+        pages.n_layers = int(k_pool.shape[0])
+        assert q.dim() == 4 and k_new.dim() == 4 and q.shape[0] == k_new.shape[0] == pages.n_layers
+        assert v_pool.stride(0) == k_pool.stride(0) and v_new.stride(0) == k_new.stride(0)
+        assert out.stride(0) == q.stride(0)
+        pages.pool_layer_stride, pages.new_layer_stride = int(k_pool.stride(0)), int(k_new.stride(0))
+        pages.q_layer_stride = int(q.stride(0))
+    need = int(load().dsbd_forest_attention_paged_workspace(C.addressof(f), C.addressof(desc), C.addressof(pages)))
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
     if status is None:

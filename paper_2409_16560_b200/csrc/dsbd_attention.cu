@@ -265,6 +265,13 @@ extern "C" int dsbd_forest_attention(const dsbd_forest_t *f, const dsbd_attn_des
                       : launch_simt<__nv_bfloat16, 128>(a, units, stream);
 }
 
+extern "C" size_t dsbd_forest_attention_paged_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d,
+                                                        const dsbd_kv_pages_t *pages) {
+    if (check(f, d) != DSBD_OK || !pages || pages->n_pages <= 0 || pages->n_layers < 0) return 0;
+    if (!attention_tc_supported(f, d, pages->n_pages) || !attention_tc_layers_ok(f, d, pages)) return 0;
+    return attention_tc_workspace(f, d, pages->n_layers);
+}
+
 extern "C" int dsbd_forest_attention_paged(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q,
                                            const void *k_new, const void *v_new, const void *k_pool,
                                            const void *v_pool, const dsbd_kv_pages_t *pages,
@@ -277,7 +284,9 @@ extern "C" int dsbd_forest_attention_paged(const dsbd_forest_t *f, const dsbd_at
         pages->n_pages <= 0 || !prefix_off || !out || !status)
         return DSBD_ERR_INVALID_ARG;
     if (!attention_tc_supported(f, d, pages->n_pages)) return DSBD_ERR_UNSUPPORTED;
-    if (workspace_bytes < attention_tc_workspace(f, d) || !workspace) return DSBD_ERR_WORKSPACE_TOO_SMALL;
+    if (pages->n_layers < 0 || !attention_tc_layers_ok(f, d, pages)) return DSBD_ERR_INVALID_ARG;
+    if (workspace_bytes < attention_tc_workspace(f, d, pages->n_layers) || !workspace)
+        return DSBD_ERR_WORKSPACE_TOO_SMALL;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) |
                            reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(k_pool) |
                            reinterpret_cast<uintptr_t>(v_pool) | reinterpret_cast<uintptr_t>(out);

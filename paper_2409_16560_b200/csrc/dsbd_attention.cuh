@@ -10,8 +10,13 @@ namespace dsbd {
 // are paged (k_prefix / v_prefix are then the page pools).
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages = 0);
 
-// Workspace bytes of the tensor-core path (work plan and partial results of split units).
-size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);
+// Workspace bytes of the tensor-core path (work plan and partial results of split units; the
+// partial results once per transformer layer of the call).
+size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int n_layers = 1);
+
+// True when the layer count and layer strides of a paged call can be served (strides are whole
+// rows of the operands' tensor maps and the row coordinates stay below 2^31).
+bool attention_tc_layers_ok(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const dsbd_kv_pages_t *pages);
 
 // Kernels one call launches: the attention kernel, plus the plan and the combine kernel when used.
 int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d);

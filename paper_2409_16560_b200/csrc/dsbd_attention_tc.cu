@@ -24,6 +24,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <algorithm>
+
 #include "dsbd_attention.cuh"
 
 using namespace dsbd;
@@ -72,6 +74,13 @@ struct TcArgs {
     const __nv_bfloat16 *q;
     __nv_bfloat16 *out;
     int32_t *status;
+    // several transformer layers in one launch (paged caches): layer l uses the same plan, page
+    // tables and forest; its pools, new keys/values, queries and outputs lie l strides further
+    int n_layers;                     // >= 1
+    int pool_layer_rows;              // rows of the pool map between consecutive layers
+    int new_layer_rows;               // rows of the k_new / v_new maps between consecutive layers
+    int64_t q_layer_stride;           // elements between consecutive layers' q (and out)
+    int slots_per_layer;              // partial-result slots of one layer
 };
 
 struct Barriers {
@@ -253,8 +262,9 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             uint32_t tile = 0;
             bool ok = true;
             const int n_items = item_count(a);
-            for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
-                const AttnItem item = get_item(a, u);
+            for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
+                const int layer = u / n_items;
+                const AttnItem item = get_item(a, u - layer * n_items);
                 if (item.b < 0) continue;
                 const int b = item.b, g = item.g;
                 const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
@@ -275,7 +285,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     if (j < nt_p) {
                         int y = (int)(row0 + (int64_t)j * kBN);
                         if (pages) {
-                            y = (page_next * a.Hkv + g) * kBN;
+                            y = (page_next * a.Hkv + g) * kBN + layer * a.pool_layer_rows;
                             if (j + 1 < nt_p) page_next = pages[j + 1];
                         }
                         tma_load_2d(ks, &map_kp, 0, y, &sb.kv_full[s]);
@@ -283,7 +293,8 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                         tma_load_2d(vs, &map_vp, 0, y, &sb.kv_full[s]);
                         tma_load_2d(vs + kTileBytes / 2, &map_vp, 64, y, &sb.kv_full[s]);
                     } else {
-                        const int x = g * kD, y = n_lo + (j - nt_p) * kBN;      // tree tile j - nt_p
+                        const int x = g * kD;                                  // tree tile j - nt_p
+                        const int y = n_lo + (j - nt_p) * kBN + layer * a.new_layer_rows;
                         tma_load_2d(ks, &map_kn, x, y, &sb.kv_full[s]);
                         tma_load_2d(ks + kTileBytes / 2, &map_kn, x + 64, y, &sb.kv_full[s]);
                         tma_load_2d(vs, &map_vn, x, y, &sb.kv_full[s]);
@@ -310,8 +321,8 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             bool ok = true;
             const uint64_t qd = desc_k_major(smem_u32(q_s));
             const int n_items = item_count(a);
-            for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
-                const AttnItem item = get_item(a, u);
+            for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
+                const AttnItem item = get_item(a, u % n_items);
                 if (item.b < 0) continue;
                 const int nt = (item.t1 - item.t0 + kBN - 1) / kBN + (item.last ? tree_tiles(a, item.b) : 0);
                 ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
@@ -357,8 +368,8 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
         uint32_t tile = 0, unit = 0;
         bool ok = true;
         const int n_items = item_count(a);
-        for (int u = blockIdx.x; u < n_items && ok; u += gridDim.x) {
-            const AttnItem item = get_item(a, u);
+        for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
+            const AttnItem item = get_item(a, u % n_items);
             if (item.b < 0) continue;
             const int b = item.b, g = item.g;
             const int64_t L = item.t1;                         // tokens beyond t1 belong to other items
@@ -376,12 +387,13 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             // ---- stage Q (rows >= M zero) and the ancestor masks; the previous unit's MMAs are done
             {
                 const int t128 = threadIdx.x;                        // 0..127
+                const __nv_bfloat16 *q_l = a.q + (int64_t)(u / n_items) * a.q_layer_stride;
                 for (int i = t128; i < QROWS * 16; i += 128) {
                     const int r = i >> 4, c = i & 15;                // row, 16-byte chunk of the 256-byte row
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (r0 + r < M) {
                         const int nd = (r0 + r) / a.group, hh = g * a.group + (r0 + r - nd * a.group);
-                        v = *reinterpret_cast<const uint4 *>(a.q + ((int64_t)(n_lo + nd) * a.Hq + hh) * kD + c * 8);
+                        v = *reinterpret_cast<const uint4 *>(q_l + ((int64_t)(n_lo + nd) * a.Hq + hh) * kD + c * 8);
                     }
                     const int half = c >> 3, cc = c & 7;
                     *reinterpret_cast<uint4 *>(q_s + half * (QROWS * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
@@ -476,9 +488,11 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             if (warp_active) {
+                const int layer = u / n_items;
                 if (item.nparts == 1) {
                     const float inv = active ? 1.f / l_run : 0.f;
-                    __nv_bfloat16 *dst = a.out + ((int64_t)(n_lo + node) * a.Hq + hq) * kD;
+                    __nv_bfloat16 *dst = a.out + (int64_t)layer * a.q_layer_stride +
+                                         ((int64_t)(n_lo + node) * a.Hq + hq) * kD;
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t ov[32];
@@ -498,7 +512,8 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     }
                 } else {
                     // partial result of this part of the unit: reference maximum, row sum, raw O
-                    float *dst = a.partial + ((int64_t)item.slot * a.max_rows + r0 + row) * 130;
+                    float *dst = a.partial +
+                                 (((int64_t)layer * a.slots_per_layer + item.slot) * a.max_rows + r0 + row) * 130;
                     if (active) { dst[0] = m_ref; dst[1] = l_run; }
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
@@ -635,10 +650,12 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, const int32_
 // Merge the parts of every split unit: out = sum_c O_c 2^(m_c - m) / sum_c l_c 2^(m_c - m).
 __global__ void __launch_bounds__(128)
 k_attn_combine(TcArgs a, const UnitParts *__restrict__ units) {
-    const int u = blockIdx.x;
+    const int u = blockIdx.x, layer = blockIdx.y;
     const UnitParts up = units[u];
     if (up.nparts <= 1) return;
     const int b = u / a.Hkv, g = u - b * a.Hkv;
+    a.partial += (int64_t)layer * a.slots_per_layer * a.max_rows * 130;
+    a.out += (int64_t)layer * a.q_layer_stride;
     const int n_lo = a.beam_node_off[b];
     const int M = (a.beam_node_off[b + 1] - n_lo) * a.group;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -713,7 +730,7 @@ int block_rows_for(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     return (int64_t)f->N * group <= (int64_t)64 * f->B ? 64 : kRows;
 }
 
-TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int n_layers = 1) {
     TcPlan p = {};
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -752,7 +769,8 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     p.off_units = off;   off = align_up(off + sizeof(UnitParts) * (size_t)f->B * d->Hkv, 256);
     p.off_partial = off;
     if (p.split)
-        off = align_up(off + sizeof(float) * 130 * (size_t)p.items_max * (size_t)(f->max_tree_nodes * group), 256);
+        off = align_up(off + sizeof(float) * 130 * (size_t)n_layers * (size_t)p.items_max *
+                                 (size_t)(f->max_tree_nodes * group), 256);
     p.total = off;
     return p;
 }
@@ -760,6 +778,27 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
 }  // namespace
 
 namespace dsbd {
+
+// Layer count and strides of a paged call, checked: the layers of one call share one tensor map
+// per operand, so a layer stride must be a whole number of map rows.
+struct LayerDims { int n_layers, pool_rows, new_rows; int64_t q_stride; bool ok; };
+
+LayerDims layer_dims(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const dsbd_kv_pages_t *pages) {
+    LayerDims L = {1, 0, 0, 0, true};
+    if (!pages || pages->n_layers <= 1) return L;
+    L.n_layers = pages->n_layers;
+    const int64_t page_elems = (int64_t)d->Hkv * kBN * kD, new_row = (int64_t)d->Hkv * kD;
+    const int64_t ps = pages->pool_layer_stride, ns = pages->new_layer_stride, qs = pages->q_layer_stride;
+    L.ok = ps >= pages->n_pages * page_elems && ps % ((int64_t)kBN * kD) == 0 &&
+           ns >= (int64_t)f->N * new_row && ns % new_row == 0 &&
+           qs >= (int64_t)f->N * d->Hq * kD && qs % 8 == 0;
+    if (!L.ok) return L;
+    const int64_t pool_rows = ps / kD, new_rows = ns / new_row;
+    // row coordinates of the maps are 32-bit
+    if (pool_rows * L.n_layers >= ((int64_t)1 << 31) || new_rows * L.n_layers >= ((int64_t)1 << 31)) L.ok = false;
+    L.pool_rows = (int)pool_rows; L.new_rows = (int)new_rows; L.q_stride = qs;
+    return L;
+}
 
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages) {
     if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
@@ -772,7 +811,13 @@ bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, i
     return encode_fn() != nullptr;
 }
 
-size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) { return make_plan(f, d).total; }
+bool attention_tc_layers_ok(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const dsbd_kv_pages_t *pages) {
+    return layer_dims(f, d, pages).ok;
+}
+
+size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int n_layers) {
+    return make_plan(f, d, n_layers < 1 ? 1 : n_layers).total;
+}
 
 int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     const TcPlan p = make_plan(f, d);
@@ -784,12 +829,18 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
                         void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream,
                         const dsbd_kv_pages_t *pages) {
     CUtensorMap kp, vp, kn, vn;
-    const uint64_t prows = pages ? (uint64_t)pages->n_pages * d->Hkv * kBN : (uint64_t)d->total_prefix * d->Hkv;
+    const LayerDims LD = layer_dims(f, d, pages);
+    if (!LD.ok) return DSBD_ERR_INVALID_ARG;
+    const int nl = LD.n_layers;
+    // one map per operand over all layers: layer l starts l * (layer stride in rows) further down
+    const uint64_t prows = pages ? (uint64_t)pages->n_pages * d->Hkv * kBN + (uint64_t)(nl - 1) * LD.pool_rows
+                                 : (uint64_t)d->total_prefix * d->Hkv;
+    const uint64_t nrows = (uint64_t)f->N + (uint64_t)(nl - 1) * LD.new_rows;
     if (!make_map(&kp, k_prefix, kD, prows, kD * 2) || !make_map(&vp, v_prefix, kD, prows, kD * 2) ||
-        !make_map(&kn, k_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2) ||
-        !make_map(&vn, v_new, (uint64_t)d->Hkv * kD, (uint64_t)f->N, (uint64_t)d->Hkv * kD * 2))
+        !make_map(&kn, k_new, (uint64_t)d->Hkv * kD, nrows, (uint64_t)d->Hkv * kD * 2) ||
+        !make_map(&vn, v_new, (uint64_t)d->Hkv * kD, nrows, (uint64_t)d->Hkv * kD * 2))
         return DSBD_ERR_CUDA;
-    const TcPlan plan = make_plan(f, d);
+    const TcPlan plan = make_plan(f, d, nl);
     if (workspace_bytes < plan.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
     char *ws = static_cast<char *>(workspace);
     TcArgs a = {};
@@ -804,6 +855,8 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.q = static_cast<const __nv_bfloat16 *>(q);
     a.out = static_cast<__nv_bfloat16 *>(out);
     a.status = status;
+    a.n_layers = nl; a.pool_layer_rows = LD.pool_rows; a.new_layer_rows = LD.new_rows;
+    a.q_layer_stride = LD.q_stride; a.slots_per_layer = (int)plan.items_max;
     UnitParts *units = nullptr;
     if (plan.chunk > 0) {
         if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
@@ -816,7 +869,14 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
         a.n_items = n_items;
         a.partial = reinterpret_cast<float *>(ws + plan.off_partial);
     }
-    const int grid = plan.grid;
+    // more layers mean more items for the same plan: the grid may grow back to the SM-filling size
+    int grid = plan.grid;
+    if (nl > 1) {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int full = a.block_rows == 64 ? 2 * sms : sms;
+        if (plan.chunk == 0) grid = (int)std::min<int64_t>((int64_t)plan.items_max * nl, full);
+    }
     // up to 64 query rows: 16 KB of Q, three stages, two CTAs per SM; more rows: one CTA per SM
     const bool small_q = a.block_rows == 64;
 #define DSBD_LAUNCH_TC(QR, ST)                                                                              \
@@ -830,7 +890,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     if (small_q) DSBD_LAUNCH_TC(64, 3);
     else DSBD_LAUNCH_TC(128, 3);
 #undef DSBD_LAUNCH_TC
-    if (plan.split) k_attn_combine<<<a.n_units, 128, 0, stream>>>(a, units);
+    if (plan.split) k_attn_combine<<<dim3(a.n_units, nl), 128, 0, stream>>>(a, units);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 

@@ -45,6 +45,11 @@ CONFIGS = {
                V=128256, sigma_p=3.0, zipf=True, sigma_n=1.0, temperature=1.0, seed=0),
     "C5": dict(R=64, W=8, tree=_chain(8), Hq=32, Hkv=8, d=128, dtype="bf16", prefix=(4096, 4096),
                V=128256, sigma_p=3.0, zipf=True, sigma_n=1.0, temperature=0.8, seed=7),
+    # a sixth shape beside the five benchmark configurations: 40 heads of 128 without grouping and
+    # a 32000-token vocabulary, the dimensions of the 13B model of the paper's experiments; the
+    # batch, widths, depth and prefix length are this build's choice
+    "C6": dict(R=8, W=4, tree=_chain(5), Hq=40, Hkv=40, d=128, dtype="bf16", prefix=(2048, 2048),
+               V=32000, sigma_p=3.0, zipf=True, sigma_n=1.0, temperature=1.0, seed=0),
 }
 
 

@@ -54,9 +54,10 @@ def _spread(B, n):
     return sorted(set(int(round(i * (B - 1) / (n - 1))) for i in range(n)))
 
 
-@pytest.mark.parametrize("name,n_beams", [("C1", None), ("C2", None), ("C3", None), ("C4", 24), ("C5", 74)])
+@pytest.mark.parametrize("name,n_beams", [("C1", None), ("C2", None), ("C3", None), ("C4", 24), ("C5", 74),
+                                          ("C6", None)])
 def test_configs_full_size(name, n_beams):
-    """The GPU runs the full configuration; the oracle checks all trees (C1-C3) or an even
+    """The GPU runs the full configuration; the oracle checks all trees (C1-C3, C6) or an even
     spread of trees (C4: 24 of about 72, C5: 74 of 512; all nodes and heads of those trees)."""
     spec = inputs.config(name)
     t = inputs.generate(spec, "cuda", parts=("attention",))

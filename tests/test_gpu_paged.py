@@ -44,7 +44,8 @@ def _gpu_paged(forest, spec, t, poff, pg):
     return out
 
 
-@pytest.mark.parametrize("name,kw,n_beams", [("C2", {}, None), ("C3", {}, 3), ("C4", {}, 4), ("C5", dict(R=3), 2)])
+@pytest.mark.parametrize("name,kw,n_beams", [("C2", {}, None), ("C3", {}, 3), ("C4", {}, 4), ("C5", dict(R=3), 2),
+                                             ("C6", {}, 8)])
 def test_paged_attention_configs(name, kw, n_beams):
     spec = inputs.config(name, **kw)
     t = inputs.generate(spec, "cuda", parts=("attention",))
@@ -80,6 +81,68 @@ def test_paged_attention_with_row_blocks():
     out = _gpu_paged(forest, spec, t, poff, pg)
     nodes, ref = _oracle_beams(forest, spec, t, poff, list(range(len(trees))))
     attention_close(to_host_f32(out), ref, bf16=True)
+
+
+@pytest.mark.parametrize("L,sizes,Hq,Hkv,n_layers", [
+    ([700, 64, 65, 130, 1], [9, 1, 16, 5, 2], 8, 2, 3),       # 64-row tile, units in plain order
+    ([6000, 4000], [7, 7], 8, 2, 4),                          # few units: split prefixes, merged per layer
+    ([900, 100, 2500, 64, 333], [45, 2, 30, 64, 12], 16, 4, 2),   # row blocks and a planned order
+    ([300, 200, 257, 40], [5, 5, 5, 5], 40, 40, 5),           # 40 heads of 128 (the Llama-2-13B shape)
+])
+def test_attention_of_several_layers_in_one_call(L, sizes, Hq, Hkv, n_layers):
+    """All transformer layers of a step in one launch: every layer has its own pools, new
+    keys/values and queries, all share the forest and the page tables.  Each layer must match the
+    oracle's attention on that layer's caches."""
+    rng = np.random.default_rng(n_layers * 10 + len(L))
+    rand_tree = lambda n: [-1] + [int(rng.integers(0, i)) for i in range(1, n)]
+    trees = [rand_tree(n) for n in sizes]
+    layers = [_custom(rng, trees, L, Hq, Hkv, 128, torch.bfloat16) for _ in range(n_layers)]
+    forest, spec, _, poff = layers[0]
+    pgs = [_paged(t, poff, Hkv, 128, 4, np.random.default_rng(5)) for _, _, t, _ in layers]   # same page ids
+    assert all(torch.equal(pg["table"], pgs[0]["table"]) for pg in pgs)
+    stack = lambda key: torch.stack([t[key] for _, _, t, _ in layers]).contiguous()
+    k_pool = torch.stack([pg["k_pool"] for pg in pgs]).contiguous()
+    v_pool = torch.stack([pg["v_pool"] for pg in pgs]).contiguous()
+    f = dsbd.Forest(forest, "cuda")
+    out, st = dsbd.forest_attention_paged(f, Hq, Hkv, 128, inputs.default_scale(128), stack("q"), stack("k_new"),
+                                          stack("v_new"), k_pool, v_pool, pgs[0]["table"], pgs[0]["page_off"],
+                                          torch.as_tensor(poff).cuda(), poff)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    for l, (_, _, t, _) in enumerate(layers):
+        nodes, ref = _oracle_beams(forest, spec, t, poff, list(range(len(trees))))
+        attention_close(to_host_f32(out[l]), ref, bf16=True)
+        # and bit for bit what a call for this layer alone gives
+        single = _gpu_paged(forest, spec, t, poff, pgs[l])
+        assert torch.equal(single, out[l])
+
+
+def test_layer_strides_are_validated():
+    """A layer stride that is not a whole number of tensor-map rows, or shorter than one layer's
+    tensor, is refused before anything is launched (the workspace query answers 0)."""
+    import ctypes as C
+    from paper_2409_16560_b200 import binding as bd
+    rng = np.random.default_rng(3)
+    forest, spec, t, poff = _custom(rng, [[-1, 0]], [100], 8, 2, 128, torch.bfloat16)
+    pg = _paged(t, poff, 2, 128, 1, rng)
+    f = dsbd.Forest(forest, "cuda").struct()
+    desc = bd._attn_desc(8, 2, 128, torch.bfloat16, 0.1, poff)
+    n_pages = int(pg["k_pool"].shape[0])
+    pool, new, q = n_pages * 2 * 64 * 128, forest["N"] * 2 * 128, forest["N"] * 8 * 128
+
+    def query(n_layers, ps, ns, qs):
+        pages = bd.KvPagesT()
+        pages.page_table, pages.page_off, pages.n_pages = bd._ptr(pg["table"]), bd._ptr(pg["page_off"]), n_pages
+        pages.n_layers, pages.pool_layer_stride, pages.new_layer_stride, pages.q_layer_stride = n_layers, ps, ns, qs
+        return int(bd.load().dsbd_forest_attention_paged_workspace(C.addressof(f), C.addressof(desc),
+                                                                   C.addressof(pages)))
+    assert query(2, pool, new, q) > 0
+    assert query(1, 0, 0, 0) > 0                      # one layer: strides ignored
+    assert query(2, pool + 64, new, q) == 0           # not a whole 64-token page row
+    assert query(2, pool - 64 * 128, new, q) == 0     # layers would overlap
+    assert query(2, pool, new + 128, q) == 0          # not a whole row of the new keys
+    assert query(2, pool, new, q - 8) == 0
+    assert query(-1, pool, new, q) == 0
 
 
 def test_unsupported_shapes_are_refused():

@@ -37,7 +37,7 @@ def _both(data, steps, thresh=None):
 
 
 @pytest.mark.parametrize("name,steps", [("C1", range(40)), ("C2", range(40)), ("C3", range(6)),
-                                        ("C4", range(3))])
+                                        ("C4", range(3)), ("C6", range(6))])
 def test_configs_full_size(name, steps):
     data = inputs.generate(inputs.config(name), "cuda", parts=("verify",))
     _both(data, steps)
@@ -174,7 +174,8 @@ def test_peaky_distributions_use_the_exact_fallback():
     assert fallbacks > 0
 
 
-@pytest.mark.parametrize("name,steps", [("C1", range(30)), ("C2", range(30)), ("C3", range(4)), ("C4", range(3))])
+@pytest.mark.parametrize("name,steps", [("C1", range(30)), ("C2", range(30)), ("C3", range(4)), ("C4", range(3)),
+                                        ("C6", range(4))])
 def test_configs_with_the_papers_warping(name, steps):
     """top-k 10 / top-p 0.8 on the joint distributions, the setting of the paper's experiments."""
     data = inputs.generate(inputs.config(name), "cuda", parts=("verify",), draft_top_k=10, draft_top_p=0.8)
