@@ -393,10 +393,12 @@ def main():
     total_ms = max_over_ranks(total_local, world, dev)
     attn_ms, ver_ms = float(np.median(t_attn)), float(np.median(t_ver))
     assert int(status.item()) == 0, "device status %d" % int(status.item())
-    st = vout["req_stats"].cpu().numpy().reshape(-1, 4).astype(float)
+    st = vout["req_stats"].cpu().numpy().reshape(-1, 8).astype(float)
     verify_stats = {"layers_per_request": float(st[:, 0].mean()), "accept_tests_per_request": float(st[:, 1].mean()),
                     "exact_recomputations_per_request": float(st[:, 2].mean()),
                     "extra_completion_passes_per_request": float(st[:, 3].mean()),
+                    "near_tie_accept_tests": int(st[:, 4].sum()), "consulted_row_pairs_per_request": float(st[:, 5].mean()),
+                    "overflowed_histograms": int(st[:, 6].sum()),
                     "output_beams_per_request": float(vout["out_width"].float().mean().item())}
 
     # the dense logits pass alone (the kernel the verify roofline is quoted on)

@@ -186,6 +186,8 @@ typedef struct {
     float top_p;
 } dsbd_verify_params_t;
 
+#define DSBD_REQ_STATS 8
+
 /* node_status */
 enum { DSBD_NODE_UNREACHED = 0, DSBD_NODE_ACCEPTED = 1, DSBD_NODE_REJECTED = 2,
        DSBD_NODE_CUT = 3, DSBD_NODE_PRUNED = 4 };
@@ -214,9 +216,13 @@ typedef struct {
     float   *lse_p;         /* [N]  log-sum-exp of each tempered logits row                  */
     float   *lse_q;
     int32_t *req_error;     /* [R]  0 or a DSBD_DEV_* code                                   */
-    int32_t *req_stats;     /* [R*4] or NULL: per request {layers verified, accept tests made,
-                                    residual masses that had to be recomputed exactly by a pass
-                                    over the rows, extra passes made for completion draws}   */
+    int32_t *req_stats;     /* [R*DSBD_REQ_STATS] or NULL, per request: 0 layers verified, 1 accept
+                                    tests made, 2 residual masses recomputed exactly by a pass over
+                                    the rows, 3 extra passes made for completion draws, 4 accept
+                                    tests with |u - ratio| < 1e-5 (near ties), 5 logits row pairs
+                                    consulted after the dense pass (live parents summed over the
+                                    verified layers), 6 layers whose histogram overflowed a word and
+                                    fell back to exact passes, 7 reserved (0)                     */
 } dsbd_verify_out_t;
 
 /* One verification step (Algorithm 1 with the dynamic width of Eqs. for P, P~, alpha_j, W_L):

@@ -19,6 +19,7 @@ SRC_DRAFT, SRC_RESIDUAL, SRC_FILL, SRC_EXTRA = 0, 1, 2, 3
 MAX_TREE_NODES = 64          # DSBD_MAX_TREE_NODES: the CUDA-core attention kernel
 MAX_TREE_NODES_TC = 128      # DSBD_MAX_TREE_NODES_TC: the tensor-core kernel (bf16, d = 128)
 MAX_LIVE = 64
+REQ_STATS = 8                # DSBD_REQ_STATS: counters per request in req_stats
 
 EXPORTS = ["dsbd_forest_attention", "dsbd_forest_attention_workspace", "dsbd_forest_attention_launches", "dsbd_verify_step",
            "dsbd_verify_workspace", "dsbd_select_width", "dsbd_node_stats", "dsbd_node_stats_static",
@@ -541,7 +542,7 @@ def alloc_verify_out(forest, out_off_host, device):
         "lse_p": torch.zeros(N, dtype=f32, device=device),
         "lse_q": torch.zeros(N, dtype=f32, device=device),
         "req_error": torch.zeros(R, dtype=i32, device=device),
-        "req_stats": torch.zeros(R * 4, dtype=i32, device=device),
+        "req_stats": torch.zeros(R * REQ_STATS, dtype=i32, device=device),
     }
     return o
 

@@ -22,8 +22,9 @@
 // alpha_j = 1 - c_{j+1}/c_j and the accept ratio of a draft x at run position j is
 // max(rho(x) - s_{j-1}, 0) / c_j with rho = p_beam(x)/q_beam(x).  F(s) = P(rho > s) - s Q(rho > s)
 // only needs the p and q mass above a ratio threshold, which is what the histogram holds; the
-// one bin that s falls into is bracketed from its two sums and its edges, and when the bracket
-// is wider than 2.5e-7 that F(s_j) is recomputed exactly by a pass over the rows.
+// one bin that s falls into is bracketed from its two sums and its edges, and when half the
+// bracket plus the bound on the histogram's fixed-point error exceeds 2.5e-7 that F(s_j) is
+// recomputed exactly by a pass over the rows.
 //
 // Building with -DDSBD_PHASE_TIMING makes k_verify record %globaltimer stamps of its phases at
 // the end of the workspace (a tuning aid; off in normal builds).
@@ -38,8 +39,10 @@ using namespace dsbd;
 namespace {
 
 constexpr int kTile = 1024;          // tokens per tile: 32 lanes x 8 x float4
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;        // streaming kernels
 constexpr int kWarps = kThreads / 32;
+constexpr int kVThreads = 512;       // the per-request kernel: two CTAs of 16 warps per SM
+constexpr int kVWarps = kVThreads / 32;
 constexpr int kMaxLive = DSBD_MAX_LIVE;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr double kLn2 = 0.6931471805599453;
@@ -131,6 +134,20 @@ k_tile_stats(const float *__restrict__ zp, const float *__restrict__ zq, int64_t
     }
 }
 
+// log-sum-exp of a tempered row from its tile statistics, by one warp (same value on every lane;
+// the order of the sums depends on T only).
+__device__ __forceinline__ double row_lse(const TileStat *s, int T, double inv_tau, int lane) {
+    double mx = -INFINITY;
+    for (int t = lane; t < T; t += 32) mx = fmax(mx, (double)s[t].mx);
+    mx = warp_max(mx);
+    double acc = 0.0;
+    if (mx > -INFINITY)
+        for (int t = lane; t < T; t += 32)
+            if (s[t].sum > 0.f) acc += (double)s[t].sum * exp(((double)s[t].mx - mx) * inv_tau);
+    acc = warp_sum(acc);
+    return (mx > -INFINITY) ? mx * inv_tau + log(acc) : -INFINITY;
+}
+
 // log-sum-exp of the tempered row from its tile statistics; one warp per (model, row).
 __global__ void k_row_finish(const TileStat *__restrict__ stats, int T, int N, int n_rows,
                              const int32_t *__restrict__ rows, const int32_t *__restrict__ n_rows_dev,
@@ -144,17 +161,8 @@ __global__ void k_row_finish(const TileStat *__restrict__ stats, int T, int N, i
     const int ri = (int)(warp % n_rows);
     const int row = rows ? rows[ri] : ri;
     if (row < 0 || row >= N) return;
-    const TileStat *s = stats + ((int64_t)model * N + row) * T;
-    double mx = -INFINITY;
-    for (int t = lane; t < T; t += 32) mx = fmax(mx, (double)s[t].mx);
-    mx = warp_max(mx);
-    double acc = 0.0;
-    if (mx > -INFINITY)
-        for (int t = lane; t < T; t += 32)
-            if (s[t].sum > 0.f) acc += (double)s[t].sum * exp(((double)s[t].mx - mx) * inv_tau);
-    acc = warp_sum(acc);
+    const double v = row_lse(stats + ((int64_t)model * N + row) * T, T, inv_tau, lane);
     if (lane == 0) {
-        const double v = (mx > -INFINITY) ? mx * inv_tau + log(acc) : -INFINITY;
         lse[(int64_t)model * N + row] = v;
         if (model == 0 && lse_p_out) lse_p_out[row] = (float)v;
         if (model == 1 && lse_q_out) lse_q_out[row] = (float)v;
@@ -214,7 +222,10 @@ struct Shared {
     int S[kMaxLive];
     int S_parent_idx[kMaxLive];
     int acc[kMaxLive];
-    float bp[kMaxLive], bq[kMaxLive];       // log2 of the beam weight minus lse*log2(e)
+    // log2 of (beam weight / sum of the row's exponentials), split so that the cell masses do not
+    // inherit the rounding of one large float: bp/bq hold the nearest integer (exact in fp32), cp/cq
+    // the factor 2^(remainder) in [2^-0.5, 2^0.5], dc = log2(cp/cq)
+    float bp[kMaxLive], bq[kMaxLive], cp[kMaxLive], cq[kMaxLive], dc[kMaxLive];
     double lwp[kMaxLive], lwq[kMaxLive];    // natural log of the beam weights
     double wp[kMaxLive];
     double s_arr[kMaxLive + 2];             // s_0 .. s_m
@@ -226,23 +237,37 @@ struct Shared {
     int bank, need_exact, res_j, run_j, chain_pos;
     int n_out, n_fill;                      // output beams so far; p_beam fills left to the whole CTA
     int n_layers, n_tests, n_exact, n_respass;
-    uint32_t wtot_p[kWarps], wtot_q[kWarps];
+    int n_near, n_rows;                     // accept tests inside the 1e-5 tie band; live rows consulted
+    unsigned long long wtot_p[kVWarps], wtot_q[kVWarps];
+    double n_cells;                         // cells that entered the layer's histogram
+    unsigned long long w_tot[4];            // what this CTA added to its w words (p, q), and their sums
+    int wrapped, n_wrapped;                 // a w word of the layer's histogram wrapped; layers where that happened
     double rho[kMaxLive], uu[kMaxLive];     // per live draft: p_beam/q_beam and its uniform
 };
 
 // mass of one cell of the residual max(p_beam - s q_beam, 0); s == 0 gives p_beam
-__device__ __forceinline__ float cell_mass(float zp, float zq, float k2, float bp, float bq, float s) {
-    const float a = exp2f(fmaf(zp, k2, bp));
-    const float b = exp2f(fmaf(zq, k2, bq));
+struct RowOff { float bp, bq, cp, cq, dc; };
+__device__ __forceinline__ float cell_mass(float zp, float zq, float k2, const RowOff &o, float s) {
+    const float a = exp2f(fmaf(zp, k2, o.bp)) * o.cp;
+    const float b = exp2f(fmaf(zq, k2, o.bq)) * o.cq;
     return fmaxf(fmaf(-s, b, a), 0.f);
+}
+// Splits b = log2(weight) - lse*log2(e) (double) into its nearest integer and the factor 2^(rest).
+__device__ __forceinline__ void split_offset(double b, float *bi, float *c, double *rest) {
+    if (b == b && fabs(b) < 1e30) {
+        const double r = rint(b);
+        *bi = (float)r; *c = (float)exp2(b - r); *rest = b - r;
+    } else {
+        *bi = (float)b; *c = 1.f; *rest = 0.0;
+    }
 }
 
 // One cluster-wide pass: tile sums of max(p_beam - s q_beam, 0) over the live rows.
 __device__ void residual_pass(const VerifyArgs &a, const Shared &sh, float s, double *sums,
                               int cta_rank, int n_cta) {
     const int lane = threadIdx.x & 31;
-    const int warp = cta_rank * kWarps + (threadIdx.x >> 5);
-    const int nwarps = n_cta * kWarps;
+    const int warp = cta_rank * kVWarps + (threadIdx.x >> 5);
+    const int nwarps = n_cta * kVWarps;
     const int items = sh.nA * a.T;
     for (int item = warp; item < items; item += nwarps) {
         const int i = item / a.T, t = item - i * a.T;
@@ -250,7 +275,7 @@ __device__ void residual_pass(const VerifyArgs &a, const Shared &sh, float s, do
         const float *rp = a.zp + (int64_t)row * a.stride;
         const float *rq = a.zq + (int64_t)row * a.stride;
         const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
-        const float bp = sh.bp[i], bq = sh.bq[i];
+        const RowOff ro = {sh.bp[i], sh.bq[i], sh.cp[i], sh.cq[i], sh.dc[i]};
         float acc = 0.f;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -259,10 +284,10 @@ __device__ void residual_pass(const VerifyArgs &a, const Shared &sh, float s, do
             load_half_tile(rq, t * kTile + half * (kTile / 2), a.V, al, lane, vq);
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
-                acc += cell_mass(vp[it].x, vq[it].x, a.k2, bp, bq, s);
-                acc += cell_mass(vp[it].y, vq[it].y, a.k2, bp, bq, s);
-                acc += cell_mass(vp[it].z, vq[it].z, a.k2, bp, bq, s);
-                acc += cell_mass(vp[it].w, vq[it].w, a.k2, bp, bq, s);
+                acc += cell_mass(vp[it].x, vq[it].x, a.k2, ro, s);
+                acc += cell_mass(vp[it].y, vq[it].y, a.k2, ro, s);
+                acc += cell_mass(vp[it].z, vq[it].z, a.k2, ro, s);
+                acc += cell_mass(vp[it].w, vq[it].w, a.k2, ro, s);
             }
         }
         const double tot = warp_sum((double)acc);
@@ -311,7 +336,7 @@ __device__ int locate_tile(F mass, int n, double target, int lane, double *befor
 
 // Inverse-CDF search inside one tile of row `row` (and its q row when s > 0): the first
 // token whose running mass reaches `target`, else the last token with mass.  -1: no mass.
-__device__ int locate_token(const VerifyArgs &a, int row, int t, float bp, float bq, float s,
+__device__ int locate_token(const VerifyArgs &a, int row, int t, const RowOff &ro, float s,
                             double target, int lane) {
     const float *rp = a.zp + (int64_t)row * a.stride;
     const float *rq = a.zq + (int64_t)row * a.stride;
@@ -326,8 +351,8 @@ __device__ int locate_token(const VerifyArgs &a, int row, int t, float bp, float
             float mv = 0.f;
             if (e + c < a.V) {
                 const float zpv = __ldg(rp + e + c);
-                mv = (s > 0.f) ? cell_mass(zpv, __ldg(rq + e + c), a.k2, bp, bq, s)
-                               : exp2f(fmaf(zpv, a.k2, bp));
+                mv = (s > 0.f) ? cell_mass(zpv, __ldg(rq + e + c), a.k2, ro, s)
+                               : exp2f(fmaf(zpv, a.k2, ro.bp)) * ro.cp;
             }
             mss[c] = mv;
             loc += (double)mv;
@@ -397,22 +422,30 @@ __device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, 
 
 // Beam weights of the live set: softmax of the cumulative scores over A (Eq. 1 factorised).
 // Called by all lanes of one warp; beam i is handled by lane i % 32.
+// Natural log of the softmax of n scores, by one warp (lanes over the scores).
+__device__ __forceinline__ void log_softmax_warp(const double *s, int n, int lane, double *out) {
+    double mx = -INFINITY;
+    for (int i = lane; i < n; i += 32) mx = fmax(mx, s[i]);
+    mx = warp_max(mx);
+    double t = 0.0;
+    for (int i = lane; i < n; i += 32) t += exp(s[i] - mx);
+    t = warp_sum(t);
+    const double lt = log(t);
+    for (int i = lane; i < n; i += 32) out[i] = (s[i] - mx) - lt;
+    __syncwarp();
+}
+
 __device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, const double *sq, int lane) {
-    double mp = -INFINITY, mq = -INFINITY;
-    for (int i = lane; i < sh.nA; i += 32) { mp = fmax(mp, sp[i]); mq = fmax(mq, sq[i]); }
-    mp = warp_max(mp); mq = warp_max(mq);
-    double tp = 0.0, tq = 0.0;
-    for (int i = lane; i < sh.nA; i += 32) { tp += exp(sp[i] - mp); tq += exp(sq[i] - mq); }
-    tp = warp_sum(tp); tq = warp_sum(tq);
-    const double ltp = log(tp), ltq = log(tq);
+    log_softmax_warp(sp, sh.nA, lane, sh.lwp);
+    log_softmax_warp(sq, sh.nA, lane, sh.lwq);
     for (int i = lane; i < sh.nA; i += 32) {
-        const double lwp = (sp[i] - mp) - ltp, lwq = (sq[i] - mq) - ltq;
+        const double lwp = sh.lwp[i], lwq = sh.lwq[i];
         sh.wp[i] = exp(lwp);
-        sh.lwp[i] = lwp;
-        sh.lwq[i] = lwq;
         const int row = sh.A[i];
-        sh.bp[i] = (float)((lwp - a.lse[row]) / kLn2);
-        sh.bq[i] = (float)((lwq - a.lse[a.N + row]) / kLn2);
+        double rest_p, rest_q;
+        split_offset((lwp - a.lse[row]) / kLn2, &sh.bp[i], &sh.cp[i], &rest_p);
+        split_offset((lwq - a.lse[a.N + row]) / kLn2, &sh.bq[i], &sh.cq[i], &rest_q);
+        sh.dc[i] = (float)(rest_p - rest_q);
     }
     __syncwarp();
 }
@@ -461,31 +494,125 @@ __device__ int width_rule(Shared &sh, int m, double thresh, int lane, int k_stop
 }
 
 // ---------------------------------------------------------------------------------------
-// Ratio histogram of one layer.  Every cell with rho = p_beam/q_beam > 1 adds its p and q mass
-// (fixed point, 2^-31) to the bin of log2(rho); bin kBins collects rho beyond the last edge.
-// F(s) for any s in [1, top] is then (sum of the bins above s) plus the straddled bin, whose
-// contribution is bracketed from its two sums and its edges.  Integer sums make the result
-// independent of the order in which warps and CTAs add.
+// Ratio histogram of one layer.  Every cell with rho = p_beam/q_beam > 1 adds its p and q mass to
+// the bin of log2(rho); bin kBins collects rho beyond the last edge.  F(s) for any s in [1, top]
+// is then (sum of the bins above s) plus the straddled bin, whose contribution is bracketed from
+// its two sums and its edges.
+//
+// Masses are summed as integers in units of 2^-44, so the sums do not depend on the order in which
+// warps and CTAs add, and a cell of mass >= 2^-20 enters without any rounding (its 24-bit
+// mantissa is a whole number of units); a smaller cell is rounded by at most 2^-45.  With n cells
+// the fixed-point error of any partial sum is therefore at most n 2^-45 (2.8e-8 for a million
+// cells), which the chain adds to its bracket.
+// In shared memory a bin has two 32-bit words per model, fed by plain (non-returning) atomic adds:
+//   w: units of 2^-44.  A cell below 2^-16 adds all of itself here (less than 2^28 units); a larger
+//      cell only its remainder below 2^-28 (less than 2^16 units).
+//   b: units of 2^-28, the whole multiples of 2^-28 of the cells of at least 2^-16; it cannot
+//      overflow because a joint distribution sums to one.
+// A w word wraps once the small cells of ONE bin that ONE CTA added reach 2^-12 of the mass --
+// twenty times what a bin holds in ordinary data, but possible when the two models' rows are
+// proportional and every cell lands in the same bin.  A wrap is detected exactly: every thread
+// keeps the 64-bit total of what it added to the w words, and the CTA compares the sum of those
+// totals with the sum of its w words; a difference marks the layer, whose residual masses are
+// then all computed by exact passes over the rows.
 // ---------------------------------------------------------------------------------------
 constexpr int kBins = 4096;
-constexpr float kFix = 2147483648.f;          // 2^31
-constexpr double kUnfix = 1.0 / 2147483648.0;
-constexpr double kGapTol = 2.5e-7;            // bracket width above which F(s) is recomputed exactly
+constexpr int kOverSlots = 256;                   // copies of the last bin (rho beyond the last edge): one per
+                                                  // warp and half-warp lane, so that none collects enough to wrap
+constexpr int kHistWords = kBins + kOverSlots + 16;  // bins 0..kBins-1, the copies of bin kBins, spare words
+static_assert(kHistWords % 4 == 0, "the arrays that share this memory need 16-byte alignment");
+constexpr float kFix = 17592186044416.f;          // 2^44
+constexpr double kUnfix = 1.0 / 17592186044416.0;
+constexpr float kBigCell = 1.f / 65536.f;         // 2^-16: cells from here on put their top part into the b word
+constexpr float kBigFix = 268435456.f;            // 2^28, the unit of the b word is 2^-28
+constexpr double kErrTol = 2.5e-7;                // error bound of F(s) above which it is recomputed exactly
+// global image of one histogram: P and Q of bin i at 2i, 2i+1 (units of 2^-44), then the cell count
+// and the number of CTAs whose w words wrapped
+constexpr int kHistLen = 2 * (kBins + 1) + 2;
+constexpr int kHistCount = 2 * (kBins + 1);
+constexpr int kHistWrapped = kHistCount + 1;
 
-__device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, uint32_t *hp,
-                               uint32_t *hq, double *sums1, int cta_rank, int n_cta) {
+constexpr int kHistArrays = 4;
+struct HistSmem { uint32_t *wp, *wq, *bp, *bq; };
+
+__device__ __forceinline__ HistSmem hist_arrays(uint32_t *base) {
+    return HistSmem{base, base + kHistWords, base + 2 * kHistWords, base + 3 * kHistWords};
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// A cell's mass as a count of 2^-44 units for the w word; a cell of at least 2^-16 (rare) first
+// moves its whole multiples of 2^-28 to the b word.  Exact for a mass of at least 2^-20.
+__device__ __forceinline__ uint32_t split_mass(float m, uint32_t *b_word) {
+    if (m >= kBigCell) {
+        const float hf = floorf(m * kBigFix);
+        m = fmaf(-hf, 1.f / kBigFix, m);                        // exact remainder, below 2^-28
+        atomicAdd(b_word, (uint32_t)hf);
+    }
+    return __float2uint_rn(m * kFix);
+}
+// Per-thread sums of one histogram pass.
+struct PassSums {
+    unsigned long long tot_p, tot_q;      // what went into the w words
+    int n;                                // cells with rho > 1
+};
+
+// The cells of one half tile (4 x float4 per lane and model) into the histogram; adds their
+// (p - q)+ to res1.
+// (ex2.approx flushes results below 2^-126 to zero; a cell enters the sums from 2^-45 on.)
+__device__ __forceinline__ void hist_half_tile(const float4 (&vp)[4], const float4 (&vq)[4], float k2,
+                                               const RowOff &o, float binscale, const HistSmem &h, float &res1,
+                                               PassSums &ps, int over_bin) {
+    const float bd = (o.bp - o.bq) + o.dc;                      // log2(rho) = (zp - zq) k2 + bd
+    uint32_t tp = 0u, tq = 0u;                                  // below 2^32: 16 cells of less than 2^28 units
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const float zp4[4] = {vp[it].x, vp[it].y, vp[it].z, vp[it].w};
+        const float zq4[4] = {vq[it].x, vq[it].y, vq[it].z, vq[it].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float dl = fmaf(zp4[c] - zq4[c], k2, bd);     // NaN compares false
+            if (dl > 0.f) {
+                const float pm = ex2_approx(fmaf(zp4[c], k2, o.bp)) * o.cp;
+                const float qm = ex2_approx(fmaf(zq4[c], k2, o.bq)) * o.cq;
+                res1 += fmaxf(pm - qm, 0.f);
+                const float bf = dl * binscale;
+                ++ps.n;
+                // (all cells beyond the last edge in one word would wrap it: every warp has its own)
+                const int bin = bf < (float)kBins ? __float2int_rz(bf) : over_bin;
+                const uint32_t ap = split_mass(pm, h.bp + bin), aq = split_mass(qm, h.bq + bin);
+                tp += ap; tq += aq;
+                atomicAdd(h.wp + bin, ap);
+                atomicAdd(h.wq + bin, aq);
+            }
+        }
+    }
+    ps.tot_p += tp; ps.tot_q += tq;
+}
+
+// One cluster-wide pass over the live rows; every CTA fills its own shared-memory histogram.
+// tot[0], tot[1] (shared memory, zero before the call): what the CTA added to its w words.
+// gh: the global image of the histogram (cell count and the last bin are added to it directly).
+__device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, const HistSmem &h,
+                               double *sums1, int cta_rank, int n_cta, unsigned long long *gh,
+                               unsigned long long *tot) {
     const int lane = threadIdx.x & 31;
-    const int warp = cta_rank * kWarps + (threadIdx.x >> 5);
-    const int nwarps = n_cta * kWarps;
+    const int warp = cta_rank * kVWarps + (threadIdx.x >> 5);
+    const int nwarps = n_cta * kVWarps;
     const int items = sh.nA * a.T;
-    uint32_t over_p = 0u, over_q = 0u;                   // cells beyond the last edge: always above s
+    PassSums ps = {0ull, 0ull, 0};
+    const int over_bin = kBins + ((threadIdx.x >> 5) & 15) * 16 + (threadIdx.x & 15);
     for (int item = warp; item < items; item += nwarps) {
         const int i = item / a.T, t = item - i * a.T;
         const int row = sh.A[i];
         const float *rp = a.zp + (int64_t)row * a.stride;
         const float *rq = a.zq + (int64_t)row * a.stride;
         const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
-        const float bp = sh.bp[i], bq = sh.bq[i];
+        const RowOff ro = {sh.bp[i], sh.bq[i], sh.cp[i], sh.cq[i], sh.dc[i]};
         float res1 = 0.f;                                // sum of (p - q)+ over the tile: residual mass at s = 1
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -493,43 +620,51 @@ __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float bins
             const int e0 = t * kTile + half * (kTile / 2);
             load_half_tile(rp, e0, a.V, al, lane, vp);
             load_half_tile(rq, e0, a.V, al, lane, vq);
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const float zp4[4] = {vp[it].x, vp[it].y, vp[it].z, vp[it].w};
-                const float zq4[4] = {vq[it].x, vq[it].y, vq[it].z, vq[it].w};
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const float xp = fmaf(zp4[c], a.k2, bp), xq = fmaf(zq4[c], a.k2, bq);
-                    const float dl = xp - xq;                       // log2(rho); NaN compares false
-                    if (dl > 0.f) {
-                        const float pm = exp2f(xp), qm = exp2f(xq);
-                        res1 += fmaxf(pm - qm, 0.f);
-                        const uint32_t fp = __float2uint_rn(pm * kFix);
-                        const uint32_t fq = __float2uint_rn(qm * kFix);
-                        const float bf = dl * binscale;
-                        if (bf < (float)kBins) {
-                            const int bin = (int)bf;
-                            atomicAdd(hp + bin, fp);
-                            atomicAdd(hq + bin, fq);
-                        } else {
-                            over_p += fp;
-                            over_q += fq;
-                        }
-                    }
-                }
-            }
+            hist_half_tile(vp, vq, a.k2, ro, binscale, h, res1, ps, over_bin);
         }
         // tile sums of the residual after ONE rejection (s_1 = 1): what a completion draw at run
         // position 2 searches, so that this common case needs no second pass over the rows
-        const double tot = warp_sum((double)res1);
-        if (lane == 0) sums1[item] = tot;
+        const double tot1 = warp_sum((double)res1);
+        if (lane == 0) sums1[item] = tot1;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        over_p += __shfl_xor_sync(kFull, over_p, o);
-        over_q += __shfl_xor_sync(kFull, over_q, o);
+        ps.n += __shfl_xor_sync(kFull, ps.n, o);
+        ps.tot_p += __shfl_xor_sync(kFull, ps.tot_p, o);
+        ps.tot_q += __shfl_xor_sync(kFull, ps.tot_q, o);
     }
-    if (lane == 0 && (over_p | over_q)) { atomicAdd(hp + kBins, over_p); atomicAdd(hq + kBins, over_q); }
+    if (lane == 0) {
+        if (ps.n) atomicAdd(gh + kHistCount, (unsigned long long)ps.n);
+        if (ps.tot_p) atomicAdd(tot, ps.tot_p);
+        if (ps.tot_q) atomicAdd(tot + 1, ps.tot_q);
+    }
+}
+
+// Adds a CTA's shared-memory histogram to its global image (64-bit sums in units of 2^-44) and
+// checks its w words against what the CTA's threads added to them (tot[0..1]; tot[2..3] must be
+// zero before the call and are used as scratch): a difference means that a word wrapped.
+__device__ void hist_flush(const HistSmem &h, unsigned long long *gh, unsigned long long *tot) {
+    unsigned long long sp = 0ull, sq = 0ull;
+    for (int i = threadIdx.x; i < kBins + kOverSlots; i += blockDim.x) {
+        const uint32_t wp = h.wp[i], wq = h.wq[i];
+        sp += wp; sq += wq;
+        const unsigned long long P = ((unsigned long long)h.bp[i] << 16) + wp;
+        const unsigned long long Q = ((unsigned long long)h.bq[i] << 16) + wq;
+        const int g = i < kBins ? i : kBins;             // the warps' copies of the last bin are one bin again
+        if (P) atomicAdd(gh + 2 * g, P);
+        if (Q) atomicAdd(gh + 2 * g + 1, Q);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sp += __shfl_xor_sync(kFull, sp, o);
+        sq += __shfl_xor_sync(kFull, sq, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (sp) atomicAdd(tot + 2, sp);
+        if (sq) atomicAdd(tot + 3, sq);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && (tot[0] != tot[2] || tot[1] != tot[3])) atomicAdd(gh + kHistWrapped, 1ull);
 }
 
 // One completion draw (residual if s_res > 0 else p_beam) by warp 0; returns the token or -1
@@ -564,8 +699,8 @@ __device__ int draw_cell(const VerifyArgs &a, const Shared &sh, double u, bool u
     if (tile < 0) return -1;
     const int ia = tile / a.T;
     *ia_out = ia;
-    return locate_token(a, sh.A[ia], tile - ia * a.T, sh.bp[ia], sh.bq[ia], use_res ? s_res : 0.f,
-                        target - before, lane);
+    const RowOff ro = {sh.bp[ia], sh.bq[ia], sh.cp[ia], sh.cq[ia], sh.dc[ia]};
+    return locate_token(a, sh.A[ia], tile - ia * a.T, ro, use_res ? s_res : 0.f, target - before, lane);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -578,7 +713,7 @@ __device__ int draw_cell(const VerifyArgs &a, const Shared &sh, double u, bool u
 // ---------------------------------------------------------------------------------------
 constexpr int kMaxTopK = 64;
 constexpr int kMaxCand = 680;      // candidate cells per model (two lists overlay one histogram array)
-constexpr int kHalf = 128;         // threads that build one model's support (the two models run side by side)
+constexpr int kHalf = 256;         // threads that build one model's support (the two models run side by side)
 // scratch of one build_support instance
 struct SupportTmp {
     float off[kMaxLive];          // log(beam weight) - lse of each live row
@@ -917,7 +1052,12 @@ __device__ void finish_supports(WarpScratch &ws, bool have_q, int lane) {
 #define TS(slot) do {} while (0)
 #endif
 
-__global__ void __launch_bounds__(kThreads, 4)
+// dynamic shared memory of k_verify: the histogram of a layer as four 32-bit arrays while it is
+// being built, then (over the same bytes) the 64-bit suffix sums of its p and q mass
+constexpr size_t kVerifyDynSmem = kHistArrays * sizeof(uint32_t) * kHistWords;
+static_assert(2 * sizeof(unsigned long long) * kHistWords <= kVerifyDynSmem, "the suffix sums fit over the building arrays");
+
+__global__ void __launch_bounds__(kVThreads, 2)
 k_verify(VerifyArgs a) {
     cg::cluster_group cluster = cg::this_cluster();
     const int n_cta = (int)cluster.num_blocks();
@@ -929,7 +1069,10 @@ k_verify(VerifyArgs a) {
     __shared__ Shared sh;
     __shared__ double sp_live[kMaxLive], sq_live[kMaxLive];
     __shared__ int8_t st[kMaxLive * kMaxLive];     // status of the request's nodes, local index
-    __shared__ __align__(16) uint32_t hp[kBins + 2], hq[kBins + 2];   // p and q mass per ratio bin, fixed point
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    uint32_t *hp = reinterpret_cast<uint32_t *>(dyn_smem), *hq = hp + kHistWords;     // first two digit arrays
+    const HistSmem hs = hist_arrays(hp);
+    unsigned long long *sufP = reinterpret_cast<unsigned long long *>(dyn_smem), *sufQ = sufP + kHistWords;
 
     // launched with programmatic stream serialization: everything before this line overlaps the
     // tail of the kernel ahead in the stream, nothing after it may run before that kernel is done
@@ -945,8 +1088,8 @@ k_verify(VerifyArgs a) {
     if (bad_widths) { W_min = W_max = W_nom = 1; }
     double *sums_base = a.tile_sums + (int64_t)r * 2 * a.max_m * ((int64_t)a.max_live * a.T);
     const int64_t slot_stride = (int64_t)a.max_live * a.T;
-    unsigned long long *ghist = a.hist + (int64_t)r * 2 * (kBins + 1);     // [2 banks][kBins+1]
-    const int hist_len = kBins + 1;
+    unsigned long long *ghist = a.hist + (int64_t)r * 2 * kHistLen;        // [2 banks][kHistLen]
+    const int hist_len = kHistLen;
     int n_out = 0;
 #ifdef DSBD_PHASE_TIMING
     int ts_n = 0;
@@ -956,20 +1099,11 @@ k_verify(VerifyArgs a) {
     if (!a.select_mode) {
         // ---- log-sum-exp of every row of the request from the dense pass's tile statistics ----
         const int n_req = n_hi - n_lo;
-        const int cw = cta_rank * kWarps + warp, ncw = n_cta * kWarps;
+        const int cw = cta_rank * kVWarps + warp, ncw = n_cta * kVWarps;
         for (int task = cw; task < 2 * n_req; task += ncw) {
             const int model = task / n_req, row = n_lo + (task - model * n_req);
-            const TileStat *ts = a.stats + ((int64_t)model * a.N + row) * a.T;
-            double mx = -INFINITY;
-            for (int t = lane; t < a.T; t += 32) mx = fmax(mx, (double)ts[t].mx);
-            mx = warp_max(mx);
-            double acc = 0.0;
-            if (mx > -INFINITY)
-                for (int t = lane; t < a.T; t += 32)
-                    if (ts[t].sum > 0.f) acc += (double)ts[t].sum * exp(((double)ts[t].mx - mx) * a.inv_tau);
-            acc = warp_sum(acc);
+            const double v = row_lse(a.stats + ((int64_t)model * a.N + row) * a.T, a.T, a.inv_tau, lane);
             if (lane == 0) {
-                const double v = (mx > -INFINITY) ? mx * a.inv_tau + log(acc) : -INFINITY;
                 a.lse_w[(int64_t)model * a.N + row] = v;
                 float *o = model ? a.out.lse_q : a.out.lse_p;
                 if (o) o[row] = (float)v;
@@ -978,7 +1112,7 @@ k_verify(VerifyArgs a) {
         __threadfence();
         cluster.sync();
         // ---- log-prob of every draft token given its parent (all nodes at once) ----
-        for (int i = cta_rank * kThreads + threadIdx.x; i < n_req; i += n_cta * kThreads) {
+        for (int i = cta_rank * kVThreads + threadIdx.x; i < n_req; i += n_cta * kVThreads) {
             const int n = n_lo + i, par = a.parent[n];
             double lp = 0.0, lq = 0.0;
             if (par >= 0) {
@@ -1005,19 +1139,19 @@ k_verify(VerifyArgs a) {
                 // stage the per-node log-probs in shared memory (the histogram arrays are idle
                 // here), then every node sums its own path to the root
                 double *slp = reinterpret_cast<double *>(hp), *slq = reinterpret_cast<double *>(hq);
-                for (int i = threadIdx.x; i < n_req; i += kThreads) {
+                for (int i = threadIdx.x; i < n_req; i += kVThreads) {
                     slp[i] = a.score_w[n_lo + i];
                     slq[i] = a.score_w[a.N + n_lo + i];
                 }
                 __syncthreads();
-                for (int b = b_lo + (int)threadIdx.x; b < b_hi; b += kThreads) {
+                for (int b = b_lo + (int)threadIdx.x; b < b_hi; b += kVThreads) {
                     const int root = a.beam_node_off[b];
                     if (a.parent[root] != -1) report(a.status, DSBD_DEV_BAD_FOREST);
                     slp[root - n_lo] = (double)a.root_logp[b];
                     slq[root - n_lo] = (double)a.root_logq[b];
                 }
                 __syncthreads();
-                for (int i = threadIdx.x; i < n_req; i += kThreads) {
+                for (int i = threadIdx.x; i < n_req; i += kVThreads) {
                     double sp = 0.0, sq = 0.0;
                     int dep = 0, cur = i;
                     while (true) {
@@ -1036,7 +1170,7 @@ k_verify(VerifyArgs a) {
                 }
                 __syncthreads();
             } else {
-                for (int b = b_lo + (int)threadIdx.x; b < b_hi; b += kThreads) {
+                for (int b = b_lo + (int)threadIdx.x; b < b_hi; b += kVThreads) {
                     const int lo = a.beam_node_off[b], hi = a.beam_node_off[b + 1];
                     for (int n = lo; n < hi; ++n) {
                         const int par = a.parent[n];
@@ -1069,11 +1203,12 @@ k_verify(VerifyArgs a) {
     }
 
     // ---- set-up ----
-    for (int i = cta_rank * kThreads + threadIdx.x; i < 2 * hist_len; i += n_cta * kThreads) ghist[i] = 0ull;
+    for (int i = cta_rank * kVThreads + threadIdx.x; i < 2 * hist_len; i += n_cta * kVThreads) ghist[i] = 0ull;
     if (warp == 0) {
         if (lane == 0) {
             sh.err = 0; sh.done = 0; sh.n_out = 0; sh.n_fill = 0;
             sh.n_layers = sh.n_tests = sh.n_exact = sh.n_respass = 0;
+            sh.n_wrapped = 0; sh.n_near = 0; sh.n_rows = 0;
             if (a.select_mode) {
                 const int lo = a.live_off[r], hi = a.live_off[r + 1];
                 sh.nA = hi - lo;
@@ -1189,7 +1324,9 @@ k_verify(VerifyArgs a) {
                     sh.uu[i] = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l, 0u, (uint32_t)i);
                 }
         }
-        for (int i = threadIdx.x; i < kBins + 2; i += blockDim.x) { hp[i] = 0u; hq[i] = 0u; }
+        for (int i = threadIdx.x; i < kHistArrays * kHistWords; i += blockDim.x) hp[i] = 0u;
+        if (threadIdx.x < 4) sh.w_tot[threadIdx.x] = 0ull;
+        if (threadIdx.x == 0) sh.wrapped = 0;
         __syncthreads();
         const int m = sh.m;
         TS(3);
@@ -1199,8 +1336,8 @@ k_verify(VerifyArgs a) {
         if (warped) {
             // ---- supports of T o p_beam and T o q_beam, then the whole chain on <= 64 cells ----
             if (!sh.err) {
-                // warps 0-3 build the support of p, warps 4-7 that of q, side by side
-                const int half = warp >> 2;
+                // the first half of the warps builds the support of p, the second that of q, side by side
+                const int half = warp / (kHalf / 32);
                 const int e_half = build_support(a, sh, half, hp, hq);
                 if (e_half && (threadIdx.x & (kHalf - 1)) == 0) wsup.tmp[half].err = e_half;
                 __syncthreads();
@@ -1241,45 +1378,50 @@ k_verify(VerifyArgs a) {
             const double top = log2((double)(m > 2 ? m : 2));          // s_j <= j <= m
             const float binscale = (float)((double)kBins / top);
             unsigned long long *gh = ghist + sh.bank * hist_len;
-            histogram_pass(a, sh, binscale, hp, hq, sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride, cta_rank,
-                           n_cta);
+            histogram_pass(a, sh, binscale, hs, sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride, cta_rank,
+                           n_cta, gh, sh.w_tot);
             __syncthreads();
             TS(4);
-            for (int i = threadIdx.x; i <= kBins; i += blockDim.x)
-                if (hp[i] | hq[i]) atomicAdd(gh + i, ((unsigned long long)hp[i] << 32) | hq[i]);
+            hist_flush(hs, gh, sh.w_tot);
             __threadfence();
             cluster.sync();
             TS(5);
+            // the merged histogram into shared memory (over the building arrays, which are flushed)
+            __syncthreads();
             for (int i = threadIdx.x; i <= kBins; i += blockDim.x) {
-                const unsigned long long v = __ldcg(gh + i);
-                hp[i] = (uint32_t)(v >> 32);
-                hq[i] = (uint32_t)v;
+                sufP[i] = __ldcg(gh + 2 * i);
+                sufQ[i] = __ldcg(gh + 2 * i + 1);
+            }
+            if (threadIdx.x == 0) {
+                sh.n_cells = (double)__ldcg(gh + kHistCount);
+                sh.wrapped = __ldcg(gh + kHistWrapped) != 0ull;
+                if (sh.wrapped) ++sh.n_wrapped;
             }
             __syncthreads();
             cluster.sync();                            // everyone has read the bank: it can be cleared
-            for (int i = cta_rank * kThreads + threadIdx.x; i < hist_len; i += n_cta * kThreads) gh[i] = 0ull;
+            for (int i = cta_rank * kVThreads + threadIdx.x; i < hist_len; i += n_cta * kVThreads) gh[i] = 0ull;
             TS(6);
-            // in-place suffix sums: hp[k] = p mass of the bins >= k (17 bins per thread)
+            // in-place suffix sums: sufP[k] = p mass of the bins >= k (17 bins per thread)
             {
-                constexpr int per = (kBins + 1 + kThreads - 1) / kThreads;
+                constexpr int per = (kBins + 1 + kVThreads - 1) / kVThreads;
                 const int lo = min((int)threadIdx.x * per, kBins + 1), hi = min(lo + per, kBins + 1);
-                uint32_t mp_ = 0u, mq_ = 0u;
-                for (int i = lo; i < hi; ++i) { mp_ += hp[i]; mq_ += hq[i]; }
-                uint32_t ap = mp_, aq = mq_;              // suffix scan inside the warp, top lane down
+                unsigned long long mp_ = 0ull, mq_ = 0ull;
+                for (int i = lo; i < hi; ++i) { mp_ += sufP[i]; mq_ += sufQ[i]; }
+                unsigned long long ap = mp_, aq = mq_;    // suffix scan inside the warp, top lane down
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t tp = __shfl_down_sync(kFull, ap, o), tq = __shfl_down_sync(kFull, aq, o);
+                    const unsigned long long tp = __shfl_down_sync(kFull, ap, o), tq = __shfl_down_sync(kFull, aq, o);
                     if (lane + o < 32) { ap += tp; aq += tq; }
                 }
                 if (lane == 0) { sh.wtot_p[warp] = ap; sh.wtot_q[warp] = aq; }
                 __syncthreads();
-                uint32_t rp_ = ap - mp_, rq_ = aq - mq_;  // mass of the lanes above in this warp
-                for (int w = warp + 1; w < kWarps; ++w) { rp_ += sh.wtot_p[w]; rq_ += sh.wtot_q[w]; }
+                unsigned long long rp_ = ap - mp_, rq_ = aq - mq_;  // mass of the lanes above in this warp
+                for (int w = warp + 1; w < kVWarps; ++w) { rp_ += sh.wtot_p[w]; rq_ += sh.wtot_q[w]; }
                 for (int i = hi - 1; i >= lo; --i) {
-                    rp_ += hp[i]; rq_ += hq[i];
-                    hp[i] = rp_; hq[i] = rq_;
+                    rp_ += sufP[i]; rq_ += sufQ[i];
+                    sufP[i] = rp_; sufQ[i] = rq_;
                 }
-                if (threadIdx.x == 0) { hp[kBins + 1] = 0u; hq[kBins + 1] = 0u; }
+                if (threadIdx.x == 0) { sufP[kBins + 1] = 0ull; sufQ[kBins + 1] = 0ull; }
             }
             __syncthreads();
 
@@ -1294,22 +1436,27 @@ k_verify(VerifyArgs a) {
                         sh.s_arr[j] = s_j;
                         sh.chain_len = j;
                         double c_next;
+                        // every partial sum of the histogram is off by at most half a unit per cell
+                        const double fix_err = sh.n_cells * (0.5 * kUnfix) * (1.0 + s_j);
+                        if (sh.wrapped) { need = 1; break; }             // a wrapped word: exact passes only
                         if (j == 1) {
-                            c_next = ((double)hp[0] - (double)hq[0]) * kUnfix;
+                            c_next = ((double)sufP[0] - (double)sufQ[0]) * kUnfix;
+                            if (fix_err > kErrTol) { need = 1; break; }
                         } else {
                             int k = (int)(log2(s_j) * (double)binscale);
                             if (k < 0) k = 0;
                             if (k >= kBins) { need = 1; break; }      // cannot happen for s_j <= m
-                            const double Pa = (double)hp[k + 1] * kUnfix, Qa = (double)hq[k + 1] * kUnfix;
-                            const double Pk = (double)(hp[k] - hp[k + 1]) * kUnfix;
-                            const double Qk = (double)(hq[k] - hq[k + 1]) * kUnfix;
+                            const double Pa = (double)sufP[k + 1] * kUnfix, Qa = (double)sufQ[k + 1] * kUnfix;
+                            const double Pk = (double)(sufP[k] - sufP[k + 1]) * kUnfix;
+                            const double Qk = (double)(sufQ[k] - sufQ[k + 1]) * kUnfix;
                             const double r_lo = (double)exp2f((float)k / binscale) * (1.0 - 2e-6);
                             const double r_hi = (double)exp2f((float)(k + 1) / binscale) * (1.0 + 2e-6);
                             const double lo_b = fmax(Pk - s_j * Qk, 0.0);
                             double q_hi = (Pk - r_lo * Qk) / (r_hi - r_lo);
                             q_hi = fmin(fmax(q_hi, 0.0), Qk);
                             const double hi_b = fmax(q_hi * (r_hi - s_j), lo_b);
-                            if (hi_b - lo_b > kGapTol) { need = 1; break; }
+                            // the midpoint of the bracket is used: half its width plus the fixed-point term
+                            if (0.5 * (hi_b - lo_b) + fix_err > kErrTol) { need = 1; break; }
                             c_next = fmax(Pa - s_j * Qa, 0.0) + 0.5 * (lo_b + hi_b);
                         }
                         sh.c_arr[j + 1] = c_next;
@@ -1367,7 +1514,7 @@ k_verify(VerifyArgs a) {
                 if (lane == 0) sh.done = 1;
             } else if (lane == 0) {
                 if (writer) a.out.layer_width[(int64_t)r * (a.gamma + 1) + (l - 1)] = W;
-                int count = 0, j = 1, err = 0, tests = 0;
+                int count = 0, j = 1, err = 0, tests = 0, near = 0;
                 for (int i = 0; i < m && count < W; ++i) {
                     const int n = sh.S[i];
                     const double rho = sh.rho[i];
@@ -1377,6 +1524,7 @@ k_verify(VerifyArgs a) {
                     if (ratio > 1.0) ratio = 1.0;
                     const double u = sh.uu[i];
                     ++tests;
+                    near += fabs(u - ratio) < 1e-5;
                     if (u <= ratio) {
                         st[n - n_lo] = DSBD_NODE_ACCEPTED;
                         if (writer) a.out.node_status[n] = DSBD_NODE_ACCEPTED;
@@ -1398,6 +1546,8 @@ k_verify(VerifyArgs a) {
                 sh.W = W;
                 sh.count = count;
                 sh.n_tests += tests;
+                sh.n_near += near;
+                sh.n_rows += sh.nA;
                 ++sh.n_layers;
                 sh.res_j = (count < W && j > 1) ? j : 0;   // residual draw at run position j needs tile sums
                 sh.run_j = j;
@@ -1490,7 +1640,7 @@ k_verify(VerifyArgs a) {
             const int base = sh.n_out, want = sh.n_fill;
             const int n_draw = min(want, max(cap - base, 0));
             __syncthreads();
-            for (int f = warp; f < n_draw; f += kWarps) {
+            for (int f = warp; f < n_draw; f += kVWarps) {
                 const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)l, 2u, (uint32_t)f);
                 int ia = 0;
                 const int tok = draw_cell(a, sh, u, false, 0.f, 0.0, nullptr, lane, &ia);
@@ -1530,7 +1680,7 @@ k_verify(VerifyArgs a) {
         const int cap = a.out.out_off[r + 1] - a.out.out_off[r];
         const int n_draw = min(W_nom, max(cap - n_out, 0));
         if (writer && threadIdx.x == 0) a.out.layer_width[(int64_t)r * (a.gamma + 1) + a.gamma] = W_nom;
-        for (int kk = warp; kk < n_draw; kk += kWarps) {
+        for (int kk = warp; kk < n_draw; kk += kVWarps) {
             const double u = decision_uniform(a.seed, a.step, (uint32_t)r, (uint32_t)(a.gamma + 1) + a.extra_layer_bias, 3u,
                                               (uint32_t)kk);
             int ia = 0;
@@ -1573,10 +1723,9 @@ k_verify(VerifyArgs a) {
             a.out.out_width[r] = n_out;
             if (a.out.req_error) a.out.req_error[r] = sh.err;
             if (a.out.req_stats) {
-                a.out.req_stats[4 * r] = sh.n_layers;
-                a.out.req_stats[4 * r + 1] = sh.n_tests;
-                a.out.req_stats[4 * r + 2] = sh.n_exact;
-                a.out.req_stats[4 * r + 3] = sh.n_respass;
+                int32_t *rs = a.out.req_stats + (int64_t)DSBD_REQ_STATS * r;
+                rs[0] = sh.n_layers; rs[1] = sh.n_tests; rs[2] = sh.n_exact; rs[3] = sh.n_respass;
+                rs[4] = sh.n_near; rs[5] = sh.n_rows; rs[6] = sh.n_wrapped; rs[7] = 0;
             }
         }
         if (sh.err) report(a.status, sh.err);
@@ -1603,7 +1752,7 @@ Layout make_layout(const dsbd_forest_t *f, int V) {
     L.sums = off;
     off = align_up(off + sizeof(double) * (size_t)f->R * 2 * L.max_m * (size_t)L.max_live * L.T, 256);
     L.hist = off;
-    off = align_up(off + sizeof(unsigned long long) * (size_t)f->R * 2 * (4096 + 1), 256);
+    off = align_up(off + sizeof(unsigned long long) * (size_t)f->R * 2 * kHistLen, 256);
 #ifdef DSBD_PHASE_TIMING
     off = align_up(off + sizeof(unsigned long long) * (size_t)f->R * 256, 256);
 #endif
@@ -1640,7 +1789,7 @@ int check_params(const dsbd_verify_params_t *p) {
 }
 
 // Cluster size: as many CTAs per request as its tile count can use, but few enough that all
-// requests are resident at once (four CTAs per SM fit).
+// requests are resident at once (two CTAs per SM fit).
 int cluster_size_for(int tiles, int R) {
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -1649,7 +1798,7 @@ int cluster_size_for(int tiles, int R) {
     else if (tiles >= 64) cs = 8;
     else if (tiles >= 32) cs = 4;
     else if (tiles >= 16) cs = 2;
-    while (cs > 1 && (long long)R * cs > 4ll * sms) cs >>= 1;
+    while (cs > 1 && (long long)R * cs > 2ll * sms) cs >>= 1;
     return cs;
 }
 
@@ -1657,10 +1806,12 @@ int launch_verify(const VerifyArgs &args, int R, int tiles, cudaStream_t stream)
     const int cs = cluster_size_for(tiles, R);
     if (cs > 8 && cudaFuncSetAttribute(k_verify, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
         return DSBD_ERR_CUDA;
+    if (cudaFuncSetAttribute(k_verify, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kVerifyDynSmem) != cudaSuccess)
+        return DSBD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(R * cs));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.blockDim = dim3(kVThreads);
+    cfg.dynamicSmemBytes = kVerifyDynSmem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -166,12 +166,86 @@ def test_peaky_distributions_use_the_exact_fallback():
         ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64))
         e, d = compare_verify(ref, gpu, forest)
         exempt += e; decisions += d
-        st = gpu["req_stats"].reshape(-1, 4)
+        st = gpu["req_stats"].reshape(-1, 8)
         assert np.array_equal(st[:, 0], np.minimum(ref["l_last"], forest["max_depth"]))   # layers verified
         assert st[:, 1].sum() == (ref["trace_kind"] == oracle.TR_ACCEPT).sum()            # accept tests
+        acc = ref["trace_kind"] == oracle.TR_ACCEPT
+        near_ref = int((np.abs(ref["trace_u"][acc] - np.minimum(ref["trace_a"][acc], 1.0)) < 1e-5).sum())
+        assert abs(int(st[:, 4].sum()) - near_ref) <= 1                                    # near ties (the band's edge may differ)
         fallbacks += int(st[:, 2].sum()); respass += int(st[:, 3].sum())
     check_exempt(exempt, decisions)
     assert fallbacks > 0
+
+
+def test_flat_tail_of_tiny_cells():
+    """Rows whose vocabulary is a few heavy tokens plus a flat tail of about 10^5 cells of
+    probability 1e-9 .. 1e-8 each (a per-cell mass near 2^-31): the tail as a whole carries
+    1e-4 .. 1e-3 of the mass, far more than the 1e-5 tie band, so a histogram that rounded such
+    cells to a coarse fixed-point unit would bias every residual mass.  Statuses, widths and
+    tokens must still match the oracle."""
+    rng = np.random.default_rng(21)
+    V, R = 120000, 6
+    forest, prm, _, _, rp, rq, stride = _random_problem(rng, R=R, V=64, gamma=3, max_w=4)
+    N = forest["N"]
+    zp = (-5.0 + 0.4 * rng.standard_normal((N, V))).astype(np.float32)
+    heavy = rng.integers(0, V, size=(N, 40))
+    for n in range(N):
+        zp[n, heavy[n]] = rng.normal(11.0, 1.5, size=40)
+    zq = (zp + 0.5 * rng.standard_normal((N, V))).astype(np.float32)
+    tok = np.zeros(N, np.int32)
+    for n in range(N):
+        par = forest["parent"][n]
+        if par >= 0:
+            tok[n] = heavy[par, rng.integers(0, 40)]
+    forest["token"] = tok
+    prm = dict(prm, V=V, temperature=1.0)
+    dz = lambda a: torch.as_tensor(a).cuda()
+    exempt = decisions = 0
+    for step in range(4):
+        prm["step"] = step
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+        assert status == 0
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64), threads=8)
+        e, d = compare_verify(ref, gpu, forest)
+        exempt += e; decisions += d
+    check_exempt(exempt, decisions)
+    # the tail is real mass: about 120000 cells of e^-5 against heavy cells of about e^11
+    tail = np.exp(zp[0].astype(np.float64)); tail[heavy[0]] = 0.0
+    assert tail.sum() / np.exp(zp[0].astype(np.float64)).sum() > 2e-5
+
+
+def test_proportional_rows_overflow_is_detected():
+    """Both models give the same next-token distribution in every row, so all cells of a row have
+    the same ratio p_beam / q_beam (the ratio of the two beam weights) and land in one histogram
+    bin: more mass than one 32-bit word of the histogram can hold.  The kernel must notice the
+    wrapped word and compute that layer's residual masses by exact passes instead."""
+    rng = np.random.default_rng(22)
+    V = 100000
+    forest, prm, _, _, rp, rq, stride = _random_problem(rng, R=4, V=64, gamma=2, max_w=4)
+    N = forest["N"]
+    zp = rng.normal(0.0, 1.0, size=(N, V)).astype(np.float32)
+    zq = zp.copy()
+    tok = np.zeros(N, np.int32)
+    for n in range(N):
+        if forest["parent"][n] >= 0:
+            tok[n] = rng.integers(0, V)
+    forest["token"] = tok
+    rq = (rp + rng.normal(0, 1.0, len(rp))).astype(np.float32)       # beam weights differ between the models
+    prm = dict(prm, V=V, temperature=1.0, thresh=0.3)
+    dz = lambda a: torch.as_tensor(a).cuda()
+    exempt = decisions = exact = wrapped = 0
+    for step in range(3):
+        prm["step"] = step
+        gpu, status = run_gpu_verify(forest, prm, dz(zp), dz(zq), dz(rp), dz(rq))
+        assert status == 0
+        ref = oracle.verify_step(forest, prm, zp, zq, rp.astype(np.float64), rq.astype(np.float64), threads=8)
+        e, d = compare_verify(ref, gpu, forest)
+        exempt += e; decisions += d
+        st = gpu["req_stats"].reshape(-1, 8)
+        exact += int(st[:, 2].sum())
+        wrapped += int(st[:, 6].sum())
+    check_exempt(exempt, decisions)
+    assert exact > 0 and wrapped > 0
 
 
 @pytest.mark.parametrize("name,steps", [("C1", range(30)), ("C2", range(30)), ("C3", range(4)), ("C4", range(3)),
