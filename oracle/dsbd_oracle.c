@@ -4,6 +4,11 @@
  * Everything here follows the paper's statements in their own order and in double
  * precision; there is no blocking, fusion or reordering.  Parity of per-seed token ids is
  * "parity unpinned" (conventions of this file); the output law is pinned by Theorem 1.
+ * With warped joints (top-k / top-p) the law is pinned at every layer for drafts drawn from the
+ * q_beam this file verifies against (the warp of the joint over the ACCEPTED beams); for drafts
+ * that a drafter drew from the warp of the joint over all its beams, layers >= 2 carry
+ * "parity unpinned: distribution under warping at l >= 2" -- pruning and warping do not
+ * commute, and the size of the difference is recorded in the tests.
  */
 #include "dsbd_oracle.h"
 

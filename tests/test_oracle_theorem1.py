@@ -229,6 +229,109 @@ def test_second_layer_law_equals_beam_sampling(case):
     assert np.abs(law - _product_law(pb, W)).max() < 1e-12
 
 
+def _warped_case(seed, top_k, top_p, need=3):
+    """A toy model and three layer-1 drafts inside the common support of the two warped joints:
+    the two with the largest ratio (accepted by tiny injected uniforms) and the one with the
+    smallest (cut once the width of 2 is reached, so its children are pruned)."""
+    model = ToyModel(seed=seed)
+    pb1 = _warp_ref(model.beam_dist("p", [(0,), (1,)]), top_k, top_p)
+    qb1 = _warp_ref(model.beam_dist("q", [(0,), (1,)]), top_k, top_p)
+    both = np.nonzero((pb1 > 0) & (qb1 > 0))[0]
+    order = both[np.argsort(-(pb1[both] / qb1[both]))]
+    cells = [int(order[0]), int(order[1]), int(order[-1])][:need]
+    assert len(set(cells)) == need
+    return model, [(c // V, c % V) for c in cells]
+
+
+def _second_layer_law(model, layer1, params, drafter_beams, live=(0, 1)):
+    """Exact law of the ordered layer-2 outputs when every layer-2 draft is an iid draw from the
+    warped q joint over the layer-1 drafts `drafter_beams` (x V) and layer 1 accepted the drafts
+    `live`; also returns the product of the warped p joint over the accepted beams."""
+    top_k, top_p = params.get("top_k", 0), params.get("top_p", 1.0)
+    ctx = [(layer1[j][0], layer1[j][1]) for j in drafter_beams]
+    qd = _warp_ref(model.beam_dist("q", ctx), top_k, top_p)
+    support = np.nonzero(qd)[0]
+    layer_lists, probs = [], []
+    for t in itertools.product(support, repeat=3):
+        layer_lists.append([layer1, [(drafter_beams[int(c) // V], int(c) % V) for c in t]])
+        probs.append(float(np.prod(qd[list(t)])))
+    assert abs(sum(probs) - 1) < 1e-12
+    law, W = _layer_law(model, layer_lists, probs, [1e-12, 1e-12], 2, params, gamma=2)
+    live_ctx = [(layer1[j][0], layer1[j][1]) for j in live]
+    order = sorted(range(len(live)), key=lambda j: (layer1[live[j]][0], live[j]))
+    pb = _warp_ref(model.beam_dist("p", [live_ctx[j] for j in order]), top_k, top_p)
+    assert abs(law.sum() - 1) < 1e-10
+    return law, _product_law(pb.reshape(len(live), V), W)
+
+
+@pytest.mark.parametrize("seed,top_k,top_p", [(2, 6, 0.9), (5, 6, 0.8), (7, 4, 1.0), (2, 0, 0.7)])
+def test_second_layer_law_with_warped_joints(seed, top_k, top_p):
+    """Layer 2 with the warping T (Section "Details": p_beam = T o (p/P), q_beam = T o (q/Q) at
+    every layer): when the live drafts are iid draws from the q_beam the verification itself
+    uses -- T applied to the joint over the ACCEPTED layer-1 beams -- the outputs follow the
+    product of T o p_beam^(2) exactly.  This pins the accept / residual arithmetic with warped
+    joints beyond the first layer."""
+    model, layer1 = _warped_case(seed, top_k or 16, top_p)
+    params = dict(W_min=2, W_max=2, W_nom=2, thresh=0.7, top_k=top_k, top_p=top_p)
+    law, expected = _second_layer_law(model, layer1, params, drafter_beams=[0, 1])
+    assert np.abs(law - expected).max() < 1e-12
+
+
+def test_warping_does_not_commute_with_pruning():
+    """The small model drafts layer 2 from T applied to the joint over ALL its layer-1 beams;
+    the verification prunes the children of rejected beams and applies T to the joint over the
+    accepted beams only.  Without warping the two agree (a restriction of the joint is the
+    joint of the restriction) and the outputs are exact.  With warping they do not: the top-k
+    cells of the large joint, restricted, are not the top-k cells of the restricted joint, so
+    the live drafts are not draws from the verification's q_beam and the output law misses the
+    product of T o p_beam^(2).  The size of the miss on this toy problem is recorded here so
+    that a change of reading shows up."""
+    model, layer1 = _warped_case(2, 16, 1.0)
+    unwarped = dict(W_min=2, W_max=2, W_nom=2, thresh=0.7)
+    law, expected = _second_layer_law(model, layer1, unwarped, drafter_beams=[0, 1, 2])
+    assert np.abs(law - expected).max() < 1e-12
+    worst = 0.0
+    for seed, top_k, top_p in [(2, 6, 0.9), (5, 6, 0.8), (7, 4, 1.0)]:
+        model, layer1 = _warped_case(seed, top_k, top_p)
+        params = dict(unwarped, top_k=top_k, top_p=top_p)
+        law, expected = _second_layer_law(model, layer1, params, drafter_beams=[0, 1, 2])
+        tv = 0.5 * np.abs(law - expected).sum()
+        assert 1e-3 < tv < 0.5
+        worst = max(worst, tv)
+    assert worst > 0.05            # total variation 0.10 .. 0.19 on these three cases
+
+
+@pytest.mark.parametrize("top_k,top_p", [(0, 1.0), (5, 0.9)])
+def test_extra_layer_draws_follow_the_warped_joint(top_k, top_p):
+    """All drafts of the only layer accepted: the extra layer's W_nom beams are draws from
+    T o p_beam over (accepted beams x V), each realised by inverse CDF over that vector."""
+    model, layer1 = _warped_case(3, top_k or 16, top_p, need=2)
+    forest, zp, zq, _, _ = build_forest(model, [layer1], gamma=1)
+    prm = dict(V=V, W_min=2, W_max=2, W_nom=3, thresh=0.7, top_k=top_k, top_p=top_p)
+    base = oracle.verify_step(forest, prm, zp, zq, model.root_logp, model.root_logq,
+                              inject_u=[[1e-12, 1e-12] + [0.5] * 6], dist=True)
+    assert base["l_last"][0] == 2 and base["out_width"][0] == 3
+    assert np.all(base["out_source"][:3] == oracle.SRC_EXTRA)
+    # accepted beams in node order, with the p joint of Eq. 1 over them
+    acc = np.nonzero((base["node_status"] == oracle.NODE_ACCEPTED) & (forest["parent"] >= 0))[0]
+    ctxs = []
+    for n in acc:
+        tree = int(np.searchsorted(forest["beam_node_off"], n, side="right") - 1)
+        ctxs.append((tree, int(forest["token"][n])))
+    pb = _warp_ref(model.beam_dist("p", ctxs), top_k, top_p)
+    extra = np.nonzero(base["trace_kind"] == oracle.TR_EXTRA)[0]
+    assert len(extra) == 3
+    for k in range(3):
+        w = base["dist"][k * len(acc) * V:(k + 1) * len(acc) * V]
+        assert np.abs(w - pb).max() < 1e-14
+    cdf = np.concatenate([[0], np.cumsum(pb)])
+    for cell in np.nonzero(pb)[0]:
+        u = (cdf[cell] + cdf[cell + 1]) / 2
+        res = oracle.verify_step(forest, prm, zp, zq, model.root_logp, model.root_logq,
+                                 inject_u=[[1e-12, 1e-12, u, 0.5, 0.5] + [0.5] * 3])
+        assert res["out_parent"][0] == acc[cell // V] and res["out_token"][0] == cell % V
+
+
 def test_sampler_realises_the_reported_mass_vector():
     """Inverse-CDF draws: a uniform in the middle of cell i's CDF interval yields cell i, and
     the interval the oracle reports is the cumulative sum of the vector it reports."""
