@@ -52,5 +52,28 @@ def build(force=False, verbose=False):
     return LIB_PATH
 
 
+WAIT_TEST_LIB = os.path.join(BUILD_DIR, "libdsbd_waittest.so")
+
+
+def build_wait_test(force=False):
+    """A second library for one test: the attention kernel compiled with DSBD_TEST_WAIT_TIMEOUT
+    (short bounded waits, one tile never delivered).  Nothing but that test loads it."""
+    if not force and os.path.exists(WAIT_TEST_LIB) and os.path.getmtime(WAIT_TEST_LIB) >= max(
+            os.path.getmtime(p) for p in _deps()):
+        return WAIT_TEST_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(BUILD_DIR, exist_ok=True)
+    objs = []
+    for src in ("dsbd_api.cu", "dsbd_attention.cu", "dsbd_attention_tc.cu"):
+        obj = os.path.join(BUILD_DIR, "waittest_" + src.replace(".cu", ".o"))
+        objs.append(obj)
+        subprocess.run([nvcc] + NVCC_FLAGS + ["-DDSBD_TEST_WAIT_TIMEOUT", "-c", os.path.join(CSRC, src), "-o", obj],
+                       check=True, stdout=subprocess.PIPE, stderr=subprocess.STDOUT)
+    tmp = WAIT_TEST_LIB + ".tmp.%d" % os.getpid()
+    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
+    os.replace(tmp, WAIT_TEST_LIB)
+    return WAIT_TEST_LIB
+
+
 if __name__ == "__main__":
     print(build(force=True, verbose=True))
