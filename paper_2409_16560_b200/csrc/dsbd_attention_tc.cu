@@ -89,12 +89,22 @@ struct TcArgs {
     int new_layer_rows;               // rows of the k_new / v_new maps between consecutive layers
     int64_t q_layer_stride;           // elements between consecutive layers' q (and out)
     int slots_per_layer;              // partial-result slots of one layer
+    // Tail split of a batch of equal-length units in unit order (no plan kernel): the units from
+    // tail_first on -- those that would leave most CTAs idle in a last, partly filled round --
+    // are cut into tail_k parts each, so that the last round has work for (nearly) every CTA.
+    int tail_first, tail_k;           // tail_k == 0: off
+    // Ragged batch of whole units without a plan kernel: every CTA ranks the units by tile count
+    // itself (longest first, ties by unit number, rounds alternating in direction) and keeps the
+    // entries of its own column.  rank_units = number of units, 0 = off.
+    int rank_units;
 };
 
+constexpr int kMaxRanked = 8;             // items of one CTA when it ranks the units itself
 struct Barriers {
     unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages], s_full[2], p_full[2], pv_done, q_full, o_full;
     uint32_t tmem_base;
     int abort;
+    int my_units[kMaxRanked];             // rank mode: the unit of this CTA's k-th item, -1 for none
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -198,14 +208,34 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
 }
 
 __device__ __forceinline__ int item_count(const TcArgs &a) {
-    return a.items ? *a.n_items : a.n_units * a.row_blocks;
+    if (a.items) return *a.n_items;
+    if (a.rank_units) return (a.rank_units + (int)gridDim.x - 1) / (int)gridDim.x * (int)gridDim.x;
+    if (a.tail_k) return a.tail_first + (a.n_units - a.tail_first) * a.tail_k;
+    return a.n_units * a.row_blocks;
 }
 // The item, with b = -1 when there is nothing to do: a padding entry of the plan, or a row block
 // beyond the rows of this tree.  All three roles of the CTA skip such items alike.
-__device__ __forceinline__ AttnItem get_item(const TcArgs &a, int it) {
+__device__ __forceinline__ AttnItem get_item(const TcArgs &a, int it, const Barriers &sb) {
     AttnItem x;
     if (a.items) {
         x = a.items[it];
+    } else if (a.rank_units) {
+        // (every item index a CTA asks for is in its own column: it % grid == blockIdx.x)
+        const int u = sb.my_units[it / (int)gridDim.x];
+        x.rb = 0; x.b = -1; x.g = 0; x.t0 = 0; x.t1 = 0; x.last = 1; x.nparts = 1; x.slot = 0;
+        if (u >= 0) {
+            x.b = u / a.Hkv; x.g = u - x.b * a.Hkv;
+            x.t1 = (int)(a.prefix_off[x.b + 1] - a.prefix_off[x.b]);
+        }
+    } else if (a.tail_k && it >= a.tail_first) {
+        // part p of tail unit u: equal parts of whole tiles, the tree tile with the last part
+        const int r = it - a.tail_first, u = a.tail_first + r / a.tail_k, p = r - (r / a.tail_k) * a.tail_k;
+        x.rb = 0;
+        x.b = u / a.Hkv; x.g = u - x.b * a.Hkv;
+        const int L = (int)(a.prefix_off[x.b + 1] - a.prefix_off[x.b]);
+        const int plen = ((L + a.tail_k - 1) / a.tail_k + kBN - 1) / kBN * kBN;
+        x.t0 = min(p * plen, L); x.t1 = min(x.t0 + plen, L);
+        x.last = (p == a.tail_k - 1); x.nparts = a.tail_k; x.slot = r;
     } else {
         const int u = it / a.row_blocks;
         x.rb = it - u * a.row_blocks;
@@ -264,6 +294,59 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&sb.tmem_base);
 
+    if (a.rank_units) {
+        // A counting sort by tile count in the (still idle) stage ring: position of a unit = units
+        // with more tiles + earlier units with as many.  Columns are mirrored in odd rounds so
+        // that the CTA with the longest item of one round gets the shortest of the next.  Every
+        // CTA computes the same order and keeps the entries of its own column.
+        int *nt_s = reinterpret_cast<int *>(stage_s);            // [n] tile count of each unit
+        int *start_s = nt_s + 2048;                              // [1024] first position of a tile count
+        const int n = a.rank_units, grid = (int)gridDim.x;
+        for (int i = threadIdx.x; i < 1024; i += kThreadsTc) start_s[i] = 0;
+        if (threadIdx.x < kMaxRanked) sb.my_units[threadIdx.x] = -1;
+        __syncthreads();
+        for (int u = threadIdx.x; u < n; u += kThreadsTc) {
+            const int b = u / a.Hkv;
+            const int nt = min((int)((a.prefix_off[b + 1] - a.prefix_off[b] + kBN - 1) / kBN), 1023);
+            nt_s[u] = nt;
+            atomicAdd(&start_s[nt], 1);                          // counts first
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // counts -> first positions, largest tile count first (lane l owns counts 32l .. 32l+31)
+            int cnt[32], mine = 0;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) { cnt[i] = start_s[1023 - (lane * 32 + i)]; mine += cnt[i]; }
+            int before = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(kFull, before, o);
+                if (lane >= o) before += t;
+            }
+            before -= mine;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) { start_s[1023 - (lane * 32 + i)] = before; before += cnt[i]; }
+            __syncwarp();
+            // units in order, 32 at a time: equal counts inside a group keep their unit order
+            for (int base = 0; base < n; base += 32) {
+                const int u = base + lane;
+                const int nt = u < n ? nt_s[u] : -1 - lane;                  // idle lanes match nobody
+                const unsigned same = __match_any_sync(kFull, nt);
+                if (u < n) {
+                    const int pos = start_s[nt] + __popc(same & ((1u << lane) - 1));
+                    const int round = pos / grid;
+                    int col = pos - round * grid;
+                    if (round & 1) col = grid - 1 - col;
+                    if (col == (int)blockIdx.x && round < kMaxRanked) sb.my_units[round] = u;
+                }
+                __syncwarp();
+                if (u < n && lane == 31 - __clz(same)) start_s[nt] += __popc(same);   // one lane per count
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+    }
+
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -272,7 +355,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const int n_items = item_count(a);
             for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
                 const int layer = u / n_items;
-                const AttnItem item = get_item(a, u - layer * n_items);
+                const AttnItem item = get_item(a, u - layer * n_items, sb);
                 if (item.b < 0) continue;
                 const int b = item.b, g = item.g;
                 const int64_t L = a.prefix_off[b + 1] - a.prefix_off[b];
@@ -333,7 +416,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const uint64_t qd = desc_k_major(smem_u32(q_s));
             const int n_items = item_count(a);
             for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
-                const AttnItem item = get_item(a, u % n_items);
+                const AttnItem item = get_item(a, u % n_items, sb);
                 if (item.b < 0) continue;
                 const int nt = (item.t1 - item.t0 + kBN - 1) / kBN + (item.last ? tree_tiles(a, item.b) : 0);
                 ok = mbar_wait(&sb.q_full, unit & 1, &sb, a.status);
@@ -380,7 +463,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
         bool ok = true;
         const int n_items = item_count(a);
         for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
-            const AttnItem item = get_item(a, u % n_items);
+            const AttnItem item = get_item(a, u % n_items, sb);
             if (item.b < 0) continue;
             const int b = item.b, g = item.g;
             const int64_t L = item.t1;                         // tokens beyond t1 belong to other items
@@ -661,8 +744,15 @@ k_attn_plan(int B, int Hkv, const int64_t *__restrict__ prefix_off, const int32_
 // Merge the parts of every split unit: out = sum_c O_c 2^(m_c - m) / sum_c l_c 2^(m_c - m).
 __global__ void __launch_bounds__(128)
 k_attn_combine(TcArgs a, const UnitParts *__restrict__ units) {
-    const int u = blockIdx.x, layer = blockIdx.y;
-    const UnitParts up = units[u];
+    const int layer = blockIdx.y;
+    int u = blockIdx.x;
+    UnitParts up;
+    if (units) {
+        up = units[u];
+    } else {                                             // tail split: block i merges tail unit i
+        up.first_slot = u * a.tail_k; up.nparts = a.tail_k;
+        u += a.tail_first;
+    }
     if (up.nparts <= 1) return;
     const int b = u / a.Hkv, g = u - b * a.Hkv;
     a.partial += (int64_t)layer * a.slots_per_layer * a.max_rows * 130;
@@ -727,6 +817,8 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, ui
 struct TcPlan {
     int grid, chunk;          // chunk == 0: one item per unit in unit order, no plan kernel
     bool split;               // units are cut into parts (partials + combine kernel)
+    int tail_first, tail_k;   // chunk == 0 only: the units from tail_first on are cut into tail_k parts
+    bool rank;                // chunk == 0 only: the CTAs order the (ragged) units themselves
     int64_t items_max;
     size_t off_items, off_units, off_partial, total;
 };
@@ -767,6 +859,34 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int n_layers
         p.chunk = 0;
         p.items_max = n_units;
         if (p.grid > n_units) p.grid = (int)n_units;
+        p.total = 256;
+        // Equal-length units that do not fill the last round of CTAs: cut the units of that round
+        // into parts so that (nearly) every CTA has a part of it.  1024 units on 296 CTAs are 3.46
+        // rounds: whole units would take the time of 4, with the last 136 units in 2 parts 3.5.
+        const int rem = (int)(n_units % p.grid);
+        const bool uniform = (int64_t)d->max_prefix * f->B == d->total_prefix;
+        if (uniform && n_units > p.grid && rem > 0) {
+            const int tiles = (int)((d->max_prefix + kBN - 1) / kBN);
+            int k = p.grid / rem;
+            if (k > 8) k = 8;
+            if (k > tiles / 8) k = tiles / 8;               // parts of at least 8 tiles
+            if (k >= 2) {
+                p.tail_first = (int)n_units - rem;
+                p.tail_k = k;
+                p.items_max = (int64_t)p.tail_first + (int64_t)rem * k;
+                p.off_partial = 256;
+                p.total = align_up(256 + sizeof(float) * 130 * (size_t)n_layers * (size_t)rem * k *
+                                             (size_t)(f->max_tree_nodes * group), 256);
+            }
+        }
+        return p;
+    }
+    // a ragged batch of whole units, few enough per CTA: no plan kernel, every CTA ranks the units
+    // itself at its start (a few microseconds in parallel instead of a serial kernel ahead of it)
+    if (!p.split && row_blocks == 1 && n_units <= 2048 && n_units <= (int64_t)kMaxRanked * p.grid) {
+        p.chunk = 0;
+        p.rank = true;
+        p.items_max = n_units;
         p.total = 256;
         return p;
     }
@@ -832,7 +952,7 @@ size_t attention_tc_workspace(const dsbd_forest_t *f, const dsbd_attn_desc_t *d,
 
 int attention_tc_launches(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     const TcPlan p = make_plan(f, d);
-    return 1 + (p.chunk > 0 ? 1 : 0) + (p.split ? 1 : 0);
+    return 1 + (p.chunk > 0 ? 1 : 0) + (p.split || p.tail_k ? 1 : 0);
 }
 
 int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const void *q, const void *k_new,
@@ -867,7 +987,14 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.out = static_cast<__nv_bfloat16 *>(out);
     a.status = status;
     a.n_layers = nl; a.pool_layer_rows = LD.pool_rows; a.new_layer_rows = LD.new_rows;
-    a.q_layer_stride = LD.q_stride; a.slots_per_layer = (int)plan.items_max;
+    a.q_layer_stride = LD.q_stride;
+    a.slots_per_layer = plan.tail_k ? (a.n_units - plan.tail_first) * plan.tail_k : (int)plan.items_max;
+    a.tail_first = plan.tail_first; a.tail_k = plan.tail_k;
+    a.rank_units = plan.rank ? a.n_units : 0;
+    if (plan.tail_k) {
+        if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
+        a.partial = reinterpret_cast<float *>(ws + plan.off_partial);
+    }
     UnitParts *units = nullptr;
     if (plan.chunk > 0) {
         if (reinterpret_cast<uintptr_t>(workspace) & 255) return DSBD_ERR_INVALID_ARG;
@@ -902,6 +1029,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     else DSBD_LAUNCH_TC(128, 3);
 #undef DSBD_LAUNCH_TC
     if (plan.split) k_attn_combine<<<dim3(a.n_units, nl), 128, 0, stream>>>(a, units);
+    else if (plan.tail_k) k_attn_combine<<<dim3(a.n_units - plan.tail_first, nl), 128, 0, stream>>>(a, nullptr);
     return cudaGetLastError() == cudaSuccess ? DSBD_OK : DSBD_ERR_CUDA;
 }
 

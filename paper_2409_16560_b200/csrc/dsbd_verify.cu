@@ -240,7 +240,7 @@ struct Shared {
     int n_near, n_rows;                     // accept tests inside the 1e-5 tie band; live rows consulted
     unsigned long long wtot_p[kVWarps], wtot_q[kVWarps];
     double n_cells;                         // cells that entered the layer's histogram
-    unsigned long long w_tot[4];            // what this CTA added to its w words (p, q), and their sums
+    unsigned long long w_tot[10];           // sums of one histogram pass: see histogram_pass / hist_merge
     int wrapped, n_wrapped;                 // a w word of the layer's histogram wrapped; layers where that happened
     double rho[kMaxLive], uu[kMaxLive];     // per live draft: p_beam/q_beam and its uniform
 };
@@ -422,6 +422,16 @@ __device__ void emit_output(const VerifyArgs &a, int r, int *n_out, int parent, 
 
 // Beam weights of the live set: softmax of the cumulative scores over A (Eq. 1 factorised).
 // Called by all lanes of one warp; beam i is handled by lane i % 32.
+// Per-node data of the request that every layer's set-up reads, kept in shared memory when the
+// request is small enough (otherwise the set-up reads the global arrays).
+constexpr int kCacheNodes = 256;
+struct NodeCache {
+    double score_p[kCacheNodes], score_q[kCacheNodes], lse_p[kCacheNodes], lse_q[kCacheNodes];
+    int16_t parent[kCacheNodes];          // local index of the parent, -1 for a root
+    uint8_t depth[kCacheNodes];
+    int on;
+};
+
 // Natural log of the softmax of n scores, by one warp (lanes over the scores).
 __device__ __forceinline__ void log_softmax_warp(const double *s, int n, int lane, double *out) {
     double mx = -INFINITY;
@@ -435,7 +445,9 @@ __device__ __forceinline__ void log_softmax_warp(const double *s, int n, int lan
     __syncwarp();
 }
 
-__device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, const double *sq, int lane) {
+// nc: the request's node cache or nullptr; n_lo: first node of the request.
+__device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, const double *sq, int lane,
+                             const NodeCache *nc = nullptr, int n_lo = 0) {
     log_softmax_warp(sp, sh.nA, lane, sh.lwp);
     log_softmax_warp(sq, sh.nA, lane, sh.lwq);
     for (int i = lane; i < sh.nA; i += 32) {
@@ -443,8 +455,10 @@ __device__ void live_weights(const VerifyArgs &a, Shared &sh, const double *sp, 
         sh.wp[i] = exp(lwp);
         const int row = sh.A[i];
         double rest_p, rest_q;
-        split_offset((lwp - a.lse[row]) / kLn2, &sh.bp[i], &sh.cp[i], &rest_p);
-        split_offset((lwq - a.lse[a.N + row]) / kLn2, &sh.bq[i], &sh.cq[i], &rest_q);
+        const double lse_p = nc ? nc->lse_p[row - n_lo] : a.lse[row];
+        const double lse_q = nc ? nc->lse_q[row - n_lo] : a.lse[a.N + row];
+        split_offset((lwp - lse_p) / kLn2, &sh.bp[i], &sh.cp[i], &rest_p);
+        split_offset((lwq - lse_q) / kLn2, &sh.bq[i], &sh.cq[i], &rest_q);
         sh.dc[i] = (float)(rest_p - rest_q);
     }
     __syncwarp();
@@ -595,11 +609,10 @@ __device__ __forceinline__ void hist_half_tile(const float4 (&vp)[4], const floa
 }
 
 // One cluster-wide pass over the live rows; every CTA fills its own shared-memory histogram.
-// tot[0], tot[1] (shared memory, zero before the call): what the CTA added to its w words.
-// gh: the global image of the histogram (cell count and the last bin are added to it directly).
+// tot (shared memory, zero before the call): [0], [1] what the CTA added to its w words, [4] the
+// cells it added.
 __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, const HistSmem &h,
-                               double *sums1, int cta_rank, int n_cta, unsigned long long *gh,
-                               unsigned long long *tot) {
+                               double *sums1, int cta_rank, int n_cta, unsigned long long *tot) {
     const int lane = threadIdx.x & 31;
     const int warp = cta_rank * kVWarps + (threadIdx.x >> 5);
     const int nwarps = n_cta * kVWarps;
@@ -634,37 +647,84 @@ __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float bins
         ps.tot_q += __shfl_xor_sync(kFull, ps.tot_q, o);
     }
     if (lane == 0) {
-        if (ps.n) atomicAdd(gh + kHistCount, (unsigned long long)ps.n);
+        if (ps.n) atomicAdd(tot + 4, (unsigned long long)ps.n);
         if (ps.tot_p) atomicAdd(tot, ps.tot_p);
         if (ps.tot_q) atomicAdd(tot + 1, ps.tot_q);
     }
 }
 
-// Adds a CTA's shared-memory histogram to its global image (64-bit sums in units of 2^-44) and
-// checks its w words against what the CTA's threads added to them (tot[0..1]; tot[2..3] must be
-// zero before the call and are used as scratch): a difference means that a word wrapped.
-__device__ void hist_flush(const HistSmem &h, unsigned long long *gh, unsigned long long *tot) {
+// Merge of the cluster's histograms, after a cluster barrier that follows the pass: every CTA sums
+// one slice of the bins over all CTAs' shared memory (distributed shared memory loads, no atomics)
+// and stores the 64-bit sums, in units of 2^-44, to the global image, which therefore needs no
+// clearing; the last CTA also folds the copies of the last bin.  Returns through tot[5] the cells
+// of the whole cluster and through tot[6] whether any CTA's w words wrapped (each CTA checks its
+// own words against what its threads added, tot[0..1]).
+// The caller puts a cluster barrier behind this before anyone reads the image or reuses the arrays.
+__device__ void hist_check_local(const HistSmem &h, unsigned long long *tot, unsigned long long *warp_p,
+                                 unsigned long long *warp_q) {
     unsigned long long sp = 0ull, sq = 0ull;
-    for (int i = threadIdx.x; i < kBins + kOverSlots; i += blockDim.x) {
-        const uint32_t wp = h.wp[i], wq = h.wq[i];
-        sp += wp; sq += wq;
-        const unsigned long long P = ((unsigned long long)h.bp[i] << 16) + wp;
-        const unsigned long long Q = ((unsigned long long)h.bq[i] << 16) + wq;
-        const int g = i < kBins ? i : kBins;             // the warps' copies of the last bin are one bin again
-        if (P) atomicAdd(gh + 2 * g, P);
-        if (Q) atomicAdd(gh + 2 * g + 1, Q);
-    }
+    for (int i = threadIdx.x; i < kBins + kOverSlots; i += blockDim.x) { sp += h.wp[i]; sq += h.wq[i]; }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         sp += __shfl_xor_sync(kFull, sp, o);
         sq += __shfl_xor_sync(kFull, sq, o);
     }
-    if ((threadIdx.x & 31) == 0) {
-        if (sp) atomicAdd(tot + 2, sp);
-        if (sq) atomicAdd(tot + 3, sq);
-    }
+    if ((threadIdx.x & 31) == 0) { warp_p[threadIdx.x >> 5] = sp; warp_q[threadIdx.x >> 5] = sq; }
     __syncthreads();
-    if (threadIdx.x == 0 && (tot[0] != tot[2] || tot[1] != tot[3])) atomicAdd(gh + kHistWrapped, 1ull);
+    if (threadIdx.x == 0) {
+        sp = sq = 0ull;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { sp += warp_p[w]; sq += warp_q[w]; }
+        tot[6] = (tot[0] != sp || tot[1] != sq) ? 1ull : 0ull;
+    }
+}
+
+__device__ void hist_merge(cg::cluster_group &cluster, const HistSmem &h, unsigned long long *gh,
+                           unsigned long long *tot, int cta_rank, int n_cta) {
+    const int per = (kBins + n_cta - 1) / n_cta;
+    const int lo = cta_rank * per, hi = min(lo + per, kBins);
+    for (int i = lo + (int)threadIdx.x; i < hi; i += blockDim.x) {
+        unsigned long long P = 0ull, Q = 0ull;
+        for (int c = 0; c < n_cta; ++c) {
+            const uint32_t *wp = cluster.map_shared_rank(h.wp, c), *wq = cluster.map_shared_rank(h.wq, c);
+            const uint32_t *bp = cluster.map_shared_rank(h.bp, c), *bq = cluster.map_shared_rank(h.bq, c);
+            P += ((unsigned long long)bp[i] << 16) + wp[i];
+            Q += ((unsigned long long)bq[i] << 16) + wq[i];
+        }
+        gh[2 * i] = P;
+        gh[2 * i + 1] = Q;
+    }
+    if (cta_rank == n_cta - 1) {
+        // the copies of the last bin (one per warp and half-warp lane, in every CTA) are one bin again
+        unsigned long long P = 0ull, Q = 0ull;
+        for (int i = kBins + (int)threadIdx.x; i < kBins + kOverSlots; i += blockDim.x)
+            for (int c = 0; c < n_cta; ++c) {
+                const uint32_t *wp = cluster.map_shared_rank(h.wp, c), *wq = cluster.map_shared_rank(h.wq, c);
+                const uint32_t *bp = cluster.map_shared_rank(h.bp, c), *bq = cluster.map_shared_rank(h.bq, c);
+                P += ((unsigned long long)bp[i] << 16) + wp[i];
+                Q += ((unsigned long long)bq[i] << 16) + wq[i];
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            P += __shfl_xor_sync(kFull, P, o);
+            Q += __shfl_xor_sync(kFull, Q, o);
+        }
+        if ((threadIdx.x & 31) == 0 && threadIdx.x < kOverSlots) {
+            if (P) atomicAdd(tot + 7, P);
+            if (Q) atomicAdd(tot + 8, Q);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) { gh[2 * kBins] = tot[7]; gh[2 * kBins + 1] = tot[8]; }
+    }
+    if (threadIdx.x == 0) {
+        unsigned long long cells = 0ull, wrapped = 0ull;
+        for (int c = 0; c < n_cta; ++c) {
+            const unsigned long long *t = cluster.map_shared_rank(tot, c);
+            cells += t[4];
+            wrapped |= t[6];
+        }
+        tot[5] = cells;
+        tot[9] = wrapped;
+    }
 }
 
 // One completion draw (residual if s_res > 0 else p_beam) by warp 0; returns the token or -1
@@ -1069,6 +1129,7 @@ k_verify(VerifyArgs a) {
     __shared__ Shared sh;
     __shared__ double sp_live[kMaxLive], sq_live[kMaxLive];
     __shared__ int8_t st[kMaxLive * kMaxLive];     // status of the request's nodes, local index
+    __shared__ NodeCache nc;
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     uint32_t *hp = reinterpret_cast<uint32_t *>(dyn_smem), *hq = hp + kHistWords;     // first two digit arrays
     const HistSmem hs = hist_arrays(hp);
@@ -1203,7 +1264,6 @@ k_verify(VerifyArgs a) {
     }
 
     // ---- set-up ----
-    for (int i = cta_rank * kVThreads + threadIdx.x; i < 2 * hist_len; i += n_cta * kVThreads) ghist[i] = 0ull;
     if (warp == 0) {
         if (lane == 0) {
             sh.err = 0; sh.done = 0; sh.n_out = 0; sh.n_fill = 0;
@@ -1254,10 +1314,26 @@ k_verify(VerifyArgs a) {
         for (int n = threadIdx.x; n < n_req_nodes && st_ok; n += blockDim.x)
             st[n] = a.parent[n_lo + n] < 0 ? DSBD_NODE_ACCEPTED : DSBD_NODE_UNREACHED;
     __threadfence();
-    cluster.sync();                                   // the histogram banks are zero from here on
+    cluster.sync();
     if (!a.select_mode && !st_ok && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_FOREST;
     if (bad_widths && threadIdx.x == 0) sh.err = DSBD_DEV_BAD_PARAM;
+    const bool cached = !a.select_mode && n_req_nodes <= kCacheNodes && a.gamma < 256;
+    if (threadIdx.x == 0) nc.on = cached ? 1 : 0;
+    if (cached)
+        for (int i = threadIdx.x; i < n_req_nodes; i += blockDim.x) {
+            const int n = n_lo + i, par = a.parent[n];
+            nc.score_p[i] = a.score[n];   nc.score_q[i] = a.score[a.N + n];
+            nc.lse_p[i] = a.lse[n];       nc.lse_q[i] = a.lse[a.N + n];
+            nc.parent[i] = (int16_t)((par >= n_lo && par < n) ? par - n_lo : -1);
+            nc.depth[i] = (uint8_t)min(max(a.depth[n], 0), 255);
+        }
     __syncthreads();
+    // node data by local index, from the cache when there is one
+    auto nd_depth = [&](int i) -> int { return cached ? (int)nc.depth[i] : a.depth[n_lo + i]; };
+    auto nd_parent = [&](int i) -> int { return cached ? (int)nc.parent[i] : a.parent[n_lo + i] - n_lo; };
+    auto nd_score = [&](int model, int i) -> double {
+        return cached ? (model ? nc.score_q[i] : nc.score_p[i]) : a.score[(int64_t)model * a.N + n_lo + i];
+    };
 
     for (int l = 1; l <= n_layers && !sh.done && !sh.err; ++l) {
         // ---- live drafts of layer l, in draw order; beam weights ----
@@ -1271,8 +1347,9 @@ k_verify(VerifyArgs a) {
                 for (int base = 0; base < n_req_nodes; base += 32) {
                     const int n = base + lane;
                     bool live = false;
-                    if (n < n_req_nodes && a.depth[n_lo + n] == l) {
-                        live = st[a.parent[n_lo + n] - n_lo] == DSBD_NODE_ACCEPTED;
+                    if (n < n_req_nodes && nd_depth(n) == l) {
+                        const int pl = nd_parent(n);
+                        live = pl >= 0 && st[pl] == DSBD_NODE_ACCEPTED;
                         if (!live) {
                             st[n] = DSBD_NODE_PRUNED;
                             if (writer) a.out.node_status[n_lo + n] = DSBD_NODE_PRUNED;
@@ -1297,7 +1374,7 @@ k_verify(VerifyArgs a) {
                 }
             }
             __syncwarp();
-            live_weights(a, sh, sp_live, sq_live, lane);
+            live_weights(a, sh, sp_live, sq_live, lane, cached ? &nc : nullptr, n_lo);
             if (lane == 0) {
                 sh.m = m;
                 sh.s_arr[0] = 0.0;
@@ -1309,12 +1386,12 @@ k_verify(VerifyArgs a) {
             if (!a.select_mode)
                 for (int i = lane; i < m; i += 32) {
                     const int n = sh.S[i];
-                    const int par = a.parent[n];
+                    const int pl = nd_parent(n - n_lo), par = n_lo + pl;
                     int ai = 0;
                     while (ai < sh.nA && sh.A[ai] != par) ++ai;
                     sh.S_parent_idx[i] = ai;
-                    const double lp = a.score[n] - a.score[par];
-                    const double lq = a.score[a.N + n] - a.score[a.N + par];
+                    const double lp = nd_score(0, n - n_lo) - nd_score(0, pl);
+                    const double lq = nd_score(1, n - n_lo) - nd_score(1, pl);
                     double rho;
                     if (lq == -INFINITY || sh.lwq[ai] == -INFINITY)
                         rho = (lp > -INFINITY && sh.lwp[ai] > -INFINITY) ? INFINITY : 0.0;
@@ -1325,7 +1402,7 @@ k_verify(VerifyArgs a) {
                 }
         }
         for (int i = threadIdx.x; i < kHistArrays * kHistWords; i += blockDim.x) hp[i] = 0u;
-        if (threadIdx.x < 4) sh.w_tot[threadIdx.x] = 0ull;
+        if (threadIdx.x < 10) sh.w_tot[threadIdx.x] = 0ull;
         if (threadIdx.x == 0) sh.wrapped = 0;
         __syncthreads();
         const int m = sh.m;
@@ -1379,27 +1456,26 @@ k_verify(VerifyArgs a) {
             const float binscale = (float)((double)kBins / top);
             unsigned long long *gh = ghist + sh.bank * hist_len;
             histogram_pass(a, sh, binscale, hs, sums_base + ((int64_t)sh.bank * a.max_m) * slot_stride, cta_rank,
-                           n_cta, gh, sh.w_tot);
+                           n_cta, sh.w_tot);
             __syncthreads();
+            hist_check_local(hs, sh.w_tot, sh.wtot_p, sh.wtot_q);
             TS(4);
-            hist_flush(hs, gh, sh.w_tot);
-            __threadfence();
-            cluster.sync();
+            cluster.sync();                            // every CTA's histogram is complete
+            hist_merge(cluster, hs, gh, sh.w_tot, cta_rank, n_cta);
+            cluster.sync();                            // the image is whole (the barrier orders the stores for
+                                                       // the cluster); nobody reads the arrays any more
             TS(5);
-            // the merged histogram into shared memory (over the building arrays, which are flushed)
-            __syncthreads();
+            // the merged histogram into shared memory (over the building arrays)
             for (int i = threadIdx.x; i <= kBins; i += blockDim.x) {
                 sufP[i] = __ldcg(gh + 2 * i);
                 sufQ[i] = __ldcg(gh + 2 * i + 1);
             }
             if (threadIdx.x == 0) {
-                sh.n_cells = (double)__ldcg(gh + kHistCount);
-                sh.wrapped = __ldcg(gh + kHistWrapped) != 0ull;
+                sh.n_cells = (double)sh.w_tot[5];
+                sh.wrapped = sh.w_tot[9] != 0ull;
                 if (sh.wrapped) ++sh.n_wrapped;
             }
             __syncthreads();
-            cluster.sync();                            // everyone has read the bank: it can be cleared
-            for (int i = cta_rank * kVThreads + threadIdx.x; i < hist_len; i += n_cta * kVThreads) gh[i] = 0ull;
             TS(6);
             // in-place suffix sums: sufP[k] = p mass of the bins >= k (17 bins per thread)
             {
@@ -1619,13 +1695,13 @@ k_verify(VerifyArgs a) {
                 int nA = 0;
                 for (int base = 0; base < n_req_nodes; base += 32) {
                     const int n = base + lane;
-                    const bool in = n < n_req_nodes && a.depth[n_lo + n] == l && st[n] == DSBD_NODE_ACCEPTED;
+                    const bool in = n < n_req_nodes && nd_depth(n) == l && st[n] == DSBD_NODE_ACCEPTED;
                     const unsigned mask = __ballot_sync(kFull, in);
                     const int pos = nA + __popc(mask & ((1u << lane) - 1));
                     if (in && pos < kMaxLive) {
                         sh.A[pos] = n_lo + n;
-                        sp_live[pos] = a.score[n_lo + n];
-                        sq_live[pos] = a.score[a.N + n_lo + n];
+                        sp_live[pos] = nd_score(0, n);
+                        sq_live[pos] = nd_score(1, n);
                     }
                     nA += __popc(mask);
                 }
