@@ -33,8 +33,8 @@ UNIT = "nodes/s"
 # from ncu captures of the same kernels on 16 of the 64 requests, scaled by 64/16 (the traffic is
 # proportional to the number of requests).  verify_step_total = the dense pass plus the
 # per-request kernel, which re-reads the live rows.
-NCU_TRAFFIC_BYTES = {"C5": {"forest_attention": 8.698e9, "verify_dense_pass": 4.750e9,
-                            "verify_step_total": 4.750e9 + 0.813e9}}
+NCU_TRAFFIC_BYTES = {"C5": {"forest_attention": 8.709e9, "verify_dense_pass": 4.748e9,
+                            "verify_step_total": 4.748e9 + 0.740e9}}
 
 
 def _peaks():
@@ -274,6 +274,70 @@ def _side_workload(dsbd, inputs, dev, name, steps, warmup, top_k=0, top_p=1.0, p
     return res
 
 
+PHASE_NAMES = {1: "start", 2: "prologue / previous layer's completion", 3: "layer set-up", 4: "histogram pass",
+               5: "merge across the cluster", 6: "image into shared memory", 7: "suffix sums", 8: "residual chain",
+               9: "width and accept loop", 10: "residual pass for a completion draw", 11: "completion draws",
+               12: "extra layer and final writes"}
+
+
+def run_verify_phases(args):
+    """--verify-phases: where the time of the per-request verification kernel goes.  Runs the
+    verification of the workload on a build of the library that stamps %globaltimer at the phase
+    boundaries (DSBD_PHASE_TIMING; slower than the product build, so the shares count, not the
+    absolute times) and prints one JSON line with the time line of the slowest request, the mean
+    per phase over all requests and the end time by number of layers verified."""
+    import torch
+    import paper_2409_16560_b200 as dsbd
+    from paper_2409_16560_b200 import binding, inputs
+    from paper_2409_16560_b200 import build as cuda_build
+    binding.use_library(cuda_build.build_phase_timing())
+    dev = torch.device("cuda", 0)
+    spec = inputs.config(args.workload)
+    if args.requests > 0:
+        spec["R"] = args.requests
+    data = inputs.generate(spec, dev, parts=("verify",), draft_top_k=args.top_k, draft_top_p=args.top_p)
+    forest, prm = data["forest"], dict(data["params"], top_k=args.top_k, top_p=args.top_p)
+    f = dsbd.Forest(forest, dev)
+    R = f.R
+    prm_dev = dict(prm, W_min_r=torch.as_tensor(prm["W_min_r"]).to(dev))
+    vout = dsbd.alloc_verify_out(f, dsbd.default_out_off(forest, prm), dev)
+    ws = torch.zeros(dsbd.verify_workspace(f, prm_dev), dtype=torch.uint8, device=dev)
+    stamps = ws[-R * 256 * 8:]                        # the stamps live behind the workspace proper
+    for step in range(args.warmup + 1):
+        stamps.zero_()
+        prm_dev["step"] = step
+        dsbd.verify_step(f, prm_dev, data["logits_p"], data["logits_q"], data["root_logp"], data["root_logq"], vout,
+                         workspace=ws)
+        torch.cuda.synchronize()
+    dbg = stamps.view(torch.int64).cpu().numpy().reshape(R, 256)
+    t0 = min(int(dbg[r, 0]) & 0xFFFFFFFFFFFF for r in range(R))
+    lines, ends, per_phase = [], [], {}
+    for r in range(R):
+        prev, line = None, []
+        for v in dbg[r]:
+            if v == 0:
+                break
+            slot, t = int(v) >> 48, int(v) & 0xFFFFFFFFFFFF
+            if prev is not None:
+                line.append((slot, (t - prev) / 1e3))
+                per_phase.setdefault(slot, []).append((t - prev) / 1e3)
+            prev = t
+        lines.append(line)
+        ends.append((prev - t0) / 1e3)
+    l_last = vout["l_last"].cpu().numpy()
+    slow = int(np.argmax(ends))
+    out = {"verify_phases": {
+        "workload": args.workload, "requests": R, "top_k": args.top_k, "top_p": args.top_p, "unit": "us",
+        "kernel_span": max(ends),
+        "end_by_l_last": {int(k): round(float(np.mean([e for e, l in zip(ends, l_last) if l == k])), 1)
+                          for k in sorted(set(l_last.tolist()))},
+        "requests_by_l_last": {int(k): int((l_last == k).sum()) for k in sorted(set(l_last.tolist()))},
+        "mean_per_phase": {PHASE_NAMES[k]: round(float(np.mean(v)), 1) for k, v in sorted(per_phase.items())},
+        "slowest_request": {"request": slow, "l_last": int(l_last[slow]),
+                            "time_line": [[PHASE_NAMES[s_], round(d, 1)] for s_, d in lines[slow]]}}}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -293,9 +357,14 @@ def main():
     ap.add_argument("--no-side-workloads", action="store_true",
                     help="skip the extra figures under 'kernels' (C4, C6, the paper's warping on C5, "
                          "several attention layers in one call)")
+    ap.add_argument("--verify-phases", action="store_true",
+                    help="print the phase time line of the per-request verification kernel (a timing "
+                         "build of the library) instead of the benchmark line")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.verify_phases:
+        return run_verify_phases(args)
 
     import torch
     import torch.distributed as dist

@@ -75,7 +75,19 @@ def load():
     path = _build.LIB_PATH
     if not os.path.exists(path) or _build.stale():
         path = _build.build()
-    lib = C.CDLL(path)
+    _lib = _declare(C.CDLL(path))
+    return _lib
+
+
+def use_library(path):
+    """Route every call of this module through another build of the library (a measuring build
+    such as the one `build.build_phase_timing()` makes).  For tools; call it before anything else."""
+    global _lib
+    _lib = _declare(C.CDLL(path))
+    return _lib
+
+
+def _declare(lib):
     lib.dsbd_status_string.restype = C.c_char_p
     lib.dsbd_status_string.argtypes = [C.c_int]
     lib.dsbd_forest_attention_workspace.restype = C.c_size_t
@@ -115,7 +127,6 @@ def load():
     lib.dsbd_draft_layer.restype = C.c_int
     lib.dsbd_draft_layer.argtypes = [C.c_int32, C.c_int32, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, _vp,
                                      _vp, C.c_size_t, _vp, _vp]
-    _lib = lib
     return lib
 
 

@@ -53,26 +53,44 @@ def build(force=False, verbose=False):
 
 
 WAIT_TEST_LIB = os.path.join(BUILD_DIR, "libdsbd_waittest.so")
+PHASES_LIB = os.path.join(BUILD_DIR, "libdsbd_phases.so")
+
+
+def _build_variant(lib_path, tag, sources, define, force):
+    if not force and os.path.exists(lib_path) and os.path.getmtime(lib_path) >= max(
+            os.path.getmtime(p) for p in _deps()):
+        return lib_path
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(BUILD_DIR, exist_ok=True)
+    objs, procs = [], []
+    for src in sources:
+        obj = os.path.join(BUILD_DIR, tag + "_" + src.replace(".cu", ".o"))
+        objs.append(obj)
+        procs.append(subprocess.Popen([nvcc] + NVCC_FLAGS + [define, "-c", os.path.join(CSRC, src), "-o", obj],
+                                      stdout=subprocess.PIPE, stderr=subprocess.STDOUT))
+    for pr in procs:
+        out = pr.communicate()[0].decode()
+        if pr.returncode:
+            print(out)
+            raise RuntimeError("nvcc failed building %s" % lib_path)
+    tmp = lib_path + ".tmp.%d" % os.getpid()
+    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
+    os.replace(tmp, lib_path)
+    return lib_path
 
 
 def build_wait_test(force=False):
     """A second library for one test: the attention kernel compiled with DSBD_TEST_WAIT_TIMEOUT
     (short bounded waits, one tile never delivered).  Nothing but that test loads it."""
-    if not force and os.path.exists(WAIT_TEST_LIB) and os.path.getmtime(WAIT_TEST_LIB) >= max(
-            os.path.getmtime(p) for p in _deps()):
-        return WAIT_TEST_LIB
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    os.makedirs(BUILD_DIR, exist_ok=True)
-    objs = []
-    for src in ("dsbd_api.cu", "dsbd_attention.cu", "dsbd_attention_tc.cu"):
-        obj = os.path.join(BUILD_DIR, "waittest_" + src.replace(".cu", ".o"))
-        objs.append(obj)
-        subprocess.run([nvcc] + NVCC_FLAGS + ["-DDSBD_TEST_WAIT_TIMEOUT", "-c", os.path.join(CSRC, src), "-o", obj],
-                       check=True, stdout=subprocess.PIPE, stderr=subprocess.STDOUT)
-    tmp = WAIT_TEST_LIB + ".tmp.%d" % os.getpid()
-    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
-    os.replace(tmp, WAIT_TEST_LIB)
-    return WAIT_TEST_LIB
+    return _build_variant(WAIT_TEST_LIB, "waittest", ("dsbd_api.cu", "dsbd_attention.cu", "dsbd_attention_tc.cu"),
+                          "-DDSBD_TEST_WAIT_TIMEOUT", force)
+
+
+def build_phase_timing(force=False):
+    """The library compiled with DSBD_PHASE_TIMING: the per-request verification kernel records
+    %globaltimer stamps of its phases behind its workspace.  Loaded by `bench.py --verify-phases`
+    only (a measuring aid, slower than the product library)."""
+    return _build_variant(PHASES_LIB, "phases", SOURCES, "-DDSBD_PHASE_TIMING", force)
 
 
 if __name__ == "__main__":

@@ -572,7 +572,6 @@ __device__ __forceinline__ uint32_t split_mass(float m, uint32_t *b_word) {
 // Per-thread sums of one histogram pass.
 struct PassSums {
     unsigned long long tot_p, tot_q;      // what went into the w words
-    int n;                                // cells with rho > 1
 };
 
 // The cells of one half tile (4 x float4 per lane and model) into the histogram; adds their
@@ -595,7 +594,6 @@ __device__ __forceinline__ void hist_half_tile(const float4 (&vp)[4], const floa
                 const float qm = ex2_approx(fmaf(zq4[c], k2, o.bq)) * o.cq;
                 res1 += fmaxf(pm - qm, 0.f);
                 const float bf = dl * binscale;
-                ++ps.n;
                 // (all cells beyond the last edge in one word would wrap it: every warp has its own)
                 const int bin = bf < (float)kBins ? __float2int_rz(bf) : over_bin;
                 const uint32_t ap = split_mass(pm, h.bp + bin), aq = split_mass(qm, h.bq + bin);
@@ -609,15 +607,14 @@ __device__ __forceinline__ void hist_half_tile(const float4 (&vp)[4], const floa
 }
 
 // One cluster-wide pass over the live rows; every CTA fills its own shared-memory histogram.
-// tot (shared memory, zero before the call): [0], [1] what the CTA added to its w words, [4] the
-// cells it added.
+// tot (shared memory, zero before the call): [0], [1] what the CTA added to its w words.
 __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, const HistSmem &h,
                                double *sums1, int cta_rank, int n_cta, unsigned long long *tot) {
     const int lane = threadIdx.x & 31;
     const int warp = cta_rank * kVWarps + (threadIdx.x >> 5);
     const int nwarps = n_cta * kVWarps;
     const int items = sh.nA * a.T;
-    PassSums ps = {0ull, 0ull, 0};
+    PassSums ps = {0ull, 0ull};
     const int over_bin = kBins + ((threadIdx.x >> 5) & 15) * 16 + (threadIdx.x & 15);
     for (int item = warp; item < items; item += nwarps) {
         const int i = item / a.T, t = item - i * a.T;
@@ -642,12 +639,10 @@ __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float bins
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        ps.n += __shfl_xor_sync(kFull, ps.n, o);
         ps.tot_p += __shfl_xor_sync(kFull, ps.tot_p, o);
         ps.tot_q += __shfl_xor_sync(kFull, ps.tot_q, o);
     }
     if (lane == 0) {
-        if (ps.n) atomicAdd(tot + 4, (unsigned long long)ps.n);
         if (ps.tot_p) atomicAdd(tot, ps.tot_p);
         if (ps.tot_q) atomicAdd(tot + 1, ps.tot_q);
     }
@@ -656,8 +651,8 @@ __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float bins
 // Merge of the cluster's histograms, after a cluster barrier that follows the pass: every CTA sums
 // one slice of the bins over all CTAs' shared memory (distributed shared memory loads, no atomics)
 // and stores the 64-bit sums, in units of 2^-44, to the global image, which therefore needs no
-// clearing; the last CTA also folds the copies of the last bin.  Returns through tot[5] the cells
-// of the whole cluster and through tot[6] whether any CTA's w words wrapped (each CTA checks its
+// clearing; the last CTA also folds the copies of the last bin.  Returns through tot[9] whether
+// any CTA's w words wrapped (each CTA checks its
 // own words against what its threads added, tot[0..1]).
 // The caller puts a cluster barrier behind this before anyone reads the image or reuses the arrays.
 __device__ void hist_check_local(const HistSmem &h, unsigned long long *tot, unsigned long long *warp_p,
@@ -716,13 +711,8 @@ __device__ void hist_merge(cg::cluster_group &cluster, const HistSmem &h, unsign
         if (threadIdx.x == 0) { gh[2 * kBins] = tot[7]; gh[2 * kBins + 1] = tot[8]; }
     }
     if (threadIdx.x == 0) {
-        unsigned long long cells = 0ull, wrapped = 0ull;
-        for (int c = 0; c < n_cta; ++c) {
-            const unsigned long long *t = cluster.map_shared_rank(tot, c);
-            cells += t[4];
-            wrapped |= t[6];
-        }
-        tot[5] = cells;
+        unsigned long long wrapped = 0ull;
+        for (int c = 0; c < n_cta; ++c) wrapped |= cluster.map_shared_rank(tot, c)[6];
         tot[9] = wrapped;
     }
 }
@@ -1471,7 +1461,7 @@ k_verify(VerifyArgs a) {
                 sufQ[i] = __ldcg(gh + 2 * i + 1);
             }
             if (threadIdx.x == 0) {
-                sh.n_cells = (double)sh.w_tot[5];
+                sh.n_cells = (double)sh.nA * (double)a.V;      // every cell of the live rows, at most
                 sh.wrapped = sh.w_tot[9] != 0ull;
                 if (sh.wrapped) ++sh.n_wrapped;
             }
