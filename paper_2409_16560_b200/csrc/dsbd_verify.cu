@@ -540,11 +540,8 @@ constexpr double kUnfix = 1.0 / 17592186044416.0;
 constexpr float kBigCell = 1.f / 65536.f;         // 2^-16: cells from here on put their top part into the b word
 constexpr float kBigFix = 268435456.f;            // 2^28, the unit of the b word is 2^-28
 constexpr double kErrTol = 2.5e-7;                // error bound of F(s) above which it is recomputed exactly
-// global image of one histogram: P and Q of bin i at 2i, 2i+1 (units of 2^-44), then the cell count
-// and the number of CTAs whose w words wrapped
+// global image of one histogram: P and Q of bin i at 2i, 2i+1 (units of 2^-44), two spare words
 constexpr int kHistLen = 2 * (kBins + 1) + 2;
-constexpr int kHistCount = 2 * (kBins + 1);
-constexpr int kHistWrapped = kHistCount + 1;
 
 constexpr int kHistArrays = 4;
 struct HistSmem { uint32_t *wp, *wq, *bp, *bq; };
@@ -789,13 +786,13 @@ static_assert(((sizeof(WarpScratch) + 15) & ~size_t(15)) + 2 * kBoundCache * siz
 static_assert(2 * kMaxCand * (sizeof(double) + sizeof(int)) <= (kBins + 2) * sizeof(uint32_t),
               "the two candidate lists overlay the other histogram array");
 
-// barrier of the 128 threads that work on one model (ids 1 and 2; 0 is __syncthreads)
+// barrier of the kHalf threads that work on one model (ids 1 and 2; 0 is __syncthreads)
 __device__ __forceinline__ void half_sync(int half) {
     asm volatile("bar.sync %0, %1;" ::"r"(half + 1), "r"(kHalf) : "memory");
 }
 
-// Support of the warped joint of one model; called by the 128 threads of half `model` of the CTA
-// (warps 0-3: p, warps 4-7: q), the two halves side by side on their own scratch.  hist_p / hist_q:
+// Support of the warped joint of one model; called by the kHalf threads of half `model` of the CTA
+// (warps 0-7: p, warps 8-15: q), the two halves side by side on their own scratch.  hist_p / hist_q:
 // the two idle histogram arrays.  Returns 0 or a DSBD_DEV_* code (the same on every thread of the
 // half).
 __device__ int build_support(const VerifyArgs &a, const Shared &sh, int model, uint32_t *hist_p, uint32_t *hist_q) {
