@@ -118,39 +118,64 @@ def job_value(nodes_per_rank, world, ms_per_step):
     return nodes_per_rank * world / (ms_per_step * 1e-3)
 
 
-def _cpu_baseline(data_host, spec, threads, budget_s=20.0):
+def _cpu_baseline(data_host, spec, threads, budget_s=20.0, gpu=None):
     """The oracle, as it stands, on a bounded sample of the workload: verification of a few
     requests and attention of a few trees; returns nodes/s of the whole step extrapolated
-    from per-node times, and a description of the sample."""
+    from per-node times, and a description of the sample.  With `gpu` (the library's outputs for
+    the same inputs and Philox step, as numpy arrays) the sampled requests and trees are also
+    compared and the counts returned as the second value."""
     import oracle
     forest = data_host["forest"]
     rbo, bno = forest["req_beam_off"], forest["beam_node_off"]
-    # verification: one request at a time until a third of the budget is used
+    par = {"verify_requests": 0, "verify_decisions": 0, "verify_mismatching_requests": 0,
+           "attention_trees": 0, "attention_max_abs_err": 0.0}
+    # verification: one request at a time until half of the budget is used
     n_ver, t_ver, reqs = 0, 0.0, 0
     for r in range(forest["R"]):
         sub = data_host["verify_sub"](r)
         t0 = time.perf_counter()
-        oracle.verify_step(*sub, trace=False, threads=threads)
+        ref = oracle.verify_step(*sub, trace=False, threads=threads)
         t_ver += time.perf_counter() - t0
         n_ver += sub[0]["N"]
         reqs += 1
+        if gpu is not None:
+            n0, n1 = int(bno[rbo[r]]), int(bno[rbo[r + 1]])
+            g0, w = int(gpu["out_off"][r]), int(ref["out_width"][0])
+            st_ref, st_gpu = ref["node_status"], gpu["node_status"][n0:n1]
+            same = (int(ref["l_last"][0]) == int(gpu["l_last"][r]) and w == int(gpu["out_width"][r])
+                    and np.array_equal(ref["layer_width"][0], gpu["layer_width"][r])
+                    and np.array_equal(st_ref, st_gpu)
+                    and np.array_equal(ref["out_token"][:w], gpu["out_token"][g0:g0 + w])
+                    and np.array_equal(ref["out_source"][:w], gpu["out_source"][g0:g0 + w])
+                    and np.array_equal(ref["out_parent"][:w] + n0, gpu["out_parent"][g0:g0 + w]))
+            par["verify_requests"] += 1
+            # decisions: accept tests (nodes accepted or rejected below the roots) and output beams drawn
+            tested = np.isin(st_ref, (1, 2)) & (sub[0]["parent"] >= 0)
+            par["verify_decisions"] += int(tested.sum()) + int((ref["out_source"][:w] != 0).sum())
+            par["verify_mismatching_requests"] += 0 if same else 1
         if t_ver > budget_s / 2 or reqs >= data_host["max_reqs"]:
             break
     n_att, t_att, beams = 0, 0.0, 0
     for b in range(forest["B"]):
         sub = data_host["attn_sub"](b)
         t0 = time.perf_counter()
-        oracle.forest_attention(*sub, threads=threads)
+        ref = oracle.forest_attention(*sub, threads=threads)
         t_att += time.perf_counter() - t0
         n_att += sub[0]["N"]
         beams += 1
+        if gpu is not None:
+            n0, n1 = int(bno[b]), int(bno[b + 1])
+            par["attention_trees"] += 1
+            par["attention_max_abs_err"] = max(par["attention_max_abs_err"],
+                                               float(np.abs(ref - gpu["attn_out"][n0:n1]).max()))
         if t_att > budget_s / 2 or beams >= data_host["max_beams"]:
             break
     per_node = t_ver / n_ver + t_att / n_att
-    return {"value": 1.0 / per_node, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": "%d of %d requests verified (%.1f s), attention of %d of %d trees (%.1f s); "
-                      "nodes/s = 1 / (verify s/node + attention s/node)" % (
-                          reqs, forest["R"], t_ver, beams, forest["B"], t_att)}
+    res = {"value": 1.0 / per_node, "unit": UNIT, "cores": threads, "kind": "oracle",
+           "sample": "%d of %d requests verified (%.1f s), attention of %d of %d trees (%.1f s); "
+                     "nodes/s = 1 / (verify s/node + attention s/node)" % (
+                         reqs, forest["R"], t_ver, beams, forest["B"], t_att)}
+    return (res, par) if gpu is not None else res
 
 
 def _host_views(data, spec):
@@ -820,9 +845,22 @@ def main():
                 k["frac_of_%s_peak" % peak_kind] = k["gbs"] / peak
                 k["frac_of_8TBs_nominal"] = k["gbs"] / 8000.0
 
-    cpu = None
+    cpu, parity = None, None
     if not args.no_cpu_baseline:
-        cpu = _cpu_baseline(_host_views(data, spec), spec, os.cpu_count() or 1)
+        # the library's results at the Philox step of the inputs' parameters, for the comparison with
+        # the oracle's sample (what the oracle computes on the way is compared, nothing is added to it)
+        attention()
+        verify(int(prm.get("step", 0)))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        gpu_res = {k: vout[k].cpu().numpy() for k in ("l_last", "out_width", "layer_width", "node_status",
+                                                      "out_token", "out_source", "out_parent")}
+        gpu_res["layer_width"] = gpu_res["layer_width"].reshape(f.R, -1)
+        gpu_res["out_off"] = np.asarray(out_off)
+        gpu_res["attn_out"] = attn_out.float().cpu().numpy()
+        cpu, parity = _cpu_baseline(_host_views(data, spec), spec, os.cpu_count() or 1, gpu=gpu_res)
+        parity["note"] = ("the oracle's sample of the cpu_baseline leg against this run's outputs; a mismatching "
+                          "request is one whose layer widths, node statuses or output beams differ in any entry")
 
     # kernels of this library per step: the attention kernel (plus its plan / combine kernels when
     # the launch shape uses them), the dense logits pass and the per-request verification kernel
@@ -841,7 +879,7 @@ def main():
                        "parallelism": "replicas x%d" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "kernels": kernels, "graph_replay_ms_per_step": graph_ms, "pipeline": pipeline,
-            "verify_stats_last_step": verify_stats, "cpu_baseline": cpu}
+            "verify_stats_last_step": verify_stats, "cpu_baseline": cpu, "parity": parity}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
