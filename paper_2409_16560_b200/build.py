@@ -47,7 +47,7 @@ def build(force=False, verbose=False):
         if p.returncode:
             raise RuntimeError("nvcc failed on %s" % src)
     tmp = LIB_PATH + ".tmp.%d" % os.getpid()
-    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
+    subprocess.run([nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", tmp] + objs + ["-lcudart"], check=True)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 
@@ -74,7 +74,7 @@ def _build_variant(lib_path, tag, sources, define, force):
             print(out)
             raise RuntimeError("nvcc failed building %s" % lib_path)
     tmp = lib_path + ".tmp.%d" % os.getpid()
-    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
+    subprocess.run([nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", tmp] + objs + ["-lcudart"], check=True)
     os.replace(tmp, lib_path)
     return lib_path
 
