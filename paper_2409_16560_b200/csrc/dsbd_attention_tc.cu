@@ -148,6 +148,12 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, int x, int y, void *bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(void *bar) {
@@ -353,6 +359,10 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             uint32_t tile = 0;
             bool ok = true;
             const int n_items = item_count(a);
+            // the prefix is read once: its lines are the first to leave L2 again, so that the queries,
+            // the tree's keys and values and the metadata the units keep coming back to stay there
+            uint64_t pol_stream;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
                 const int layer = u / n_items;
                 const AttnItem item = get_item(a, u - layer * n_items, sb);
@@ -382,10 +392,10 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                             y = (page_next * a.Hkv + g) * kBN + layer * a.pool_layer_rows;
                             if (j + 1 < nt_p) page_next = pages[j + 1];
                         }
-                        tma_load_2d(ks, &map_kp, 0, y, &sb.kv_full[s]);
-                        tma_load_2d(ks + kTileBytes / 2, &map_kp, 64, y, &sb.kv_full[s]);
-                        tma_load_2d(vs, &map_vp, 0, y, &sb.kv_full[s]);
-                        tma_load_2d(vs + kTileBytes / 2, &map_vp, 64, y, &sb.kv_full[s]);
+                        tma_load_2d_hint(ks, &map_kp, 0, y, &sb.kv_full[s], pol_stream);
+                        tma_load_2d_hint(ks + kTileBytes / 2, &map_kp, 64, y, &sb.kv_full[s], pol_stream);
+                        tma_load_2d_hint(vs, &map_vp, 0, y, &sb.kv_full[s], pol_stream);
+                        tma_load_2d_hint(vs + kTileBytes / 2, &map_vp, 64, y, &sb.kv_full[s], pol_stream);
                     } else {
                         const int x = g * kD;                                  // tree tile j - nt_p
                         const int y = n_lo + (j - nt_p) * kBN + layer * a.new_layer_rows;
@@ -809,7 +819,8 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, ui
     const cuuint32_t box[2] = {64, (cuuint32_t)kBN};
     const cuuint32_t el[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, el,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
