@@ -7,10 +7,12 @@
 //
 // CTA = 6 warps, two CTAs per SM:
 //   warps 0-3  softmax: warp w owns TMEM lanes 32w..32w+31 = query rows 32w..32w+31, one row per
-//              thread, so row max / row sum are thread-local.  They also stage Q (swizzled, by
-//              hand) at the start of a unit and write O at its end.
+//              thread, so row max / row sum are thread-local.  They write O at a unit's end.
 //   warp 4     TMA producer: K and V tiles (2 x 64x64 bf16 boxes each, 128-byte swizzle) into a
-//              ring of shared-memory stages, completion on mbarriers.
+//              ring of shared-memory stages, completion on mbarriers; and the unit's query rows
+//              (two boxes of 64 columns x group heads x nodes of a 3-D map over q), issued as soon
+//              as the previous unit's last Q K^T product has completed, so that the copy runs
+//              behind that unit's last softmax, P V product and output write.
 //   warp 5     MMA issuer (one lane): S = Q K^T (M128 N64 K16 x 8, both operands K-major in
 //              shared memory) into one of two S buffers in TMEM, one tile ahead, so that it runs
 //              while the softmax warps work on the previous tile; after they have written P
@@ -69,7 +71,8 @@ struct AttnItem { int b, g, t0, t1, last, nparts, slot, rb; };
 struct TcArgs {
     int B, N, Hq, Hkv, group, n_units;
     int max_rows;                     // max over trees of nodes * group
-    int block_rows;                   // query rows per row block: 64 or 128 (the kernel's Q tile)
+    int block_rows;                   // query rows per row block: whole nodes, at most the kernel's Q tile (64 or 128)
+    int nodes_per_block;              // block_rows / group
     int row_blocks;                   // ceil(max_rows / block_rows)
     const AttnItem *items;            // nullptr: one item per unit, in unit order
     const int *n_items;               // device count of items (with items)
@@ -88,6 +91,7 @@ struct TcArgs {
     int pool_layer_rows;              // rows of the pool map between consecutive layers
     int new_layer_rows;               // rows of the k_new / v_new maps between consecutive layers
     int64_t q_layer_stride;           // elements between consecutive layers' q (and out)
+    int q_layer_nodes;                // the same in nodes (rows of the query map between consecutive layers)
     int slots_per_layer;              // partial-result slots of one layer
     // Tail split of a batch of equal-length units in unit order (no plan kernel): the units from
     // tail_first on -- those that would leave most CTAs idle in a last, partly filled round --
@@ -101,7 +105,7 @@ struct TcArgs {
 
 constexpr int kMaxRanked = 8;             // items of one CTA when it ranks the units itself
 struct Barriers {
-    unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages], s_full[2], p_full[2], pv_done, q_full, o_full;
+    unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages], s_full[2], p_full[2], pv_done, q_full, q_empty, o_full;
     uint32_t tmem_base;
     int abort;
     int my_units[kMaxRanked];             // rank mode: the unit of this CTA's k-th item, -1 for none
@@ -152,6 +156,12 @@ __device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *m
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int x, int y, int z, void *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -269,7 +279,7 @@ template <int QROWS, int kStages>
 __global__ void __launch_bounds__(kThreadsTc, 2)
 k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_constant__ CUtensorMap map_vp,
                  const __grid_constant__ CUtensorMap map_kn, const __grid_constant__ CUtensorMap map_vn,
-                 TcArgs a) {
+                 const __grid_constant__ CUtensorMap map_q, TcArgs a) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr uint32_t kQBytes = QROWS * kD * 2;
     unsigned char *q_s = smem;                               // [2 halves][QROWS rows][128 B], swizzled
@@ -285,7 +295,8 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
         for (int s = 0; s < kStages; ++s) { mbar_init(&sb.kv_full[s], 1); mbar_init(&sb.kv_empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sb.s_full[b], 1); mbar_init(&sb.p_full[b], 4); }
         mbar_init(&sb.pv_done, 1);
-        mbar_init(&sb.q_full, 128);
+        mbar_init(&sb.q_full, 1);
+        mbar_init(&sb.q_empty, 1);
         mbar_init(&sb.o_full, 1);
         sb.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -356,7 +367,7 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t tile = 0;
+            uint32_t tile = 0, unit = 0;
             bool ok = true;
             const int n_items = item_count(a);
             // the prefix is read once: its lines are the first to leave L2 again, so that the queries,
@@ -376,6 +387,19 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                 const int nt_p = (item.t1 - item.t0 + kBN - 1) / kBN;
                 const int n_lo = a.beam_node_off[b];
                 const int nt = nt_p + (item.last ? tree_tiles(a, b) : 0);
+                // The unit's query rows: one box per 64-column half, rows = (node, query head of this
+                // KV head) in the order the MMA reads them.  The single Q buffer is free once the
+                // previous unit's last Q K^T product has completed, which is while that unit's last
+                // softmax, P V product and output write are still running: the copy hides behind them.
+                if (unit > 0) ok = mbar_wait(&sb.q_empty, (unit - 1) & 1, &sb, a.status);
+                if (!ok) break;
+                {
+                    const int z = n_lo + item.rb * a.nodes_per_block + layer * a.q_layer_nodes;
+                    mbar_expect_tx(&sb.q_full, (uint32_t)a.block_rows * kD * 2);
+                    tma_load_3d(q_s, &map_q, 0, g * a.group, z, &sb.q_full);
+                    tma_load_3d(q_s + QROWS * 128, &map_q, 64, g * a.group, z, &sb.q_full);
+                }
+                ++unit;
                 for (int j = 0; j < nt && ok; ++j, ++tile) {
                     const int s = tile % kStages;
                     const uint32_t par = (tile / kStages) & 1;
@@ -447,8 +471,13 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     return true;
                 };
                 if (ok) ok = issue_s(tile);
+                if (ok && nt == 1) tc_commit(&sb.q_empty);       // the unit's last (only) Q K^T product
                 for (int j = 0; j < nt && ok; ++j, ++tile) {
-                    if (j + 1 < nt) { ok = issue_s(tile + 1); if (!ok) break; }
+                    if (j + 1 < nt) {
+                        ok = issue_s(tile + 1);
+                        if (!ok) break;
+                        if (j + 2 == nt) tc_commit(&sb.q_empty);
+                    }
                     const int s = tile % kStages;
                     ok = mbar_wait(&sb.p_full[tile & 1], (tile >> 1) & 1, &sb, a.status);
                     if (!ok) break;
@@ -482,29 +511,12 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             const int n_tree = a.beam_node_off[b + 1] - n_lo;
             const int nt = nt_p + (item.last ? (n_tree + kBN - 1) / kBN : 0);
             const int M = n_tree * a.group;
-            const int r0 = item.rb * QROWS;                     // first row of this row block
-            // (with the 64-row tile the MMA's rows 64..127 hold no query: never active)
-            const bool warp_active = warp * 32 < QROWS && r0 + warp * 32 < M;
-            const bool active = row < QROWS && r0 + row < M;
+            const int r0 = item.rb * a.block_rows;              // first row of this row block
+            // (the MMA's rows from block_rows on hold no query of this block: never active)
+            const bool warp_active = warp * 32 < a.block_rows && r0 + warp * 32 < M;
+            const bool active = row < a.block_rows && r0 + row < M;
             const int node = active ? (r0 + row) / a.group : 0;
             const int hq = g * a.group + (active ? r0 + row - node * a.group : 0);
-            // ---- stage Q (rows >= M zero) and the ancestor masks; the previous unit's MMAs are done
-            {
-                const int t128 = threadIdx.x;                        // 0..127
-                const __nv_bfloat16 *q_l = a.q + (int64_t)(u / n_items) * a.q_layer_stride;
-                for (int i = t128; i < QROWS * 16; i += 128) {
-                    const int r = i >> 4, c = i & 15;                // row, 16-byte chunk of the 256-byte row
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (r0 + r < M) {
-                        const int nd = (r0 + r) / a.group, hh = g * a.group + (r0 + r - nd * a.group);
-                        v = *reinterpret_cast<const uint4 *>(q_l + ((int64_t)(n_lo + nd) * a.Hq + hh) * kD + c * 8);
-                    }
-                    const int half = c >> 3, cc = c & 7;
-                    *reinterpret_cast<uint4 *>(q_s + half * (QROWS * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(&sb.q_full);
-            }
             // ancestor-or-self mask of this row's node: walk up the tree
             unsigned long long anc_lo = 0ull, anc_hi = 0ull;       // nodes 0..63, 64..127
             {
@@ -824,6 +836,20 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// q as [nodes, Hq, 128] bf16: boxes of 64 columns x `group` heads x `nodes` nodes, i.e. the query rows
+// of one KV head for a run of nodes, in (node, head) order.
+bool make_map_q(CUtensorMap *m, const void *base, uint64_t Hq, uint64_t nodes_total, uint32_t group, uint32_t nodes) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, Hq, nodes_total};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, Hq * kD * 2};
+    const cuuint32_t box[3] = {64, group, nodes};
+    const cuuint32_t el[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, el,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Launch shape shared by the workspace query and the launch.
 struct TcPlan {
     int grid, chunk;          // chunk == 0: one item per unit in unit order, no plan kernel
@@ -838,10 +864,16 @@ struct TcPlan {
 // forests whose AVERAGE tree has at most 64 rows even when the largest is bigger (a sampled
 // forest puts most drafts under a few roots and leaves the other trees tiny): the big trees then
 // run as several 64-row blocks, the many small ones at the faster shape.
-int block_rows_for(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+int tile_rows_for(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
     const int group = d->Hq / d->Hkv;
     if (f->max_tree_nodes * group <= 64) return 64;
-    return (int64_t)f->N * group <= (int64_t)64 * f->B ? 64 : kRows;
+    return ((int64_t)f->N * group <= (int64_t)64 * f->B && group <= 64) ? 64 : kRows;
+}
+// Rows of a row block: whole nodes (the copy engine fetches a block's query rows as a box of nodes x
+// heads), as many as the tile holds.
+int block_rows_for(const dsbd_forest_t *f, const dsbd_attn_desc_t *d) {
+    const int group = d->Hq / d->Hkv;
+    return tile_rows_for(f, d) / group * group;
 }
 
 TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int n_layers = 1) {
@@ -850,7 +882,7 @@ TcPlan make_plan(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int n_layers
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int group = d->Hq / d->Hkv;
     const int block_rows = block_rows_for(f, d);
-    const bool small_q = block_rows == 64;
+    const bool small_q = tile_rows_for(f, d) == 64;
     p.grid = small_q ? 2 * sms : sms;
     const int row_blocks = (f->max_tree_nodes * group + block_rows - 1) / block_rows;
     const int64_t n_units = (int64_t)f->B * d->Hkv * row_blocks;     // counted with their row blocks
@@ -933,7 +965,7 @@ LayerDims layer_dims(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const ds
     const int64_t ps = pages->pool_layer_stride, ns = pages->new_layer_stride, qs = pages->q_layer_stride;
     L.ok = ps >= pages->n_pages * page_elems && ps % ((int64_t)kBN * kD) == 0 &&
            ns >= (int64_t)f->N * new_row && ns % new_row == 0 &&
-           qs >= (int64_t)f->N * d->Hq * kD && qs % 8 == 0;
+           qs >= (int64_t)f->N * d->Hq * kD && qs % ((int64_t)d->Hq * kD) == 0;
     if (!L.ok) return L;
     const int64_t pool_rows = ps / kD, new_rows = ns / new_row;
     // row coordinates of the maps are 32-bit
@@ -944,6 +976,7 @@ LayerDims layer_dims(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const ds
 
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages) {
     if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
+    if (d->Hq / d->Hkv > kRows) return false;                                // a node's rows fit one tile
     if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows * 8) return false;      // up to 8 row blocks
     if (f->max_tree_nodes > 2 * kBN) return false;                           // two tree tiles
     if (d->total_prefix <= 0) return false;
@@ -970,7 +1003,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
                         const void *v_new, const void *k_prefix, const void *v_prefix, const int64_t *prefix_off,
                         void *out, void *workspace, size_t workspace_bytes, int32_t *status, cudaStream_t stream,
                         const dsbd_kv_pages_t *pages) {
-    CUtensorMap kp, vp, kn, vn;
+    CUtensorMap kp, vp, kn, vn, qm;
     const LayerDims LD = layer_dims(f, d, pages);
     if (!LD.ok) return DSBD_ERR_INVALID_ARG;
     const int nl = LD.n_layers;
@@ -982,6 +1015,12 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
         !make_map(&kn, k_new, (uint64_t)d->Hkv * kD, nrows, (uint64_t)d->Hkv * kD * 2) ||
         !make_map(&vn, v_new, (uint64_t)d->Hkv * kD, nrows, (uint64_t)d->Hkv * kD * 2))
         return DSBD_ERR_CUDA;
+    const int group = d->Hq / d->Hkv, block_rows = block_rows_for(f, d);
+    const int64_t q_layer_nodes = nl > 1 ? LD.q_stride / ((int64_t)d->Hq * kD) : 0;
+    if ((uint64_t)f->N + (uint64_t)(nl - 1) * q_layer_nodes >= ((uint64_t)1 << 31)) return DSBD_ERR_UNSUPPORTED;
+    if (!make_map_q(&qm, q, (uint64_t)d->Hq, (uint64_t)f->N + (uint64_t)(nl - 1) * q_layer_nodes, (uint32_t)group,
+                    (uint32_t)(block_rows / group)))
+        return DSBD_ERR_CUDA;
     const TcPlan plan = make_plan(f, d, nl);
     if (workspace_bytes < plan.total) return DSBD_ERR_WORKSPACE_TOO_SMALL;
     char *ws = static_cast<char *>(workspace);
@@ -989,7 +1028,8 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.B = f->B; a.N = f->N; a.Hq = d->Hq; a.Hkv = d->Hkv; a.group = d->Hq / d->Hkv;
     a.n_units = f->B * d->Hkv;
     a.max_rows = f->max_tree_nodes * a.group;
-    a.block_rows = block_rows_for(f, d);
+    a.block_rows = block_rows;
+    a.nodes_per_block = block_rows / group;
     a.row_blocks = (a.max_rows + a.block_rows - 1) / a.block_rows;
     a.scale_log2 = d->scale * 1.4426950408889634f;
     a.beam_node_off = f->beam_node_off; a.parent = f->parent; a.prefix_off = prefix_off;
@@ -999,6 +1039,7 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     a.status = status;
     a.n_layers = nl; a.pool_layer_rows = LD.pool_rows; a.new_layer_rows = LD.new_rows;
     a.q_layer_stride = LD.q_stride;
+    a.q_layer_nodes = (int)q_layer_nodes;
     a.slots_per_layer = plan.tail_k ? (a.n_units - plan.tail_first) * plan.tail_k : (int)plan.items_max;
     a.tail_first = plan.tail_first; a.tail_k = plan.tail_k;
     a.rank_units = plan.rank ? a.n_units : 0;
@@ -1023,18 +1064,18 @@ int launch_attention_tc(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const
     if (nl > 1) {
         int dev = 0, sms = 148;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        const int full = a.block_rows == 64 ? 2 * sms : sms;
+        const int full = tile_rows_for(f, d) == 64 ? 2 * sms : sms;
         if (plan.chunk == 0) grid = (int)std::min<int64_t>((int64_t)plan.items_max * nl, full);
     }
     // up to 64 query rows: 16 KB of Q, three stages, two CTAs per SM; more rows: one CTA per SM
-    const bool small_q = a.block_rows == 64;
+    const bool small_q = tile_rows_for(f, d) == 64;
 #define DSBD_LAUNCH_TC(QR, ST)                                                                              \
     do {                                                                                                   \
         constexpr uint32_t bytes = smem_bytes(QR, ST);                                                     \
         if (cudaFuncSetAttribute(k_forest_attn_tc<QR, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
                                  (int)bytes) != cudaSuccess)                                               \
             return DSBD_ERR_CUDA;                                                                          \
-        k_forest_attn_tc<QR, ST><<<grid, kThreadsTc, bytes, stream>>>(kp, vp, kn, vn, a);                  \
+        k_forest_attn_tc<QR, ST><<<grid, kThreadsTc, bytes, stream>>>(kp, vp, kn, vn, qm, a);                  \
     } while (0)
     if (small_q) DSBD_LAUNCH_TC(64, 3);
     else DSBD_LAUNCH_TC(128, 3);
