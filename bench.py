@@ -33,7 +33,7 @@ UNIT = "nodes/s"
 # from ncu captures of the same kernels on 16 of the 64 requests, scaled by 64/16 (the traffic is
 # proportional to the number of requests).  verify_step_total = the dense pass plus the
 # per-request kernel, which re-reads the live rows.
-NCU_TRAFFIC_BYTES = {"C5": {"forest_attention": 8.709e9, "verify_dense_pass": 4.748e9,
+NCU_TRAFFIC_BYTES = {"C5": {"forest_attention": 8.665e9, "verify_dense_pass": 4.748e9,
                             "verify_step_total": 4.748e9 + 0.740e9}}
 
 
