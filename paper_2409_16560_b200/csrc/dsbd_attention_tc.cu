@@ -370,10 +370,12 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
             uint32_t tile = 0, unit = 0;
             bool ok = true;
             const int n_items = item_count(a);
-            // the prefix is read once: its lines are the first to leave L2 again, so that the queries,
+            // a prefix that is read once: its lines are the first to leave L2 again, so that the queries,
             // the tree's keys and values and the metadata the units keep coming back to stay there
+            // (with several row blocks per unit the blocks read the same prefix: ordinary policy)
             uint64_t pol_stream;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            if (a.row_blocks == 1) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol_stream));
             for (int u = blockIdx.x; u < n_items * a.n_layers && ok; u += gridDim.x) {
                 const int layer = u / n_items;
                 const AttnItem item = get_item(a, u - layer * n_items, sb);
