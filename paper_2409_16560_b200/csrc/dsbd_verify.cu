@@ -556,29 +556,34 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// A cell's mass as a count of 2^-44 units for the w word; a cell of at least 2^-16 (rare) first
-// moves its whole multiples of 2^-28 to the b word.  Exact for a mass of at least 2^-20.
-__device__ __forceinline__ uint32_t split_mass(float m, uint32_t *b_word) {
-    if (m >= kBigCell) {
-        const float hf = floorf(m * kBigFix);
-        m = fmaf(-hf, 1.f / kBigFix, m);                        // exact remainder, below 2^-28
-        atomicAdd(b_word, (uint32_t)hf);
-    }
-    return __float2uint_rn(m * kFix);
-}
 // Per-thread sums of one histogram pass.
 struct PassSums {
-    unsigned long long tot_p, tot_q;      // what went into the w words
+    unsigned long long tot;               // what went into the w words (p and q together)
 };
 
 // The cells of one half tile (4 x float4 per lane and model) into the histogram; adds their
-// (p - q)+ to res1.
+// (p - q)+, in units of 2^-44, to res1u.
+// The work per cell decides the speed of this pass (it is bound by instruction issue, not by
+// memory), so the common case is straight-line code: masses are computed directly in units
+// (the row's factor 2^rest carries the 2^44), the bin comes from an fma onto 1.5 * 2^23 whose
+// low mantissa bits are then the integer (no conversion instruction), the two atomic adds, the
+// residual sum and the check sum are predicated on p_beam > q_beam inside one asm block, and only a
+// cell of at least 2^-16 (rare) takes a branch.
+// wbase: shared-memory byte address of wp[0] minus 4 * (the bits of the fma's constant), so that
+// the address of a bin's word is wbase + 4 * (bits of the fma's result); the q array follows the p
+// array at kHistWords words, the b arrays at twice that.
 // (ex2.approx flushes results below 2^-126 to zero; a cell enters the sums from 2^-45 on.)
+constexpr float kBinMagic = 12582912.f;                         // 1.5 * 2^23
+constexpr float kBigUnits = 268435456.f;                        // 2^28 units = a cell of 2^-16
 __device__ __forceinline__ void hist_half_tile(const float4 (&vp)[4], const float4 (&vq)[4], float k2,
-                                               const RowOff &o, float binscale, const HistSmem &h, float &res1,
-                                               PassSums &ps, int over_bin) {
-    const float bd = (o.bp - o.bq) + o.dc;                      // log2(rho) = (zp - zq) k2 + bd
-    uint32_t tp = 0u, tq = 0u;                                  // below 2^32: 16 cells of less than 2^28 units
+                                               const RowOff &o, float binscale, float half_bin, float top, uint32_t wbase,
+                                               float &res1u, PassSums &ps, uint32_t over_bits) {
+    // dl = log2(rho) - half: the half bin (in log2 units) that turns the fma's round-to-nearest into
+    // the bin's floor is part of the row offset, so p_beam > q_beam reads dl > -half
+    const float bd = ((o.bp - o.bq) + o.dc) - half_bin;
+    const float pass_thr = -half_bin;
+    const float cpu = o.cp * kFix, cqu = o.cq * kFix;           // exact: powers of two
+    uint32_t t0 = 0u, t1 = 0u;                                  // each below 2^32: 8 cells x 2 x less than 2^28 units
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
         const float zp4[4] = {vp[it].x, vp[it].y, vp[it].z, vp[it].w};
@@ -586,33 +591,60 @@ __device__ __forceinline__ void hist_half_tile(const float4 (&vp)[4], const floa
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const float dl = fmaf(zp4[c] - zq4[c], k2, bd);     // NaN compares false
-            if (dl > 0.f) {
-                const float pm = ex2_approx(fmaf(zp4[c], k2, o.bp)) * o.cp;
-                const float qm = ex2_approx(fmaf(zq4[c], k2, o.bq)) * o.cq;
-                res1 += fmaxf(pm - qm, 0.f);
-                const float bf = dl * binscale;
-                // (all cells beyond the last edge in one word would wrap it: every warp has its own)
-                const int bin = bf < (float)kBins ? __float2int_rz(bf) : over_bin;
-                const uint32_t ap = split_mass(pm, h.bp + bin), aq = split_mass(qm, h.bq + bin);
-                tp += ap; tq += aq;
-                atomicAdd(h.wp + bin, ap);
-                atomicAdd(h.wq + bin, aq);
+            float pmu = ex2_approx(fmaf(zp4[c], k2, o.bp)) * cpu;
+            float qmu = ex2_approx(fmaf(zq4[c], k2, o.bq)) * cqu;
+            const float diff = fmaxf(pmu - qmu, 0.f);
+            // floor(log2(rho) * binscale) in the low bits (round to nearest of x - 0.5; an x that is a
+            // whole number may fall to either side, both within the bins' edge tolerance)
+            const float tb = fmaf(dl, binscale, kBinMagic);
+            // (all cells beyond the last edge in one word would wrap it: every warp and half-warp
+            // lane has its own copy of that bin)
+            const uint32_t bits = dl < top ? __float_as_uint(tb) : over_bits;
+            const uint32_t addr = wbase + (bits << 2);
+            if (pmu >= kBigUnits && dl > pass_thr) {
+                // whole multiples of 2^-28 of a big cell go to the b word (units of 2^-28), the
+                // remainder (below 2^16 units) stays for the w word
+                const float hp = floorf(pmu * (1.f / 65536.f));
+                pmu = fmaf(-hp, 65536.f, pmu);
+                asm volatile("red.shared.add.u32 [%0+%1], %2;" ::"r"(addr), "n"(2 * kHistWords * 4), "r"((uint32_t)hp) : "memory");
+                if (qmu >= kBigUnits) {
+                    const float hq = floorf(qmu * (1.f / 65536.f));
+                    qmu = fmaf(-hq, 65536.f, qmu);
+                    asm volatile("red.shared.add.u32 [%0+%1], %2;" ::"r"(addr), "n"(3 * kHistWords * 4), "r"((uint32_t)hq) : "memory");
+                }
             }
+            const uint32_t ap = __float2uint_rn(pmu), aq = __float2uint_rn(qmu);
+            uint32_t &tacc = (it < 2) ? t0 : t1;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "setp.gt.f32 p, %2, %8;\n\t"
+                "@p red.shared.add.u32 [%3], %4;\n\t"
+                "@p red.shared.add.u32 [%3+%6], %5;\n\t"
+                "@p add.f32 %0, %0, %7;\n\t"
+                "@p add.u32 %1, %1, %4;\n\t"
+                "@p add.u32 %1, %1, %5;\n\t}"
+                : "+f"(res1u), "+r"(tacc)
+                : "f"(dl), "r"(addr), "r"(ap), "r"(aq), "n"(kHistWords * 4), "f"(diff), "f"(pass_thr)
+                : "memory");
         }
     }
-    ps.tot_p += tp; ps.tot_q += tq;
+    ps.tot += (unsigned long long)t0 + t1;
 }
 
 // One cluster-wide pass over the live rows; every CTA fills its own shared-memory histogram.
-// tot (shared memory, zero before the call): [0], [1] what the CTA added to its w words.
+// tot (shared memory, zero before the call): [0] what the CTA added to its w words (p and q).
 __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float binscale, const HistSmem &h,
                                double *sums1, int cta_rank, int n_cta, unsigned long long *tot) {
     const int lane = threadIdx.x & 31;
     const int warp = cta_rank * kVWarps + (threadIdx.x >> 5);
     const int nwarps = n_cta * kVWarps;
     const int items = sh.nA * a.T;
-    PassSums ps = {0ull, 0ull};
-    const int over_bin = kBins + ((threadIdx.x >> 5) & 15) * 16 + (threadIdx.x & 15);
+    PassSums ps = {0ull};
+    const uint32_t magic_bits = __float_as_uint(kBinMagic);
+    const uint32_t wbase = (uint32_t)__cvta_generic_to_shared(h.wp) - (magic_bits << 2);
+    const uint32_t over_bits = magic_bits + (uint32_t)(kBins + ((threadIdx.x >> 5) & 15) * 16 + (threadIdx.x & 15));
+    const float half_bin = 0.5f / binscale;                      // half a bin in log2 units
+    const float top = (float)kBins / binscale - half_bin;        // log2 of the last edge (minus the half), as the bins see it
     for (int item = warp; item < items; item += nwarps) {
         const int i = item / a.T, t = item - i * a.T;
         const int row = sh.A[i];
@@ -620,37 +652,30 @@ __device__ void histogram_pass(const VerifyArgs &a, const Shared &sh, float bins
         const float *rq = a.zq + (int64_t)row * a.stride;
         const bool al = ((reinterpret_cast<uintptr_t>(rp) | reinterpret_cast<uintptr_t>(rq)) & 15) == 0;
         const RowOff ro = {sh.bp[i], sh.bq[i], sh.cp[i], sh.cq[i], sh.dc[i]};
-        float res1 = 0.f;                                // sum of (p - q)+ over the tile: residual mass at s = 1
+        float res1u = 0.f;                               // sum of (p - q)+ over the tile in units: residual mass at s = 1
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             float4 vp[4], vq[4];
             const int e0 = t * kTile + half * (kTile / 2);
             load_half_tile(rp, e0, a.V, al, lane, vp);
             load_half_tile(rq, e0, a.V, al, lane, vq);
-            hist_half_tile(vp, vq, a.k2, ro, binscale, h, res1, ps, over_bin);
+            hist_half_tile(vp, vq, a.k2, ro, binscale, half_bin, top, wbase, res1u, ps, over_bits);
         }
         // tile sums of the residual after ONE rejection (s_1 = 1): what a completion draw at run
         // position 2 searches, so that this common case needs no second pass over the rows
-        const double tot1 = warp_sum((double)res1);
+        const double tot1 = warp_sum((double)res1u) * kUnfix;
         if (lane == 0) sums1[item] = tot1;
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        ps.tot_p += __shfl_xor_sync(kFull, ps.tot_p, o);
-        ps.tot_q += __shfl_xor_sync(kFull, ps.tot_q, o);
-    }
-    if (lane == 0) {
-        if (ps.tot_p) atomicAdd(tot, ps.tot_p);
-        if (ps.tot_q) atomicAdd(tot + 1, ps.tot_q);
-    }
+    for (int o = 16; o > 0; o >>= 1) ps.tot += __shfl_xor_sync(kFull, ps.tot, o);
+    if (lane == 0 && ps.tot) atomicAdd(tot, ps.tot);
 }
 
 // Merge of the cluster's histograms, after a cluster barrier that follows the pass: every CTA sums
 // one slice of the bins over all CTAs' shared memory (distributed shared memory loads, no atomics)
 // and stores the 64-bit sums, in units of 2^-44, to the global image, which therefore needs no
 // clearing; the last CTA also folds the copies of the last bin.  Returns through tot[9] whether
-// any CTA's w words wrapped (each CTA checks its
-// own words against what its threads added, tot[0..1]).
+// any CTA's w words wrapped (each CTA checks its own words against what its threads added, tot[0]).
 // The caller puts a cluster barrier behind this before anyone reads the image or reuses the arrays.
 __device__ void hist_check_local(const HistSmem &h, unsigned long long *tot, unsigned long long *warp_p,
                                  unsigned long long *warp_q) {
@@ -666,7 +691,7 @@ __device__ void hist_check_local(const HistSmem &h, unsigned long long *tot, uns
     if (threadIdx.x == 0) {
         sp = sq = 0ull;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { sp += warp_p[w]; sq += warp_q[w]; }
-        tot[6] = (tot[0] != sp || tot[1] != sq) ? 1ull : 0ull;
+        tot[6] = (tot[0] != sp + sq) ? 1ull : 0ull;               // a wrapped word lowers sp + sq by 2^32
     }
 }
 
