@@ -270,6 +270,12 @@ __device__ __forceinline__ int tree_tiles(const TcArgs &a, int b) {
     return (a.beam_node_off[b + 1] - a.beam_node_off[b] + kBN - 1) / kBN;
 }
 
+__device__ __forceinline__ float ex2_ftz(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t *>(&v);
@@ -553,13 +559,17 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                         const int64_t left = L - item.t0 - (int64_t)j * kBN;
                         vis = left >= 64 ? ~0ull : ((1ull << left) - 1);
                     }
+                    // The softmax warps set the pace of a unit (one row per thread, 64 columns in sequence),
+                    // so the common tile -- every token visible -- does no masking, the scale is folded
+                    // into the exponent's fma, and the exponential is the bare ex2.approx.
+                    if (vis != ~0ull) {
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) {
-                        const float xv = ((vis >> c) & 1ull) ? __uint_as_float(sv[c >> 5][c & 31]) * a.scale_log2
-                                                             : -INFINITY;
-                        sv[c >> 5][c & 31] = __float_as_uint(xv);
-                        mx = fmaxf(mx, xv);
+                        for (int c = 0; c < 64; ++c)
+                            if (!((vis >> c) & 1ull)) sv[c >> 5][c & 31] = 0xff800000u;      // -inf: weight 0
                     }
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sv[c >> 5][c & 31]));
+                    mx *= a.scale_log2;                                  // scale > 0 (checked by the host)
                     // lazy rescale: move the reference only when some row of the warp needs it
                     const bool need = mx > m_ref + 8.f;
                     if (__any_sync(kFull, need)) {
@@ -586,8 +596,8 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        const float p0 = exp2f(__uint_as_float(sv[(2 * c) >> 5][(2 * c) & 31]) - m_use);
-                        const float p1 = exp2f(__uint_as_float(sv[(2 * c + 1) >> 5][(2 * c + 1) & 31]) - m_use);
+                        const float p0 = ex2_ftz(fmaf(__uint_as_float(sv[(2 * c) >> 5][(2 * c) & 31]), a.scale_log2, -m_use));
+                        const float p1 = ex2_ftz(fmaf(__uint_as_float(sv[(2 * c + 1) >> 5][(2 * c + 1) & 31]), a.scale_log2, -m_use));
                         const uint32_t pk = pack_bf16(p0, p1);
                         // the row sum must match what the tensor core will see: the rounded values
                         l_run += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
@@ -979,6 +989,7 @@ LayerDims layer_dims(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, const ds
 bool attention_tc_supported(const dsbd_forest_t *f, const dsbd_attn_desc_t *d, int64_t n_pages) {
     if (d->dtype != DSBD_DTYPE_BF16 || d->d != kD) return false;
     if (d->Hq / d->Hkv > kRows) return false;                                // a node's rows fit one tile
+    if (!(d->scale > 0.f)) return false;                                     // the row maximum is taken before scaling
     if (f->max_tree_nodes * (d->Hq / d->Hkv) > kRows * 8) return false;      // up to 8 row blocks
     if (f->max_tree_nodes > 2 * kBN) return false;                           // two tree tiles
     if (d->total_prefix <= 0) return false;
