@@ -567,8 +567,13 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                         for (int c = 0; c < 64; ++c)
                             if (!((vis >> c) & 1ull)) sv[c >> 5][c & 31] = 0xff800000u;      // -inf: weight 0
                     }
+                    {   // four independent chains: this warp has its scheduler nearly to itself, so a
+                        // 64-long dependent chain would be pure latency
+                        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sv[c >> 5][c & 31]));
+                        for (int c = 0; c < 64; ++c) m4[c & 3] = fmaxf(m4[c & 3], __uint_as_float(sv[c >> 5][c & 31]));
+                        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+                    }
                     mx *= a.scale_log2;                                  // scale > 0 (checked by the host)
                     // lazy rescale: move the reference only when some row of the warp needs it
                     const bool need = mx > m_ref + 8.f;
@@ -594,15 +599,18 @@ k_forest_attn_tc(const __grid_constant__ CUtensorMap map_kp, const __grid_consta
                     }
                     uint32_t pv[32];
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                    float l4[4] = {0.f, 0.f, 0.f, 0.f};                  // (independent chains again)
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
                         const float p0 = ex2_ftz(fmaf(__uint_as_float(sv[(2 * c) >> 5][(2 * c) & 31]), a.scale_log2, -m_use));
                         const float p1 = ex2_ftz(fmaf(__uint_as_float(sv[(2 * c + 1) >> 5][(2 * c + 1) & 31]), a.scale_log2, -m_use));
                         const uint32_t pk = pack_bf16(p0, p1);
                         // the row sum must match what the tensor core will see: the rounded values
-                        l_run += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+                        l4[c & 1] += __uint_as_float(pk << 16);
+                        l4[2 + (c & 1)] += __uint_as_float(pk & 0xffff0000u);
                         pv[c] = pk;
                     }
+                    l_run += (l4[0] + l4[1]) + (l4[2] + l4[3]);
                     tmem_st32(tmem + lane_base + s_col, pv);
                     tmem_wait_st();
                 }
